@@ -1,0 +1,227 @@
+"""CPU oracle for the STWQ quantized linear layer: ctypes front end to stwq_oracle.c.
+
+TEST INFRASTRUCTURE ONLY. Nothing on the product path imports this package; the
+GPU library never calls it and it never imports the GPU library. It is loaded by
+the tests, by the smoke check and by the benchmark's CPU-baseline leg.
+
+All arithmetic lives in stwq_oracle.c (one plain C function per step of the
+method, each citing the passage of the paper it follows). This module only
+compiles that file with gcc and marshals numpy arrays.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "stwq_oracle.c")
+_LIB = os.path.join(_HERE, "libstwq_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with strict IEEE semantics (no contraction, no fast-math)."""
+    if force or (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        cmd = ["gcc", "-O2", "-std=c11", "-D_GNU_SOURCE", "-fopenmp", "-ffp-contract=off",
+               "-fno-fast-math", "-shared", "-fPIC", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _f32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.float32)
+
+
+def _ptr(a, ct):
+    return None if a is None else a.ctypes.data_as(C.POINTER(ct))
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            L = C.CDLL(build())
+            fp, ip, bp, dp = (C.POINTER(C.c_float), C.POINTER(C.c_int32), C.POINTER(C.c_int8),
+                              C.POINTER(C.c_double))
+            L.orc_num_threads.restype = C.c_int
+            L.orc_delta.restype = C.c_float
+            L.orc_delta.argtypes = [C.c_float, C.c_int]
+            L.orc_eq1_quantize.argtypes = [fp, C.c_int64, C.c_float, C.c_float, C.c_int, ip, fp, ip]
+            L.orc_eq1_dequantize.argtypes = [ip, C.c_int64, C.c_float, C.c_int32, fp]
+            L.orc_quantize_div.argtypes = [fp, C.c_int64, C.c_float, C.c_int, bp]
+            L.orc_gps_fold.argtypes = [fp, C.c_int, C.c_int, fp, C.c_int, bp, fp]
+            L.orc_stwq_calibrate.restype = C.c_int
+            L.orc_stwq_calibrate.argtypes = [fp, ip, C.c_int64, C.c_int, C.c_int, fp, C.c_int,
+                                             C.c_uint32, fp]
+            for f in (L.orc_quantize, L.orc_quantize_exact_div):
+                f.restype = C.c_int
+                f.argtypes = [fp, ip, C.c_int64, C.c_int, fp, fp, C.c_int, C.c_int, bp]
+            L.orc_igemm.argtypes = [bp, bp, C.c_int64, C.c_int, C.c_int, ip]
+            L.orc_epilogue.restype = C.c_int
+            L.orc_epilogue.argtypes = [ip, ip, C.c_int64, C.c_int, fp, C.c_int, fp, fp, C.c_int, dp, dp]
+            L.orc_qlinear.restype = C.c_int
+            L.orc_qlinear.argtypes = [fp, ip, C.c_int64, C.c_int, C.c_int, bp, fp, fp, C.c_int, fp, fp,
+                                      C.c_int, C.c_int, dp, bp, ip, dp]
+            L.orc_gps.argtypes = [fp, C.c_int64, C.c_int, fp, C.c_int, C.c_int, C.c_uint32, C.c_int,
+                                  fp, ip]
+            L.orc_gps_gain.restype = C.c_double
+            L.orc_gps_gain.argtypes = [C.c_double] * 4
+            _lib = L
+    return _lib
+
+
+def num_threads() -> int:
+    return int(lib().orc_num_threads())
+
+
+def delta(a: float, bits: int) -> float:
+    """Scale of the symmetric b-bit quantizer with range [-a, a] (Eq. 1)."""
+    return float(lib().orc_delta(np.float32(a), bits))
+
+
+def eq1_quantize(x, x_down, x_up, bits):
+    """Eq. 1 as printed: unsigned codes, scale and zero point."""
+    x = _f32(x).ravel()
+    code = np.empty(x.size, np.int32)
+    d = C.c_float()
+    z = C.c_int32()
+    lib().orc_eq1_quantize(_ptr(x, C.c_float), x.size, np.float32(x_down), np.float32(x_up), bits,
+                           _ptr(code, C.c_int32), C.byref(d), C.byref(z))
+    return code, float(d.value), int(z.value)
+
+
+def eq1_dequantize(code, delta_, z):
+    code = np.ascontiguousarray(code, np.int32).ravel()
+    out = np.empty(code.size, np.float32)
+    lib().orc_eq1_dequantize(_ptr(code, C.c_int32), code.size, np.float32(delta_), int(z),
+                             _ptr(out, C.c_float))
+    return out
+
+
+def quantize_div(x, delta_, bits):
+    """Signed codes clamp(round(x / delta)) of the symmetric quantizer."""
+    x = _f32(x)
+    q = np.empty(x.shape, np.int8)
+    lib().orc_quantize_div(_ptr(x, C.c_float), x.size, np.float32(delta_), bits, _ptr(q, C.c_int8))
+    return q
+
+
+def gps_fold(W, s_ch, bits):
+    """Eq. 2 weight side + per-output-channel quantization. Returns (Wq int8 [N,K], s_w [N])."""
+    W = _f32(W)
+    s_ch = _f32(s_ch)
+    N, K = W.shape
+    Wq = np.empty((N, K), np.int8)
+    s_w = np.empty(N, np.float32)
+    lib().orc_gps_fold(_ptr(W, C.c_float), N, K, _ptr(s_ch, C.c_float), bits, _ptr(Wq, C.c_int8),
+                       _ptr(s_w, C.c_float))
+    return Wq, s_w
+
+
+def stwq_calibrate(X, pos_ids, P, s_ch, bits, pct_ppm):
+    """Section 4.2: per-position static scales by nearest-rank percentile. Returns s_tok [P]."""
+    X = _f32(X)
+    pos_ids = np.ascontiguousarray(pos_ids, np.int32)
+    s_ch = _f32(s_ch)
+    rows, K = X.shape
+    s_tok = np.empty(P, np.float32)
+    st = lib().orc_stwq_calibrate(_ptr(X, C.c_float), _ptr(pos_ids, C.c_int32), rows, K, P,
+                                  _ptr(s_ch, C.c_float), bits, int(pct_ppm), _ptr(s_tok, C.c_float))
+    if st == -1:
+        raise ValueError("pos_ids outside [0, P)")
+    if st == -2:
+        raise ValueError("non-finite calibration value")
+    return s_tok
+
+
+def quantize(X, pos_ids, s_ch, s_tok, bits, exact_div=False):
+    """Activation quantization with static per-position scales. Returns Xq int8 [M,K]."""
+    X = _f32(X)
+    pos_ids = np.ascontiguousarray(pos_ids, np.int32)
+    s_ch = _f32(s_ch)
+    s_tok = _f32(s_tok)
+    M, K = X.shape
+    Xq = np.empty((M, K), np.int8)
+    f = lib().orc_quantize_exact_div if exact_div else lib().orc_quantize
+    st = f(_ptr(X, C.c_float), _ptr(pos_ids, C.c_int32), M, K, _ptr(s_ch, C.c_float),
+           _ptr(s_tok, C.c_float), s_tok.size, bits, _ptr(Xq, C.c_int8))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return Xq
+
+
+def igemm(Xq, Wq):
+    """acc[m,n] = sum_k Xq[m,k] * Wq[n,k] in int32."""
+    Xq = np.ascontiguousarray(Xq, np.int8)
+    Wq = np.ascontiguousarray(Wq, np.int8)
+    M, K = Xq.shape
+    N, K2 = Wq.shape
+    assert K == K2
+    acc = np.empty((M, N), np.int32)
+    lib().orc_igemm(_ptr(Xq, C.c_int8), _ptr(Wq, C.c_int8), M, N, K, _ptr(acc, C.c_int32))
+    return acc
+
+
+def epilogue(acc, pos_ids, s_tok, s_w, bias, act):
+    """Dequantize + bias + activation in double. Returns (Y, mag)."""
+    acc = np.ascontiguousarray(acc, np.int32)
+    pos_ids = np.ascontiguousarray(pos_ids, np.int32)
+    s_tok, s_w, bias = _f32(s_tok), _f32(s_w), _f32(bias)
+    M, N = acc.shape
+    Y = np.empty((M, N), np.float64)
+    mag = np.empty((M, N), np.float64)
+    st = lib().orc_epilogue(_ptr(acc, C.c_int32), _ptr(pos_ids, C.c_int32), M, N, _ptr(s_tok, C.c_float),
+                            s_tok.size, _ptr(s_w, C.c_float), _ptr(bias, C.c_float), act,
+                            _ptr(Y, C.c_double), _ptr(mag, C.c_double))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return Y, mag
+
+
+def qlinear(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act=0):
+    """The whole quantized linear. Returns dict(Y float64, Xq int8, acc int32, mag float64)."""
+    X = _f32(X)
+    pos_ids = np.ascontiguousarray(pos_ids, np.int32)
+    Wq = np.ascontiguousarray(Wq, np.int8)
+    s_w, s_tok, s_ch, bias = _f32(s_w), _f32(s_tok), _f32(s_ch), _f32(bias)
+    M, K = X.shape
+    N = Wq.shape[0]
+    assert Wq.shape[1] == K
+    Y = np.empty((M, N), np.float64)
+    mag = np.empty((M, N), np.float64)
+    Xq = np.empty((M, K), np.int8)
+    acc = np.empty((M, N), np.int32)
+    st = lib().orc_qlinear(_ptr(X, C.c_float), _ptr(pos_ids, C.c_int32), M, K, N, _ptr(Wq, C.c_int8),
+                           _ptr(s_w, C.c_float), _ptr(s_tok, C.c_float), s_tok.size,
+                           _ptr(s_ch, C.c_float), _ptr(bias, C.c_float), bits, act,
+                           _ptr(Y, C.c_double), _ptr(Xq, C.c_int8), _ptr(acc, C.c_int32),
+                           _ptr(mag, C.c_double))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return {"Y": Y, "Xq": Xq, "acc": acc, "mag": mag}
+
+
+def gps(X, W, bits, pct_ppm=999900, variant=0):
+    """Algorithm 1. X [T,K] calibration rows, W [N,K]. Returns (s [K] float32, k_star)."""
+    X = _f32(X)
+    W = _f32(W)
+    T, K = X.shape
+    N = W.shape[0]
+    assert W.shape[1] == K
+    s = np.empty(K, np.float32)
+    ks = C.c_int32()
+    lib().orc_gps(_ptr(X, C.c_float), T, K, _ptr(W, C.c_float), N, bits, int(pct_ppm), variant,
+                  _ptr(s, C.c_float), C.byref(ks))
+    return s, int(ks.value)
+
+
+def gps_gain(A, B, s_k, s_i):
+    """Scaling gain of Eq. 13 / Eq. 15 given A = sum W^2 dX^2 and B = sum dW^2 X^2."""
+    return float(lib().orc_gps_gain(A, B, s_k, s_i))

@@ -1,0 +1,461 @@
+/*
+ * CPU oracle for the static-token-wise-quantized (STWQ) linear layer of PTQ4ARVG.
+ *
+ * TEST INFRASTRUCTURE ONLY. This file is the slow, plain definition of what the
+ * GPU library must compute. It shares no code with the CUDA path and is never on
+ * the product path: only the tests, the smoke check and the benchmark's CPU
+ * baseline leg may load it.
+ *
+ * Every function names the passage of the paper it follows. Where the paper is
+ * silent the reading taken is stated next to the code. Parity status: every
+ * function here is pinned by the CPU tests (closed forms, brute force, textbook
+ * special cases); none is "parity unpinned".
+ *
+ * Layout conventions: X is [rows, K] row-major (K = the paper's n input
+ * channels), W is [N, K] row-major (the transpose of the paper's n x m W, N =
+ * the paper's m output channels), Y is [rows, N] row-major.
+ *
+ * Arithmetic: fp32 where a decision (a code, a scale) is taken, because the
+ * deployed path takes it in fp32; fp64 for the dequantized output. Build with
+ * -O2 -ffp-contract=off and without fast-math so every fp32 operation below is
+ * one IEEE-754 operation in the order written.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* ------------------------------------------------------------------------- */
+/* Code range of a b-bit signed container.                                    */
+static int orc_qmax(int bits) { return (1 << (bits - 1)) - 1; }
+static int orc_qmin(int bits) { return -(1 << (bits - 1)); }
+
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Eq. 1, general (asymmetric) form, exactly as printed:
+ *   delta = (x_up - x_down) / (2^b - 1),  z = round(-x_down / delta),
+ *   code  = clamp(round(x / delta) + z, 0, 2^b - 1),
+ * and the dequantizer of Appendix A.1:  x_hat = delta * (code - z).
+ * round() is round-to-nearest; ties go to even (the paper does not fix the tie
+ * rule; this is the IEEE default and what hardware converts do).
+ * Outputs: codes in [0, 2^b-1] as int32, and (optionally) delta and z.
+ */
+void orc_eq1_quantize(const float* x, int64_t n, float x_down, float x_up, int bits,
+                      int32_t* code, float* delta_out, int32_t* z_out)
+{
+    const float levels = (float)((1 << bits) - 1);
+    float delta = (x_up - x_down) / levels;
+    if (!(delta > 0.0f)) delta = 1.0f;
+    const int32_t z = (int32_t)nearbyintf(-x_down / delta);
+    for (int64_t i = 0; i < n; ++i) {
+        float r = nearbyintf(x[i] / delta) + (float)z;
+        if (r < 0.0f) r = 0.0f;
+        if (r > levels) r = levels;
+        code[i] = (int32_t)r;
+    }
+    if (delta_out) *delta_out = delta;
+    if (z_out) *z_out = z;
+}
+
+void orc_eq1_dequantize(const int32_t* code, int64_t n, float delta, int32_t z, float* x_hat)
+{
+    for (int64_t i = 0; i < n; ++i) x_hat[i] = delta * (float)(code[i] - z);
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Symmetric specialisation of Eq. 1 used by the deployed path: the range is
+ * [-a, a], so R = 2a and delta = 2a / (2^b - 1). The zero point of Eq. 1 is then
+ * round((2^b - 1) / 2) = 2^(b-1); subtracting it from the unsigned code gives a
+ * signed code in [-2^(b-1), 2^(b-1) - 1], i.e. [-128,127] for b = 8 and
+ * [-32,31] for b = 6, and the dequantizer becomes x_hat = delta * code.
+ * Guards (the paper gives none): a == 0 gives delta = 1; delta is floored at
+ * 2^-64 so that its reciprocal is finite.
+ */
+float orc_delta(float a, int bits)
+{
+    const float levels = (float)((1 << bits) - 1);
+    if (!(a > 0.0f)) return 1.0f;
+    float delta = (a + a) / levels;
+    const float floor_ = 5.421010862427522e-20f; /* 2^-64 */
+    if (delta < floor_) delta = floor_;
+    return delta;
+}
+
+/* round-to-nearest-even then clamp to the signed b-bit range; NaN gives 0. */
+static int32_t orc_code(float u, int bits)
+{
+    if (u != u) return 0;
+    float r = nearbyintf(u);
+    const float lo = (float)orc_qmin(bits), hi = (float)orc_qmax(bits);
+    if (r < lo) r = lo;
+    if (r > hi) r = hi;
+    return (int32_t)r;
+}
+
+/* q(x) = clamp(round(x / delta)) with a true division (Eq. 1), signed codes. */
+void orc_quantize_div(const float* x, int64_t n, float delta, int bits, int8_t* q)
+{
+    for (int64_t i = 0; i < n; ++i) q[i] = (int8_t)orc_code(x[i] / delta, bits);
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Equivalent scaling, weight side (Eq. 2: Y = (X / s)(s * W)) followed by
+ * per-output-channel weight quantization (Appendix B: channel-wise weights) with
+ * min-max range calibration (Section 3), in the symmetric form above:
+ *   W'[n,k] = W[n,k] * s_ch[k]        (s_ch == NULL means all ones)
+ *   a_n     = max_k |W'[n,k]|
+ *   s_w[n]  = delta(a_n)
+ *   Wq[n,k] = clamp(round(W'[n,k] / s_w[n]))     (true division)
+ */
+void orc_gps_fold(const float* W, int N, int K, const float* s_ch, int bits,
+                  int8_t* Wq, float* s_w)
+{
+    for (int n = 0; n < N; ++n) {
+        const float* w = W + (int64_t)n * K;
+        float a = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            float v = s_ch ? w[k] * s_ch[k] : w[k];
+            float av = fabsf(v);
+            if (av > a) a = av;
+        }
+        const float d = orc_delta(a, bits);
+        s_w[n] = d;
+        for (int k = 0; k < K; ++k) {
+            float v = s_ch ? w[k] * s_ch[k] : w[k];
+            Wq[(int64_t)n * K + k] = (int8_t)orc_code(v / d, bits);
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * STWQ calibration (Section 4.2): one static quantization range per token
+ * position, set offline by percentile calibration over the calibration samples.
+ * For position p the population is |X[r,k] * rc[k]| over every calibration row r
+ * with pos_ids[r] == p and every channel k, where rc[k] = 1 / s_ch[k] is the
+ * activation side of Eq. 2 (s_ch == NULL: no scaling). The range half-width a_p
+ * is the nearest-rank percentile: with n_p values sorted ascending, the value of
+ * rank ceil(pct * n_p) (1-based), pct given in parts per million; no
+ * interpolation. pct = 100 % is min-max calibration. s_tok[p] = delta(a_p).
+ * A position with no rows gets s_tok = 1.
+ * Returns 0, or -1 if a pos_id is outside [0, P), -2 on a non-finite value.
+ */
+static int orc_cmp_float(const void* a, const void* b)
+{
+    const float fa = *(const float*)a, fb = *(const float*)b;
+    return (fa > fb) - (fa < fb);
+}
+
+int orc_stwq_calibrate(const float* X, const int32_t* pos_ids, int64_t rows, int K, int P,
+                       const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok)
+{
+    int64_t* count = (int64_t*)calloc((size_t)P, sizeof(int64_t));
+    for (int64_t r = 0; r < rows; ++r) {
+        if (pos_ids[r] < 0 || pos_ids[r] >= P) { free(count); return -1; }
+        count[pos_ids[r]] += 1;
+    }
+    float* rc = (float*)malloc(sizeof(float) * (size_t)K);
+    for (int k = 0; k < K; ++k) rc[k] = s_ch ? 1.0f / s_ch[k] : 1.0f;
+
+    int status = 0;
+    for (int p = 0; p < P; ++p) {
+        const int64_t n_p = count[p] * (int64_t)K;
+        if (n_p == 0) { s_tok[p] = 1.0f; continue; }
+        float* v = (float*)malloc(sizeof(float) * (size_t)n_p);
+        int64_t j = 0;
+        for (int64_t r = 0; r < rows; ++r) {
+            if (pos_ids[r] != p) continue;
+            for (int k = 0; k < K; ++k) {
+                const float x = X[r * K + k];
+                const float t = s_ch ? x * rc[k] : x;
+                if (!isfinite(t)) status = -2;
+                v[j++] = fabsf(t);
+            }
+        }
+        qsort(v, (size_t)n_p, sizeof(float), orc_cmp_float);
+        uint64_t rank = ((uint64_t)pct_ppm * (uint64_t)n_p + 999999ull) / 1000000ull;
+        if (rank < 1) rank = 1;
+        if (rank > (uint64_t)n_p) rank = (uint64_t)n_p;
+        s_tok[p] = orc_delta(v[rank - 1], bits);
+        free(v);
+    }
+    free(rc);
+    free(count);
+    return status;
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Step 1 of the quantized linear: activation quantization with the static
+ * per-position scale (Eq. 1 applied to the left factor of Eq. 2, Section 4.2).
+ *   Xq[m,k] = clamp(round( (X[m,k] * rc[k]) * rt[pos[m]] ))
+ * with rc[k] = 1/s_ch[k] and rt[p] = 1/s_tok[p] formed once in fp32. The
+ * deployed path multiplies by reciprocals instead of dividing twice per element;
+ * the product is taken in this order, each multiply rounded to fp32.
+ * NaN gives code 0; +-Inf saturate.
+ * Returns 0, or -1 if a pos_id is outside [0, P).
+ */
+int orc_quantize(const float* X, const int32_t* pos_ids, int64_t M, int K,
+                 const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq)
+{
+    float* rc = (float*)malloc(sizeof(float) * (size_t)K);
+    for (int k = 0; k < K; ++k) rc[k] = s_ch ? 1.0f / s_ch[k] : 1.0f;
+    int status = 0;
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) { status = -1; break; }
+        const float rt = 1.0f / s_tok[p];
+        for (int k = 0; k < K; ++k) {
+            const float x = X[m * K + k];
+            const float t = s_ch ? x * rc[k] : x;
+            const float u = t * rt;
+            Xq[m * K + k] = (int8_t)orc_code(u, bits);
+        }
+    }
+    free(rc);
+    return status;
+}
+
+/*
+ * The same step with two true divisions per element, (x / s_ch[k]) / s_tok[p]:
+ * the literal reading of Eq. 1 and Eq. 2. Information only (how many codes the
+ * reciprocal form moves); not the parity definition.
+ */
+int orc_quantize_exact_div(const float* X, const int32_t* pos_ids, int64_t M, int K,
+                           const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq)
+{
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) return -1;
+        for (int k = 0; k < K; ++k) {
+            const double x = X[m * K + k];
+            const double t = s_ch ? x / (double)s_ch[k] : x;
+            const float u = (float)(t / (double)s_tok[p]);
+            Xq[m * K + k] = (int8_t)orc_code(u, bits);
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Step 2: Y = X W of Section 3 on the integer codes, int32 accumulation:
+ *   acc[m,n] = sum_k Xq[m,k] * Wq[n,k].
+ * |acc| <= K * 2^14, so int32 cannot overflow for K < 131072.
+ */
+void orc_igemm(const int8_t* Xq, const int8_t* Wq, int64_t M, int N, int K, int32_t* acc)
+{
+#pragma omp parallel for schedule(static)
+    for (int64_t m = 0; m < M; ++m) {
+        const int8_t* x = Xq + m * K;
+        for (int n = 0; n < N; ++n) {
+            const int8_t* w = Wq + (int64_t)n * K;
+            int32_t s = 0;
+            for (int k = 0; k < K; ++k) s += (int32_t)x[k] * (int32_t)w[k];
+            acc[m * N + n] = s;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Step 3: dequantization (Appendix A.1, x_hat = delta * code, applied to the
+ * product of two quantized factors), bias, optional GELU; in double.
+ *   z = acc * (s_tok[pos[m]] * s_w[n]) + bias[n]
+ *   act 0: y = z
+ *   act 1: y = z * 0.5 * (1 + erf(z / sqrt 2))                    (GELU, erf form)
+ *   act 2: y = z * 0.5 * (1 + tanh(sqrt(2/pi) (z + 0.044715 z^3))) (GELU, tanh form)
+ * mag (optional) receives |acc * s_tok * s_w| + |bias|, the magnitude the
+ * tolerance of the parity tests is relative to.
+ */
+int orc_epilogue(const int32_t* acc, const int32_t* pos_ids, int64_t M, int N,
+                 const float* s_tok, int P, const float* s_w, const float* bias, int act,
+                 double* Y, double* mag)
+{
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) return -1;
+        const double st = (double)s_tok[p];
+        for (int n = 0; n < N; ++n) {
+            const double prod = (double)acc[m * N + n] * (st * (double)s_w[n]);
+            const double b = bias ? (double)bias[n] : 0.0;
+            const double z = prod + b;
+            double y = z;
+            if (act == 1) y = z * 0.5 * (1.0 + erf(z / sqrt(2.0)));
+            else if (act == 2)
+                y = z * 0.5 * (1.0 + tanh(sqrt(2.0 / M_PI) * (z + 0.044715 * z * z * z)));
+            Y[m * N + n] = y;
+            if (mag) mag[m * N + n] = fabs(prod) + fabs(b);
+        }
+    }
+    return 0;
+}
+
+/*
+ * The whole quantized linear: quantize -> integer GEMM -> dequantize.
+ * Xq_out, acc_out and mag may be NULL. Returns 0 or -1 (bad pos_id).
+ */
+int orc_qlinear(const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
+                const int8_t* Wq, const float* s_w, const float* s_tok, int P,
+                const float* s_ch, const float* bias, int bits, int act,
+                double* Y, int8_t* Xq_out, int32_t* acc_out, double* mag)
+{
+    int8_t* Xq = Xq_out ? Xq_out : (int8_t*)malloc((size_t)(M * K));
+    int32_t* acc = acc_out ? acc_out : (int32_t*)malloc(sizeof(int32_t) * (size_t)(M * N));
+    int st = orc_quantize(X, pos_ids, M, K, s_ch, s_tok, P, bits, Xq);
+    if (st == 0) {
+        orc_igemm(Xq, Wq, M, N, K, acc);
+        st = orc_epilogue(acc, pos_ids, M, N, s_tok, P, s_w, bias, act, Y, mag);
+    }
+    if (!Xq_out) free(Xq);
+    if (!acc_out) free(acc);
+    return st;
+}
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Gain-Projected Scaling, Algorithm 1 (Appendix F), with Eq. 13-16 of Section 4.1.
+ * Inputs: calibration activations X [T, K], weights W [N, K] (paper: n x m,
+ * transposed here), bit width, percentile for the activation range.
+ *
+ * 1. Quantize X per tensor (Step 3 of Section 4.1 assumes per-tensor activation
+ *    quantization; range by percentile calibration) and W per output channel
+ *    (min-max), both with the symmetric quantizer above; dX = X - Q(X),
+ *    dW = W - Q(W).
+ * 2. R_x[k] = max_t X[t,k] - min_t X[t,k]; k* = the channel with the largest
+ *    range (lowest index on ties).
+ * 3. s_k* = sqrt(R_x[k*] / R_w[k*]), where R_w[k*] is the range of the weights
+ *    that multiply channel k* (max_n W[n,k*] - min_n W[n,k*]): the only slice
+ *    that s_k* rescales, so that R_x/s = R_w*s holds after scaling.
+ * 4. For every other channel i (Eq. 16 as printed, variant 0):
+ *      s_i = s_k* * sqrt(sum_t sum_n |dW[n,i] X[t,i]|) / sqrt(sum_t sum_n |W[n,i] dX[t,i]|)
+ *    the sums also running over the calibration rows t (the expectation in
+ *    Eq. 5-6). Variant 1 is the exact stationary point of the gain of Eq. 15:
+ *      s_i = s_k* * (sum dW^2 X^2 / sum W^2 dX^2)^(1/4).
+ *    The two agree when there is one output channel and one row (Eq. 14).
+ * Guards (the paper gives none): a zero numerator, denominator or weight range
+ * gives s_i = 1; s is clamped to [1e-4, 1e4].
+ * k_star_out (optional) receives k*.
+ */
+void orc_gps(const float* X, int64_t T, int K, const float* W, int N, int bits,
+             uint32_t pct_ppm, int variant, float* s, int32_t* k_star_out)
+{
+    /* 1. quantization errors */
+    const int64_t nx = T * (int64_t)K;
+    float* ax = (float*)malloc(sizeof(float) * (size_t)nx);
+    for (int64_t i = 0; i < nx; ++i) ax[i] = fabsf(X[i]);
+    qsort(ax, (size_t)nx, sizeof(float), orc_cmp_float);
+    uint64_t rank = ((uint64_t)pct_ppm * (uint64_t)nx + 999999ull) / 1000000ull;
+    if (rank < 1) rank = 1;
+    if (rank > (uint64_t)nx) rank = (uint64_t)nx;
+    const float dx_scale = orc_delta(ax[rank - 1], bits);
+    free(ax);
+
+    double* dX = (double*)malloc(sizeof(double) * (size_t)nx);
+    for (int64_t i = 0; i < nx; ++i) {
+        const float xhat = dx_scale * (float)orc_code(X[i] / dx_scale, bits);
+        dX[i] = (double)X[i] - (double)xhat;
+    }
+    double* dW = (double*)malloc(sizeof(double) * (size_t)N * (size_t)K);
+    for (int n = 0; n < N; ++n) {
+        float a = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            const float av = fabsf(W[(int64_t)n * K + k]);
+            if (av > a) a = av;
+        }
+        const float d = orc_delta(a, bits);
+        for (int k = 0; k < K; ++k) {
+            const float w = W[(int64_t)n * K + k];
+            const float what = d * (float)orc_code(w / d, bits);
+            dW[(int64_t)n * K + k] = (double)w - (double)what;
+        }
+    }
+
+    /* 2. channel with the largest activation range */
+    int kstar = 0;
+    double best = -1.0;
+    for (int k = 0; k < K; ++k) {
+        double hi = -INFINITY, lo = INFINITY;
+        for (int64_t t = 0; t < T; ++t) {
+            const double v = X[t * K + k];
+            if (v > hi) hi = v;
+            if (v < lo) lo = v;
+        }
+        const double r = hi - lo;
+        if (r > best) { best = r; kstar = k; }
+    }
+
+    /* 3. s_k* equalises the two ranges */
+    double whi = -INFINITY, wlo = INFINITY;
+    for (int n = 0; n < N; ++n) {
+        const double v = W[(int64_t)n * K + kstar];
+        if (v > whi) whi = v;
+        if (v < wlo) wlo = v;
+    }
+    const double rw = whi - wlo;
+    double sk = (rw > 0.0 && best > 0.0) ? sqrt(best / rw) : 1.0;
+
+    /* 4. the remaining channels */
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < K; ++i) {
+        double si;
+        if (i == kstar) {
+            si = sk;
+        } else {
+            double num = 0.0, den = 0.0;
+            for (int64_t t = 0; t < T; ++t) {
+                const double x = X[t * K + i];
+                const double dx = dX[t * K + i];
+                for (int n = 0; n < N; ++n) {
+                    const double w = W[(int64_t)n * K + i];
+                    const double dw = dW[(int64_t)n * K + i];
+                    if (variant == 0) {
+                        num += fabs(dw * x);
+                        den += fabs(w * dx);
+                    } else {
+                        num += (dw * x) * (dw * x);
+                        den += (w * dx) * (w * dx);
+                    }
+                }
+            }
+            if (!(num > 0.0) || !(den > 0.0)) si = 1.0;
+            else if (variant == 0) si = sk * sqrt(num) / sqrt(den);
+            else si = sk * sqrt(sqrt(num / den));
+        }
+        if (si < 1e-4) si = 1e-4;
+        if (si > 1e4) si = 1e4;
+        s[i] = (float)si;
+    }
+    if (k_star_out) *k_star_out = kstar;
+    free(dX);
+    free(dW);
+}
+
+/*
+ * The scaling gain of Eq. 13 / Eq. 15 for one channel i, as a function of a
+ * trial s_i with s_k* fixed; summed over outputs and calibration rows. Used by
+ * the tests to check that the closed form is where this function peaks.
+ *   g(s_i) = 1/2 sum (W^2 dX^2 + dW^2 X^2) - s_i^2/(2 s_k^2) sum W^2 dX^2
+ *            - s_k^2/(2 s_i^2) sum dW^2 X^2
+ * The caller passes the two sums: A = sum W^2 dX^2, B = sum dW^2 X^2.
+ */
+double orc_gps_gain(double A, double B, double s_k, double s_i)
+{
+    return 0.5 * (A + B) - (s_i * s_i) / (2.0 * s_k * s_k) * A
+           - (s_k * s_k) / (2.0 * s_i * s_i) * B;
+}
