@@ -1,0 +1,167 @@
+/*
+ * libstwq - static-token-wise-quantized (STWQ) linear layer for NVIDIA B200 (sm_100a).
+ *
+ * The inference hot path of PTQ4ARVG's quantized decoder, as a C library:
+ *
+ *   offline   stwq_calibrate   per-token-position activation scales      (Section 4.2)
+ *   offline   gps_fold         fold the per-channel scale into W, quantize W (Eq. 2, Appendix B)
+ *   online    stwq_quantize    X -> int8 codes with the static scales     (Eq. 1, Eq. 2, Section 4.2)
+ *   online    qlinear          quantize -> int8 GEMM -> dequantize (+bias, +GELU)
+ *   online    qlinear_q        the same from precomputed codes
+ *
+ * Notation: M rows (tokens x batch), K input channels (the paper's n), N output
+ * channels (the paper's m), P token positions (the paper's T), b in {8, 6} bits,
+ * qmin = -2^(b-1), qmax = 2^(b-1) - 1, D = 2^b - 1.
+ *
+ * Conventions for every call
+ *  - Every pointer is a DEVICE pointer owned by the caller unless it is said to be a host
+ *    pointer. The library never frees or keeps caller memory. Matrices are row-major and
+ *    dense: X [M,K], W and Wq [N,K] (the nn.Linear layout, i.e. the paper's W transposed),
+ *    Y [M,N].
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Calls
+ *    enqueue work and return; they do not synchronise, except where stated.
+ *  - Return value: STWQ_OK (0) or a negative STWQ_ERR_* code. Argument errors are detected
+ *    on the host before anything is enqueued. Errors only the device can see (a pos_id
+ *    outside [0,P), a non-finite calibration value, a device-side wait that ran out) are
+ *    recorded in the context and read with stwq_device_status().
+ *  - A context may be used from one host thread at a time.
+ *  - Alignment: X, Xq, Wq, Y 16-byte aligned; K a multiple of 16.
+ */
+#ifndef STWQ_H
+#define STWQ_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+#if defined(__GNUC__)
+#pragma GCC visibility push(default)   /* the entry points below are the library's only exports */
+#endif
+
+typedef struct stwq_ctx stwq_ctx;
+
+enum {
+    STWQ_OK = 0,
+    STWQ_ERR_NULL = -1,           /* a required pointer is NULL                              */
+    STWQ_ERR_DIM = -2,            /* a size is zero, negative or beyond what is supported    */
+    STWQ_ERR_ALIGN = -3,          /* pointer or K alignment rule violated                    */
+    STWQ_ERR_BITS = -4,           /* bits is not 6 or 8, or act / out_dtype / pct invalid    */
+    STWQ_ERR_ARCH = -5,           /* the device is not compute capability 10.x               */
+    STWQ_ERR_CUDA = -6,           /* a CUDA call failed; see stwq_last_cuda_error()          */
+    STWQ_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired; output is invalid   */
+    STWQ_ERR_POS_RANGE = -8,      /* a pos_id was outside [0,P); that row was written as 0   */
+    STWQ_ERR_NONFINITE = -9,      /* calibration saw NaN or Inf                              */
+    STWQ_ERR_NOMEM = -10          /* workspace allocation failed                             */
+};
+
+/* activation applied by the epilogue */
+enum { STWQ_ACT_NONE = 0, STWQ_ACT_GELU_ERF = 1, STWQ_ACT_GELU_TANH = 2 };
+/* element type of Y. INT32 returns the raw accumulators (no scale, bias or activation). */
+enum { STWQ_OUT_F32 = 0, STWQ_OUT_BF16 = 1, STWQ_OUT_INT32 = 2 };
+
+/*
+ * Create a context on `device` (a CUDA ordinal). Synchronous. Allocates a small status
+ * word and, lazily, workspace (the int8 copy of X used by qlinear, calibration histograms).
+ * Fails with STWQ_ERR_ARCH unless the device is compute capability 10.x.
+ * stwq_destroy frees everything the context allocated; it synchronises the device.
+ */
+int stwq_create(stwq_ctx** out, int device);
+void stwq_destroy(stwq_ctx* ctx);
+
+/*
+ * Pre-size the workspace so that later calls allocate nothing: room for an [M,K] int8
+ * activation copy and for calibration over P positions. Synchronous (may allocate).
+ * Without it the first call that needs more workspace allocates (and synchronises) itself.
+ */
+int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P);
+
+/*
+ * Static token-wise calibration (Section 4.2: one set of quantization parameters per token
+ * position, fixed offline by percentile calibration).
+ * For each position p, over every row r with pos_ids[r] == p and every channel k:
+ *     v = | Xcal[r,k] * (1 / s_ch[k]) |          (fp32; s_ch == NULL means no scaling)
+ *     a_p = the value of rank ceil(pct_ppm * n_p / 1e6) among the n_p values, ascending
+ *           (nearest rank, no interpolation; pct_ppm = 1000000 is min-max calibration)
+ *     s_tok[p] = 2 a_p / D   (fp32 division; 1 if a_p == 0 or no row has position p;
+ *                             floored at 2^-64)
+ * Xcal [rows,K] fp32, pos_ids [rows] int32 in [0,P), s_tok [P] fp32 out.
+ * pct_ppm in 1..1000000. Exact (an order statistic), independent of row order.
+ */
+int stwq_calibrate(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K,
+                   int P, const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok,
+                   void* stream);
+
+/*
+ * Equivalent scaling, weight side (Eq. 2: Y = (X / s)(s * W)), then per-output-channel
+ * min-max weight quantization with the symmetric form of Eq. 1:
+ *     W'[n,k] = W[n,k] * s_ch[k]                  (s_ch == NULL: W' = W)
+ *     a_n = max_k |W'[n,k]|,   s_w[n] = 2 a_n / D  (1 if a_n == 0)
+ *     Wq[n,k] = clamp(round(W'[n,k] / s_w[n]), qmin, qmax)      (IEEE division, ties to even)
+ * W [N,K] fp32 in, Wq [N,K] int8 out, s_w [N] fp32 out.
+ */
+int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
+             float* s_w, void* stream);
+
+/*
+ * Activation quantization with static per-position scales (Eq. 1 on the left factor of
+ * Eq. 2; Section 4.2):
+ *     Xq[m,k] = clamp(round((X[m,k] * rc[k]) * rt[pos_ids[m]]), qmin, qmax)
+ * rc[k] = 1 / s_ch[k] (1 if s_ch == NULL), rt[p] = 1 / s_tok[p], both IEEE fp32; the two
+ * multiplies are rounded separately in this order; ties to even; NaN -> 0, +-Inf saturate.
+ * X [M,K] fp32, pos_ids [M] int32, s_ch [K] or NULL, s_tok [P], Xq [M,K] int8 out.
+ * A row whose pos_id is outside [0,P) is written as zeros and STWQ_ERR_POS_RANGE is recorded.
+ */
+int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
+                  const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream);
+
+/*
+ * The quantized linear layer: stwq_quantize into context workspace, then
+ *     acc[m,n] = sum_k Xq[m,k] * Wq[n,k]                          (int32, exact)
+ *     z = float(acc) * (s_tok[pos_ids[m]] * s_w[n]) + bias[n]     (fp32: one multiply for the
+ *                                                   scale, one fused multiply-add; Appendix A.1)
+ *     Y[m,n] = act(z)  cast to out_dtype
+ * bias == NULL means zero. out_dtype STWQ_OUT_INT32 stores acc itself.
+ * Calls with few rows (M <= 256, the raster-order decode step where a batch advances one
+ * token position at a time) are routed to a bandwidth-bound variant that streams Wq once
+ * across all SMs; the result is the same.
+ * Extra alignment: N a multiple of 8 for bf16 output gives vector stores; other N work but
+ * store element by element.
+ */
+int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
+            const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+            const float* bias, int bits, int act, int out_dtype, void* Y, void* stream);
+
+/* GEMM + epilogue of qlinear from codes the caller already holds (Xq [M,K] int8). */
+int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+              const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
+              int act, int out_dtype, void* Y, void* stream);
+
+/*
+ * Synchronise `stream`, then return and clear the status recorded by device code since the
+ * last call: STWQ_OK, STWQ_ERR_POS_RANGE, STWQ_ERR_NONFINITE or STWQ_ERR_DEVICE_TIMEOUT.
+ */
+int stwq_device_status(stwq_ctx* ctx, void* stream);
+
+/*
+ * Options (for tests and tuning). STWQ_OPT_GEMM_PATH: 0 = choose by shape (default),
+ * 1 = always the tiled tensor-core GEMM, 2 = always the few-row (decode) variant (M <= 256 only).
+ * STWQ_OPT_WAIT_LIMIT_MS: limit of every device-side wait in milliseconds (default 2000).
+ */
+enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2 };
+int stwq_set_option(stwq_ctx* ctx, int option, int value);
+
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t stwq_launch_count(const stwq_ctx* ctx);
+
+/* Text for a status code; the cudaError_t of the last STWQ_ERR_CUDA on this context. */
+const char* stwq_strerror(int status);
+int stwq_last_cuda_error(const stwq_ctx* ctx);
+
+#if defined(__GNUC__)
+#pragma GCC visibility pop
+#endif
+#ifdef __cplusplus
+}
+#endif
+#endif /* STWQ_H */

@@ -1,0 +1,283 @@
+// C ABI of libstwq: context management, argument validation, and the composition of the
+// kernels into the calls declared in stwq.h. No arithmetic of the method lives here.
+#include <cuda.h>
+
+#include <new>
+
+#include "stwq_internal.cuh"
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int check_bits(int bits) { return (bits == 8 || bits == 6) ? STWQ_OK : STWQ_ERR_BITS; }
+
+int ensure_xq(stwq_ctx* ctx, size_t bytes)
+{
+    if (ctx->ws_xq_bytes >= bytes) return STWQ_OK;
+    if (ctx->ws_xq) {
+        cudaError_t e = cudaFree(ctx->ws_xq);           // synchronises
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->ws_xq = nullptr;
+        ctx->ws_xq_bytes = 0;
+    }
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return STWQ_ERR_NOMEM;
+    }
+    ctx->ws_xq = static_cast<int8_t*>(p);
+    ctx->ws_xq_bytes = bytes;
+    return STWQ_OK;
+}
+
+int ensure_cal(stwq_ctx* ctx, int P)
+{
+    const size_t bytes = stwq_calibrate_ws_bytes(P);
+    if (ctx->ws_cal_bytes >= bytes) return STWQ_OK;
+    if (ctx->ws_cal) {
+        cudaError_t e = cudaFree(ctx->ws_cal);
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->ws_cal = nullptr;
+        ctx->ws_cal_bytes = 0;
+    }
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return STWQ_ERR_NOMEM;
+    }
+    ctx->ws_cal = p;
+    ctx->ws_cal_bytes = bytes;
+    return STWQ_OK;
+}
+
+// Make the context's device current for the duration of a call.
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            cudaSetDevice(dev);
+            switched = true;
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+int check_gemm_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
+                    const float* s_w, const float* s_tok, int P, int act, int out_dtype, const void* Y)
+{
+    if (!A || !Wq || !Y) return STWQ_ERR_NULL;
+    if (out_dtype != STWQ_OUT_INT32 && (!pos_ids || !s_w || !s_tok)) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || N <= 0 || P <= 0) return STWQ_ERR_DIM;
+    if (M > (int64_t)0x7fffff00 || K >= 131072) return STWQ_ERR_DIM;   // int32 accumulation bound
+    if ((K & 15) != 0 || !aligned16(A) || !aligned16(Wq) || !aligned16(Y)) return STWQ_ERR_ALIGN;
+    if (act < STWQ_ACT_NONE || act > STWQ_ACT_GELU_TANH) return STWQ_ERR_BITS;
+    if (out_dtype < STWQ_OUT_F32 || out_dtype > STWQ_OUT_INT32) return STWQ_ERR_BITS;
+    return STWQ_OK;
+}
+
+int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+             const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
+             int out_dtype, void* Y, cudaStream_t st)
+{
+    const bool can_decode = M <= 256;
+    bool decode = can_decode;
+    if (ctx->gemm_path == 1) decode = false;
+    if (ctx->gemm_path == 2 && !can_decode) return STWQ_ERR_DIM;
+    if (decode)
+        return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+    return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int stwq_create(stwq_ctx** out, int device)
+{
+    if (!out) return STWQ_ERR_NULL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        (void)cudaGetLastError();
+        return STWQ_ERR_CUDA;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return STWQ_ERR_CUDA;
+    if (prop.major != 10) return STWQ_ERR_ARCH;
+    stwq_ctx* ctx = new (std::nothrow) stwq_ctx();
+    if (!ctx) return STWQ_ERR_NOMEM;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    ctx->l2_bytes = prop.l2CacheSize;
+    ctx->gemm_path = 0;
+    ctx->wait_limit_ms = 2000;
+    DeviceGuard g(device);
+    cudaError_t e = cudaMalloc(reinterpret_cast<void**>(&ctx->d_status), 256);
+    if (e == cudaSuccess) e = cudaMemset(ctx->d_status, 0, 256);
+    if (e != cudaSuccess) {
+        delete ctx;
+        return STWQ_ERR_CUDA;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn) {
+        cudaFree(ctx->d_status);
+        delete ctx;
+        return STWQ_ERR_CUDA;
+    }
+    ctx->encode_tiled = fn;
+    *out = ctx;
+    return STWQ_OK;
+}
+
+void stwq_destroy(stwq_ctx* ctx)
+{
+    if (!ctx) return;
+    DeviceGuard g(ctx->device);
+    cudaDeviceSynchronize();
+    if (ctx->ws_xq) cudaFree(ctx->ws_xq);
+    if (ctx->ws_cal) cudaFree(ctx->ws_cal);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    delete ctx;
+}
+
+int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (M < 0 || K < 0 || P < 0) return STWQ_ERR_DIM;
+    DeviceGuard g(ctx->device);
+    int rc = STWQ_OK;
+    if (M > 0 && K > 0) rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc == STWQ_OK && P > 0) rc = ensure_cal(ctx, P);
+    return rc;
+}
+
+int stwq_set_option(stwq_ctx* ctx, int option, int value)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (option == STWQ_OPT_GEMM_PATH && value >= 0 && value <= 2) {
+        ctx->gemm_path = value;
+        return STWQ_OK;
+    }
+    if (option == STWQ_OPT_WAIT_LIMIT_MS && value >= 1 && value <= 60000) {
+        ctx->wait_limit_ms = value;
+        return STWQ_OK;
+    }
+    return STWQ_ERR_DIM;
+}
+
+int stwq_calibrate(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K, int P,
+                   const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, void* stream)
+{
+    if (!ctx || !Xcal || !pos_ids || !s_tok) return STWQ_ERR_NULL;
+    if (rows <= 0 || K <= 0 || P <= 0 || P > (1 << 20)) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    int rc = ensure_cal(ctx, P);
+    if (rc != STWQ_OK) return rc;
+    return stwq_launch_calibrate(ctx, ctx->ws_cal, Xcal, pos_ids, rows, K, P, s_ch, bits, pct_ppm, s_tok,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
+             float* s_w, void* stream)
+{
+    if (!ctx || !W || !Wq || !s_w) return STWQ_ERR_NULL;
+    if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_fold(ctx, W, N, K, s_ch, bits, Wq, s_w, static_cast<cudaStream_t>(stream));
+}
+
+int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
+                  const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream)
+{
+    if (!ctx || !X || !pos_ids || !s_tok || !Xq) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || P <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if ((K & 15) != 0 || !aligned16(X) || !aligned16(Xq)) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, Xq,
+                                static_cast<cudaStream_t>(stream));
+}
+
+int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+              const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
+              int out_dtype, void* Y, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    DeviceGuard g(ctx->device);
+    return run_gemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
+                    static_cast<cudaStream_t>(stream));
+}
+
+int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
+            const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+            const float* bias, int bits, int act, int out_dtype, void* Y, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (!pos_ids || !s_tok || !s_w) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(X, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc != STWQ_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
+    if (rc != STWQ_OK) return rc;
+    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+}
+
+int stwq_device_status(stwq_ctx* ctx, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint32_t h = 0;
+    cudaError_t e = cudaMemcpyAsync(&h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    if (h & STWQ_DEV_TIMEOUT) return STWQ_ERR_DEVICE_TIMEOUT;
+    if (h & STWQ_DEV_POS_RANGE) return STWQ_ERR_POS_RANGE;
+    if (h & STWQ_DEV_NONFINITE) return STWQ_ERR_NONFINITE;
+    return STWQ_OK;
+}
+
+int64_t stwq_launch_count(const stwq_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int stwq_last_cuda_error(const stwq_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
+
+const char* stwq_strerror(int status)
+{
+    switch (status) {
+        case STWQ_OK: return "ok";
+        case STWQ_ERR_NULL: return "a required pointer is NULL";
+        case STWQ_ERR_DIM: return "a size is out of range";
+        case STWQ_ERR_ALIGN: return "alignment rule violated (16-byte pointers, K multiple of 16)";
+        case STWQ_ERR_BITS: return "unsupported bits / activation / output type / percentile";
+        case STWQ_ERR_ARCH: return "device is not compute capability 10.x";
+        case STWQ_ERR_CUDA: return "a CUDA call failed";
+        case STWQ_ERR_DEVICE_TIMEOUT: return "a device-side wait expired";
+        case STWQ_ERR_POS_RANGE: return "a position id was outside [0, P)";
+        case STWQ_ERR_NONFINITE: return "calibration input contains NaN or Inf";
+        case STWQ_ERR_NOMEM: return "workspace allocation failed";
+        default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,71 @@
+// Internal declarations shared by the translation units of libstwq.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "stwq.h"
+
+// Bits of the device status word (OR-ed by kernels, read by stwq_device_status).
+#define STWQ_DEV_POS_RANGE 1u
+#define STWQ_DEV_NONFINITE 2u
+#define STWQ_DEV_TIMEOUT 4u
+
+struct stwq_ctx {
+    int device;
+    int sm_count;
+    int l2_bytes;
+    int last_cuda_error;
+    int gemm_path;             // STWQ_OPT_GEMM_PATH
+    int wait_limit_ms;         // STWQ_OPT_WAIT_LIMIT_MS
+    int64_t launches;
+    uint64_t configured_mask;  // kernels whose shared-memory attribute is already set
+    uint32_t* d_status;        // device status word
+    int8_t* ws_xq;             // workspace: int8 copy of X for qlinear
+    size_t ws_xq_bytes;
+    void* ws_cal;              // workspace: calibration histograms and selection state
+    size_t ws_cal_bytes;
+    void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
+};
+
+// Launchers (host). Each returns STWQ_OK or STWQ_ERR_CUDA and bumps ctx->launches.
+int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
+                         const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
+                         cudaStream_t st);
+int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
+                     int8_t* Wq, float* s_w, cudaStream_t st);
+size_t stwq_calibrate_ws_bytes(int P);
+int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids,
+                          int64_t rows, int K, int P, const float* s_ch, int bits, uint32_t pct_ppm,
+                          float* s_tok, cudaStream_t st);
+int stwq_launch_qgemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
+                      int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
+                      const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
+int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
+                       int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
+                       const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
+
+static inline int stwq_cuda_fail(stwq_ctx* ctx, cudaError_t e)
+{
+    if (ctx) ctx->last_cuda_error = (int)e;
+    return STWQ_ERR_CUDA;
+}
+
+#ifdef __CUDACC__
+// delta of the symmetric b-bit quantizer with range [-a, a]: 2a / (2^b - 1) in IEEE fp32,
+// 1 for a == 0, floored at 2^-64.
+__device__ __forceinline__ float stwq_delta(float a, int bits)
+{
+    if (!(a > 0.0f)) return 1.0f;
+    const float levels = (float)((1 << bits) - 1);
+    float d = __fdiv_rn(__fadd_rn(a, a), levels);
+    return fmaxf(d, 5.421010862427522e-20f);
+}
+
+// round to nearest even (NaN -> 0, +-Inf and large values saturate), clamp to the b-bit range.
+// Rounding then clamping equals clamping then rounding because the bounds are integers.
+__device__ __forceinline__ int stwq_code(float u, int qmin, int qmax)
+{
+    return max(min(__float2int_rn(u), qmax), qmin);
+}
+#endif

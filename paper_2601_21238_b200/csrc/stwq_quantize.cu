@@ -1,0 +1,101 @@
+// Activation quantization with static per-token-position scales (Eq. 1 applied to the left
+// factor of Eq. 2; Section 4.2):  Xq[m,k] = clamp(round((X[m,k] * rc[k]) * rt[pos[m]])).
+//
+// HBM-bound streaming kernel: 4 bytes in, 1 byte out per element. A warp owns a span of 512
+// consecutive columns; lane l handles the four float4 at columns 4*(32*j + l), j = 0..3, so
+// every warp-wide load is one contiguous 512-byte request and every warp-wide store one
+// contiguous 128-byte request. The span of a warp never changes, so the 16 reciprocal channel
+// scales a lane needs stay in registers for the whole kernel; the per-row reciprocal token scale
+// is one IEEE division per row and warp.
+#include "stwq_internal.cuh"
+
+namespace {
+
+constexpr int kSpan = 512;          // columns per warp and row
+constexpr int kThreads = 256;
+
+__device__ __forceinline__ float4 ld_stream(const float* p)
+{
+    float4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+__global__ void __launch_bounds__(kThreads)
+quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
+                const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin,
+                int qmax, int8_t* __restrict__ Xq, int spans, int64_t row_stride,
+                uint32_t* __restrict__ status)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int span = (int)(warp % spans);
+    int64_t m = warp / spans;
+    const int col0 = span * kSpan + lane * 4;
+
+    // reciprocal channel scales of this lane's 16 columns (1 where there is no scaling)
+    float rc[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int c = col0 + j * 128;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
+    }
+
+    for (; m < M; m += row_stride) {
+        const int p = pos_ids[m];
+        const bool ok = (p >= 0) && (p < P);
+        const float rt = ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
+        if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+        const float* xrow = X + m * K;
+        int8_t* qrow = Xq + m * K;
+        float4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = col0 + j * 128;
+            if (c < K) v[j] = ld_stream(xrow + c);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = col0 + j * 128;
+            if (c < K) {
+                int q0 = stwq_code(__fmul_rn(__fmul_rn(v[j].x, rc[j * 4 + 0]), rt), qmin, qmax);
+                int q1 = stwq_code(__fmul_rn(__fmul_rn(v[j].y, rc[j * 4 + 1]), rt), qmin, qmax);
+                int q2 = stwq_code(__fmul_rn(__fmul_rn(v[j].z, rc[j * 4 + 2]), rt), qmin, qmax);
+                int q3 = stwq_code(__fmul_rn(__fmul_rn(v[j].w, rc[j * 4 + 3]), rt), qmin, qmax);
+                if (!ok) q0 = q1 = q2 = q3 = 0;
+                const uint32_t packed = (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) |
+                                        ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+                *reinterpret_cast<uint32_t*>(qrow + c) = packed;
+            }
+        }
+    }
+}
+
+}  // namespace
+
+int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
+                         const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
+                         cudaStream_t st)
+{
+    const int spans = (K + kSpan - 1) / kSpan;
+    const int warps_per_block = kThreads / 32;
+    // enough warps for every SM to hold 8 blocks, rounded so that each warp keeps one span
+    int64_t want_warps = (int64_t)ctx->sm_count * 8 * warps_per_block;
+    int64_t rows_in_flight = want_warps / spans;
+    if (rows_in_flight < 1) rows_in_flight = 1;
+    if (rows_in_flight > M) rows_in_flight = M;
+    // total warps must be rows_in_flight * spans and a multiple of warps_per_block
+    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    const int64_t blocks = rows_in_flight * spans / warps_per_block;
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    quantize_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(X, pos_ids, M, K, s_ch, s_tok, P, qmin,
+                                                           qmax, Xq, spans, rows_in_flight,
+                                                           ctx->d_status);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
