@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the STWQ quantized linear hot path on B200.
+
+A step is one pass of the whole hot path (activation quantize -> int8 GEMM -> dequantize
+epilogue, i.e. one `qlinear` call) over each of the four block linears of the VAR-d16-shaped
+workload (batch 16 x 680 tokens, hidden 1024: qkv, proj, fc1+GELU, fc2; W8A8, bf16 output),
+on seeded synthetic inputs already resident in HBM. The metric is int8 TOPS of the whole step
+(2*M*N*K per layer over the step time, quantize kernels included).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config 2]
+
+Prints one JSON line (rank 0). With N > 1 (torchrun) every rank runs the same per-GPU batch on
+its own rows (weak scaling, no collective on the data path); time is the max over ranks.
+`--impl reference` times the CPU oracle on the host cores instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+PCT = 999900
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+INT8_OVER_BF16 = 2.0          # nominal dense tensor ratio (4.5 vs 2.25 PFLOP/s)
+# DRAM bytes (read + write) per launch of the dominant kernel from the ncu capture summarised in
+# profiles/; None until a capture of this workload exists.
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        d["_source"] = "measured"
+        return d
+    d = dict(FALLBACK_PEAKS)
+    d["_source"] = "fallback"
+    return d
+
+
+def stand_in_channel_scales(layer: wl.Layer) -> np.ndarray:
+    """Seeded stand-in for the offline GPS vector (the benchmark's GPU arm may not run the CPU
+    oracle that computes it): larger on the outlier channels, log-normal jitter elsewhere."""
+    z = wl.normals(layer.seed, 8, 0, layer.K)
+    return (np.sqrt(wl.outlier_factors(layer)) * np.exp(0.25 * z)).astype(np.float32)
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.idx}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, smax, reasons, power = [], [], set(), []
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+                power.append(float(f[3]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                               f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------ GPU arm
+def setup_layers(ctx, torch, dev, layers, calib_samples):
+    """Offline part, on the GPU: fold + quantize weights, calibrate per-position scales; then the
+    step's activations (drawn on the device)."""
+    T = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    out = []
+    for L in layers:
+        W = T(wl.weights(L))
+        s_ch = T(stand_in_channel_scales(L)) if L.use_gps else None
+        Wq = torch.empty((L.N, L.K), dtype=torch.int8, device=dev)
+        s_w = torch.empty(L.N, device=dev)
+        ctx.gps_fold(W, s_ch, L.bits, Wq, s_w)
+        Xc, pc = wl.calibration(L, calib_samples)
+        s_tok = torch.empty(L.P, device=dev)
+        Xc_d, pc_d = T(Xc), T(pc)
+        ctx.stwq_calibrate(Xc_d, pc_d, L.P, s_ch, L.bits, PCT, s_tok)
+        X, pos = wl.activations_device(L, dev)
+        ydt = {"bf16": torch.bfloat16, "fp32": torch.float32}[L.out_dtype]
+        Y = torch.empty((L.M, L.N), dtype=ydt, device=dev)
+        Xq = torch.empty((L.M, L.K), dtype=torch.int8, device=dev)
+        torch.cuda.synchronize()
+        del W, Xc_d, pc_d
+        out.append(dict(L=L, Wq=Wq, s_w=s_w, s_ch=s_ch, s_tok=s_tok, bias=T(wl.bias(L)), X=X, pos=pos, Y=Y,
+                        Xq=Xq, out_code=1 if L.out_dtype == "bf16" else 0))
+    ctx.check_device_status()
+    return out
+
+
+def run_step(ctx, S):
+    for s in S:
+        L = s["L"]
+        ctx.qlinear(s["X"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["s_ch"], s["bias"], L.bits, L.act,
+                    s["out_code"], s["Y"])
+
+
+def gpu_arm(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2601_21238_b200 as pk
+    from paper_2601_21238_b200 import build as pkbuild
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path for the product arm")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if rank == 0:
+        pkbuild.build()
+    if world > 1:
+        dist.barrier()
+    ctx = pk.Context(local)
+    layers = wl.config_layers(args.config)
+    S = setup_layers(ctx, torch, dev, layers, args.calib_samples)
+    ops_step = sum(L.ops for L in layers)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if world == 1:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing: K whole steps --------------------------------------------
+    for _ in range(args.warmup):
+        run_step(ctx, S)
+    sampler = ClockSampler(local)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    launches0 = ctx.stwq_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        run_step(ctx, S)
+    e1.record()
+    barrier()
+    launches = ctx.stwq_launch_count() - launches0
+    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    clocks = sampler.stop() if rank == 0 else None
+    ctx.check_device_status()
+    ms_step = ms_total / args.steps
+    value = world * ops_step / (ms_step * 1e-3) / 1e12
+
+    # ---- per-kernel timing on the same stream: quantize and GEMM+epilogue separately --------
+    def time_calls(fn):
+        evs = []
+        for _ in range(args.steps):
+            for s in S:
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn(s)
+                b.record()
+                evs.append((s["L"].name, a, b))
+        torch.cuda.synchronize()
+        acc = {}
+        for name, a, b in evs:
+            acc.setdefault(name, []).append(a.elapsed_time(b))
+        return {k: sum(v) / len(v) for k, v in acc.items()}
+
+    tq = time_calls(lambda s: ctx.stwq_quantize(s["X"], s["pos"], s["s_ch"], s["s_tok"], s["L"].bits, s["Xq"]))
+    tg = time_calls(lambda s: ctx.qlinear_q(s["Xq"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["bias"],
+                                            s["L"].act, s["out_code"], s["Y"]))
+    peaks = measured_peaks()
+    per_layer = []
+    for s in S:
+        L = s["L"]
+        qbytes = 5.0 * L.M * L.K
+        per_layer.append({"layer": L.name, "M": L.M, "K": L.K, "N": L.N,
+                          "gemm_ms": round(tg[L.name], 5), "gemm_tops": round(L.ops / tg[L.name] / 1e9, 1),
+                          "quantize_ms": round(tq[L.name], 5),
+                          "quantize_gbs": round(qbytes / tq[L.name] / 1e6, 1)})
+    gemm_ms = sum(tg.values())
+    achieved = ops_step / (gemm_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+    roofline = {"kernel": "qgemm_kernel (tcgen05 kind::i8 GEMM + dequant epilogue)", "bound": "tensor",
+                "achieved": round(achieved, 1), "peak": round(peak, 1), "unit": "TOP/s",
+                "frac": round(achieved / peak, 4),
+                "peak_source": f"2 x bf16_tflops of {peaks['_source']} peaks (burst)",
+                "avg_launch_ms": round(gemm_ms / len(S), 5), "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH,
+                "quantize": {"bound": "hbm", "achieved": round(sum(5.0 * s["L"].M * s["L"].K for s in S)
+                                                                / (sum(tq.values()) * 1e-3) / 1e9, 1),
+                             "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                             "frac": round(sum(5.0 * s["L"].M * s["L"].K for s in S)
+                                           / (sum(tq.values()) * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}}
+
+    # ---- end to end: pinned host X -> device -> qlinear -> device -> pinned host Y ------------
+    hX = [torch.empty((s["L"].M, s["L"].K), dtype=torch.float32).pin_memory() for s in S]
+    hY = [torch.empty_like(s["Y"], device="cpu").pin_memory() for s in S]
+    for h, s in zip(hX, S):
+        h.copy_(s["X"])
+    torch.cuda.synchronize()
+    h2d = sum(h.numel() * h.element_size() for h in hX)
+    d2h = sum(h.numel() * h.element_size() for h in hY)
+
+    def e2e_step():
+        for s, hx, hy in zip(S, hX, hY):
+            L = s["L"]
+            s["X"].copy_(hx, non_blocking=True)
+            ctx.qlinear(s["X"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["s_ch"], s["bias"], L.bits, L.act,
+                        s["out_code"], s["Y"])
+            hy.copy_(s["Y"], non_blocking=True)
+
+    for _ in range(min(args.warmup, 3)):
+        e2e_step()
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        e2e_step()
+    e1.record()
+    barrier()
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
+    e2e = {"value": round(world * ops_step / (e2e_ms * 1e-3) / 1e12, 3), "unit": "TOPS",
+           "ms_per_step": round(e2e_ms, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+    ctx.check_device_status()
+
+    line = {"metric": "qlinear int8 TOPS (quantize + int8 GEMM + dequant epilogue, whole step)",
+            "value": round(value, 2), "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(ms_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": f"config {args.config}: " + ", ".join(
+                           f"{L.name} {L.K}->{L.N}" for L in layers) + f"; M={layers[0].M} per GPU, W8A8, "
+                           f"{layers[0].out_dtype} out",
+                       "l2": "inputs larger than L2 (one step touches ~0.6 GB per GPU)",
+                       "s_ch": "seeded stand-in for the GPS vector on qkv/fc1", "calib_samples": args.calib_samples},
+            "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "layers": per_layer,
+            "pct_of_nominal_int8_peak": round(100 * achieved / 4500.0, 2)}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(S, layers, torch, rows=args.cpu_rows)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------ CPU oracle
+def cpu_baseline(S, layers, torch, rows):
+    """The oracle's qlinear on the host cores over the first `rows` rows of every layer."""
+    import oracle
+    total_ops, total_s = 0.0, 0.0
+    for s in S:
+        L = s["L"]
+        r = min(rows, L.M)
+        X = s["X"][:r].cpu().numpy()
+        pos = s["pos"][:r].cpu().numpy()
+        args = (X, pos, s["Wq"].cpu().numpy(), s["s_w"].cpu().numpy(), s["s_tok"].cpu().numpy(),
+                None if s["s_ch"] is None else s["s_ch"].cpu().numpy(), s["bias"].cpu().numpy(), L.bits, L.act)
+        t0 = time.perf_counter()
+        oracle.qlinear(*args)
+        total_s += time.perf_counter() - t0
+        total_ops += 2.0 * r * L.N * L.K
+    return {"value": round(total_ops / total_s / 1e12, 5), "unit": "TOPS", "cores": oracle.num_threads(),
+            "kind": "oracle", "seconds": round(total_s, 2),
+            "sample": f"first {rows} rows of each of the {len(S)} layers, all output columns"}
+
+
+def reference_arm(args):
+    """The CPU oracle as the reference implementation: same metric, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    layers = wl.config_layers(args.config)
+    rows = args.ref_rows
+    prepared = []
+    for L in layers:
+        W = wl.weights(L)
+        s_ch = stand_in_channel_scales(L) if L.use_gps else None
+        Wq, s_w = oracle.gps_fold(W, s_ch, L.bits)
+        Xc, pc = wl.calibration(L, 2)
+        s_tok = oracle.stwq_calibrate(Xc, pc, L.P, s_ch, L.bits, PCT)
+        X = wl.activations(L, rows=slice(0, rows))
+        pos = wl.positions(L)[:rows]
+        prepared.append((L, X, pos, Wq, s_w, s_tok, s_ch, wl.bias(L)))
+    ops = sum(2.0 * rows * L.N * L.K for L in layers)
+
+    def step():
+        for L, X, pos, Wq, s_w, s_tok, s_ch, b in prepared:
+            oracle.qlinear(X, pos, Wq, s_w, s_tok, s_ch, b, L.bits, L.act)
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / args.steps
+    v = round(ops / dt / 1e12, 5)
+    sample = f"first {rows} rows of each layer per step, all output columns"
+    line = {"impl": "reference", "metric": "qlinear int8 TOPS (quantize + int8 GEMM + dequant epilogue, whole step)",
+            "value": v, "unit": "TOPS", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": {"workload": f"config {args.config} (CPU oracle, {sample})"},
+            "cpu_baseline": {"value": v, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": v, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload family 1..5 (default: VAR-d16 block)")
+    ap.add_argument("--calib-samples", type=int, default=32)
+    ap.add_argument("--cpu-rows", type=int, default=4096)
+    ap.add_argument("--ref-rows", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        gpu_arm(args)
+
+
+if __name__ == "__main__":
+    main()

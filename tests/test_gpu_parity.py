@@ -1,0 +1,332 @@
+"""GPU-vs-oracle parity through the C ABI. Integer results (codes, scales chosen by an order
+statistic, int32 accumulators) must be bit-exact; floating-point outputs within
+|y - y_ref| <= rtol * (|y_ref| + |acc*s_tok*s_w| + |bias|), rtol = 1e-5 (fp32) / 1e-2 (bf16).
+"""
+import numpy as np
+import pytest
+
+import oracle
+import workloads as wl
+from layer_setup import PCT, assert_close, prepare, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+RTOL = {"fp32": 1e-5, "bf16": 1e-2}
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    import paper_2601_21238_b200 as pk
+    from paper_2601_21238_b200 import binding as B
+    from paper_2601_21238_b200 import build as pkbuild
+    pkbuild.build()
+    ctx = pk.Context(0)
+    dev = torch.device("cuda:0")
+
+    class G:
+        pass
+    g = G()
+    g.torch, g.ctx, g.dev, g.B = torch, ctx, dev, B
+    g.T = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    yield g
+    ctx.close()
+
+
+rng = np.random.default_rng(7)
+
+
+def _out_tensor(g, M, N, out):
+    dt = {"fp32": g.torch.float32, "bf16": g.torch.bfloat16, "int32": g.torch.int32}[out]
+    return g.torch.full((M, N), -3, dtype=dt, device=g.dev)
+
+
+def _out_code(g, out):
+    return {"fp32": g.B.OUT_F32, "bf16": g.B.OUT_BF16, "int32": g.B.OUT_INT32}[out]
+
+
+# ----------------------------------------------------------------------------- quantize
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(1, 16, 1), (7, 48, 3), (300, 1040, 11), (64, 1920, 64), (513, 512, 680),
+                                   (40, 5120, 5), (1000, 16, 2)])
+def test_quantize_codes_bit_exact(gpu, bits, shape):
+    M, K, P = shape
+    X = (rng.standard_normal((M, K)) * 3).astype(np.float32)
+    pos = rng.integers(0, P, M).astype(np.int32)            # shuffled positions
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    s_tok = rng.uniform(0.01, 0.1, P).astype(np.float32)
+    X.flat[:4] = [np.nan, np.inf, -np.inf, 1e30]            # NaN -> 0, Inf and huge saturate
+    if M > 2:
+        X[1] = 0.0                                          # all-zero row
+        X[2] = 1e4                                          # saturating row
+    for sc in (s_ch, None):
+        ref = oracle.quantize(X, pos, sc, s_tok, bits)
+        Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+        gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
+        assert gpu.ctx.stwq_device_status() == 0
+        np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
+
+
+def test_quantize_reports_bad_position_and_zeroes_the_row(gpu):
+    M, K, P = 20, 64, 4
+    X = rng.standard_normal((M, K)).astype(np.float32)
+    pos = rng.integers(0, P, M).astype(np.int32)
+    pos[5], pos[11] = P, -1
+    s_tok = rng.uniform(0.01, 0.1, P).astype(np.float32)
+    Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+    gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), None, gpu.T(s_tok), 8, Xq)
+    assert gpu.ctx.stwq_device_status() == -8               # STWQ_ERR_POS_RANGE
+    assert gpu.ctx.stwq_device_status() == 0                # reading clears it
+    got = Xq.cpu().numpy()
+    assert not got[5].any() and not got[11].any()
+    good = np.ones(M, bool)
+    good[[5, 11]] = False
+    np.testing.assert_array_equal(got[good], oracle.quantize(X[good], pos[good], None, s_tok, 8))
+
+
+def test_host_argument_validation(gpu):
+    L, h = gpu.ctx.lib, gpu.ctx.handle
+    X = gpu.torch.zeros((4, 32), device=gpu.dev)
+    pos = gpu.torch.zeros(4, dtype=gpu.torch.int32, device=gpu.dev)
+    s_tok = gpu.torch.ones(1, device=gpu.dev)
+    Xq = gpu.torch.zeros((4, 32), dtype=gpu.torch.int8, device=gpu.dev)
+    p = lambda t: t.data_ptr()
+    assert L.stwq_quantize(h, p(X), p(pos), 4, 32, None, p(s_tok), 1, 7, p(Xq), None) == -4    # bits
+    assert L.stwq_quantize(h, p(X), p(pos), 4, 24, None, p(s_tok), 1, 8, p(Xq), None) == -3    # K % 16
+    assert L.stwq_quantize(h, p(X) + 4, p(pos), 4, 16, None, p(s_tok), 1, 8, p(Xq), None) == -3
+    assert L.stwq_quantize(h, p(X), p(pos), 0, 32, None, p(s_tok), 1, 8, p(Xq), None) == -2    # M
+    assert L.stwq_quantize(h, None, p(pos), 4, 32, None, p(s_tok), 1, 8, p(Xq), None) == -1
+    assert L.stwq_calibrate(h, p(X), p(pos), 4, 32, 1, None, 8, 0, p(s_tok), None) == -4       # pct
+    assert L.stwq_set_option(h, 99, 0) == -2
+    assert gpu.ctx.stwq_device_status() == 0
+
+
+# ----------------------------------------------------------------------------- gps_fold
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(1, 16), (70, 208), (256, 1024), (33, 7680)])
+def test_gps_fold_bit_exact(gpu, bits, shape):
+    N, K = shape
+    W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    W[N // 2] = 0.0                                         # dead output channel -> s_w = 1
+    s_ch = rng.uniform(0.3, 4, K).astype(np.float32)
+    for sc in (s_ch, None):
+        Wq_r, sw_r = oracle.gps_fold(W, sc, bits)
+        Wq = gpu.torch.full((N, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+        sw = gpu.torch.zeros(N, device=gpu.dev)
+        gpu.ctx.gps_fold(gpu.T(W), gpu.T(sc), bits, Wq, sw)
+        np.testing.assert_array_equal(sw.cpu().numpy(), sw_r)
+        np.testing.assert_array_equal(Wq.cpu().numpy(), Wq_r)
+
+
+# ----------------------------------------------------------------------------- stwq_calibrate
+@pytest.mark.parametrize("pct", [1000000, PCT, 990000, 500000, 1])
+def test_calibrate_bit_exact(gpu, pct):
+    S, P, K = 6, 9, 112
+    pos = np.tile(np.arange(P, dtype=np.int32), S)
+    X = (rng.standard_normal((S * P, K)) * (1 + pos[:, None])).astype(np.float32)
+    X[3] = 0.0
+    perm = rng.permutation(S * P)                           # row order must not matter
+    X, pos = X[perm], pos[perm]
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    for bits in (8, 6):
+        for sc in (s_ch, None):
+            ref = oracle.stwq_calibrate(X, pos, P + 2, sc, bits, pct)   # two positions never seen
+            out = gpu.torch.zeros(P + 2, device=gpu.dev)
+            gpu.ctx.stwq_calibrate(gpu.T(X), gpu.T(pos), P + 2, gpu.T(sc), bits, pct, out)
+            assert gpu.ctx.stwq_device_status() == 0
+            np.testing.assert_array_equal(out.cpu().numpy(), ref)
+
+
+def test_calibrate_config1_full_size(gpu):
+    L = wl.config_layers(1)[0]
+    par = prepare(L)
+    out = gpu.torch.zeros(L.P, device=gpu.dev)
+    gpu.ctx.stwq_calibrate(gpu.T(par["Xc"]), gpu.T(par["pc"]), L.P, gpu.T(par["s_ch"]), 8, PCT, out)
+    assert gpu.ctx.stwq_device_status() == 0
+    np.testing.assert_array_equal(out.cpu().numpy(), par["s_tok"])
+    # 16 calibration rows of one sink-like position scaled up: only that position's scale moves
+    Xs = par["Xc"].copy()
+    Xs[par["pc"] == 0] *= 64
+    out2 = gpu.torch.zeros(L.P, device=gpu.dev)
+    gpu.ctx.stwq_calibrate(gpu.T(Xs), gpu.T(par["pc"]), L.P, gpu.T(par["s_ch"]), 8, PCT, out2)
+    o2 = out2.cpu().numpy()
+    np.testing.assert_array_equal(o2[1:], par["s_tok"][1:])
+    assert o2[0] == par["s_tok"][0] * 64
+
+
+def test_calibrate_flags_nonfinite_and_bad_positions(gpu):
+    X = rng.standard_normal((12, 32)).astype(np.float32)
+    pos = (np.arange(12) % 3).astype(np.int32)
+    out = gpu.torch.zeros(3, device=gpu.dev)
+    Xb = X.copy()
+    Xb[4, 4] = np.inf
+    gpu.ctx.stwq_calibrate(gpu.T(Xb), gpu.T(pos), 3, None, 8, PCT, out)
+    assert gpu.ctx.stwq_device_status() == -9
+    pb = pos.copy()
+    pb[0] = 3
+    gpu.ctx.stwq_calibrate(gpu.T(X), gpu.T(pb), 3, None, 8, PCT, out)
+    assert gpu.ctx.stwq_device_status() == -8
+
+
+# ----------------------------------------------------------------------------- GEMM accumulators
+GEMM_SHAPES = [(1, 16, 16), (128, 256, 128), (128, 128, 2048), (129, 257, 16), (300, 520, 144), (77, 8, 48),
+               (256, 512, 384), (640, 1000, 1008), (1000, 136, 8192), (257, 3072, 1024), (2000, 1920, 1920)]
+
+
+@pytest.mark.parametrize("path", [1, 0])
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+def test_int32_accumulators_bit_exact(gpu, shape, path):
+    M, N, K = shape
+    Xq = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    Wq = rng.integers(-128, 128, (N, K)).astype(np.int8)
+    Xq[0], Wq[0] = -128, -128                              # extreme accumulator K * 2^14
+    ref = oracle.igemm(Xq, Wq)
+    Y = _out_tensor(gpu, M, N, "int32")
+    gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, path)
+    try:
+        gpu.ctx.qlinear_q(gpu.T(Xq), None, gpu.T(Wq), None, None, None, 0, gpu.B.OUT_INT32, Y)
+        assert gpu.ctx.stwq_device_status() == 0
+    finally:
+        gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
+    np.testing.assert_array_equal(Y.cpu().numpy(), ref)
+
+
+def test_repeat_runs_are_bitwise_identical(gpu):
+    M, N, K = 900, 1024, 2048
+    Xq = gpu.T(rng.integers(-128, 128, (M, K)).astype(np.int8))
+    Wq = gpu.T(rng.integers(-128, 128, (N, K)).astype(np.int8))
+    a, b = _out_tensor(gpu, M, N, "int32"), _out_tensor(gpu, M, N, "int32")
+    gpu.ctx.qlinear_q(Xq, None, Wq, None, None, None, 0, gpu.B.OUT_INT32, a)
+    gpu.ctx.qlinear_q(Xq, None, Wq, None, None, None, 0, gpu.B.OUT_INT32, b)
+    assert gpu.torch.equal(a, b)
+
+
+# ----------------------------------------------------------------------------- whole qlinear
+def _run_qlinear(gpu, L, par, X, pos, out, act=None, path=0):
+    M = X.shape[0]
+    Y = _out_tensor(gpu, M, L.N, out)
+    gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, path)
+    try:
+        gpu.ctx.qlinear(gpu.T(X) if isinstance(X, np.ndarray) else X, gpu.T(pos) if isinstance(pos, np.ndarray) else pos,
+                        gpu.T(par["Wq"]), gpu.T(par["s_w"]), gpu.T(par["s_tok"]), gpu.T(par["s_ch"]),
+                        gpu.T(par["bias"]), L.bits, L.act if act is None else act, _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+    finally:
+        gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
+    return Y.float().cpu().numpy() if out != "int32" else Y.cpu().numpy()
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("out", ["fp32", "bf16"])
+def test_qlinear_small_ragged(gpu, bits, act, out):
+    """Several tiles with ragged M, N and K tails; every activation and output type."""
+    L = wl.scaled(wl.config_layers(1)[0], K=400, N=328, P=37, batch=9, bits=bits, act=act)
+    par = prepare(L, samples=8, gps_n=64)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], bits, act)
+    acc = _run_qlinear(gpu, L, par, X, pos, "int32")
+    np.testing.assert_array_equal(acc, ref["acc"])
+    assert_close(_run_qlinear(gpu, L, par, X, pos, out), ref, RTOL[out], f"b{bits} act{act} {out}")
+    # without bias and without channel scale
+    par2 = dict(par, bias=None)
+    ref2 = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], None, bits, act)
+    assert_close(_run_qlinear(gpu, L, par2, X, pos, out), ref2, RTOL[out], "no bias")
+
+
+@pytest.mark.parametrize("out", ["fp32", "bf16"])
+def test_config1_full(gpu, out):
+    """Config 1: one W8A8 linear over the 680-token VAR pyramid, K = N = 1024, every element."""
+    L = wl.config_layers(1)[0]
+    par = prepare(L)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 0)
+    # the offline calls reproduce the oracle's parameters bit for bit
+    Wq = gpu.torch.zeros((L.N, L.K), dtype=gpu.torch.int8, device=gpu.dev)
+    sw = gpu.torch.zeros(L.N, device=gpu.dev)
+    gpu.ctx.gps_fold(gpu.T(par["W"]), gpu.T(par["s_ch"]), 8, Wq, sw)
+    np.testing.assert_array_equal(Wq.cpu().numpy(), par["Wq"])
+    np.testing.assert_array_equal(sw.cpu().numpy(), par["s_w"])
+    Xq = gpu.torch.zeros((L.M, L.K), dtype=gpu.torch.int8, device=gpu.dev)
+    gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), gpu.T(par["s_ch"]), gpu.T(par["s_tok"]), 8, Xq)
+    np.testing.assert_array_equal(Xq.cpu().numpy(), ref["Xq"])
+    np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32"), ref["acc"])
+    assert_close(_run_qlinear(gpu, L, par, X, pos, out), ref, RTOL[out], "config 1")
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config2_full(gpu, idx):
+    """Config 2 (VAR-d16 block, batch 16 x 680 tokens): every element of every layer, in the
+    launch configuration the benchmark times (bf16 output, fused GELU on fc1)."""
+    L = wl.config_layers(2)[idx]
+    par = prepare(L, samples=8)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, L.act)
+    np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32"), ref["acc"])
+    assert_close(_run_qlinear(gpu, L, par, X, pos, "bf16"), ref, RTOL["bf16"], L.name)
+    assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32"), ref, RTOL["fp32"], L.name)
+
+
+def _sampled_full_size(gpu, L, samples=4):
+    """Full-size layer drawn on the device; the oracle recomputes a sample of rows (all columns)."""
+    par = prepare(L, samples=samples, gps_n=96)
+    Xd, posd = wl.activations_device(L, gpu.dev)
+    rows = sample_rows(L.M)
+    rt = gpu.torch.from_numpy(rows).to(gpu.dev)
+    Xs, ps = Xd[rt].cpu().numpy(), posd[rt].cpu().numpy()
+    ref = oracle.qlinear(Xs, ps, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], L.bits, L.act)
+    for out in ("int32", "bf16"):
+        M = L.M
+        Y = _out_tensor(gpu, M, L.N, out)
+        gpu.ctx.qlinear(Xd, posd, gpu.T(par["Wq"]), gpu.T(par["s_w"]), gpu.T(par["s_tok"]), gpu.T(par["s_ch"]),
+                        gpu.T(par["bias"]), L.bits, L.act, _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+        got = Y[rt]
+        if out == "int32":
+            np.testing.assert_array_equal(got.cpu().numpy(), ref["acc"])
+        else:
+            assert_close(got.float().cpu().numpy(), ref, RTOL["bf16"], f"cfg{L.config} {L.name} b{L.bits}")
+        del Y
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("idx", [0, 1, 2, 3])
+def test_config3_sampled(gpu, idx, bits):
+    """Config 3 (VAR-d30 block, batch 32 x 680, hidden 1920), W8A8 and W6A6, full size on the GPU."""
+    _sampled_full_size(gpu, wl.config_layers(3, bits=bits)[idx])
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config5_sampled(gpu, idx, bits):
+    """Config 5 (MAR-Huge prefill, M = 65536, hidden 1280), W6A6 and W8A8, full size on the GPU."""
+    _sampled_full_size(gpu, wl.config_layers(5, bits=bits)[idx])
+
+
+@pytest.mark.parametrize("path", [0, 1])
+@pytest.mark.parametrize("idx", [0, 1])
+def test_config4_decode_full(gpu, idx, path):
+    """Config 4 (raster-order decode step): 256 rows that share one token position."""
+    L = wl.config_layers(4)[idx]
+    par = prepare(L, samples=4, gps_n=64)
+    for step in (0, 1):
+        X, pos = wl.activations(L, step), wl.positions(L, step)
+        assert len(set(pos.tolist())) == 1
+        ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 0)
+        np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", path=path), ref["acc"])
+        assert_close(_run_qlinear(gpu, L, par, X, pos, "bf16", path=path), ref, RTOL["bf16"], L.name)
+        assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32", path=path), ref, RTOL["fp32"], L.name)
+
+
+def test_decode_rows_with_mixed_positions_and_few_rows(gpu):
+    """The few-row path makes no assumption that positions are shared; also M = 1 and M = 37."""
+    L = wl.scaled(wl.config_layers(4)[0], K=512, N=1024, P=16)
+    par = prepare(L, samples=4, gps_n=64)
+    for M in (1, 37, 256):
+        X = wl.activations(L)[:M]
+        pos = rng.integers(0, L.P, M).astype(np.int32)
+        ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 1)
+        for path in (0, 2):
+            np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", act=1, path=path), ref["acc"])
+            assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32", act=1, path=path), ref, RTOL["fp32"], "decode")
