@@ -145,7 +145,9 @@ int stwq_device_status(stwq_ctx* ctx, void* stream);
 
 /*
  * Options (for tests and tuning). STWQ_OPT_GEMM_PATH: 0 = choose by shape (default),
- * 1 = always the tiled tensor-core GEMM, 2 = always the few-row (decode) variant (M <= 256 only).
+ * 1 = always a tiled tensor-core GEMM, 2 = always the few-row (decode) variant (M <= 256 only),
+ * 3 = always the single-CTA tiled GEMM (the fallback used when N or the s_w / bias pointers
+ * do not meet the 16-byte rules of the CTA-pair kernel).
  * STWQ_OPT_WAIT_LIMIT_MS: limit of every device-side wait in milliseconds (default 2000).
  */
 enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2 };

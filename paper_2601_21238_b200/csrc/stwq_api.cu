@@ -91,10 +91,12 @@ int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M,
 {
     const bool can_decode = M <= 256;
     bool decode = can_decode;
-    if (ctx->gemm_path == 1) decode = false;
+    if (ctx->gemm_path == 1 || ctx->gemm_path == 3) decode = false;
     if (ctx->gemm_path == 2 && !can_decode) return STWQ_ERR_DIM;
     if (decode)
         return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+    if (ctx->gemm_path != 3 && stwq_qgemm2_supported(N, out_dtype, s_w, bias))
+        return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
     return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
 }
 
@@ -166,7 +168,7 @@ int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P)
 int stwq_set_option(stwq_ctx* ctx, int option, int value)
 {
     if (!ctx) return STWQ_ERR_NULL;
-    if (option == STWQ_OPT_GEMM_PATH && value >= 0 && value <= 2) {
+    if (option == STWQ_OPT_GEMM_PATH && value >= 0 && value <= 3) {
         ctx->gemm_path = value;
         return STWQ_OK;
     }
@@ -174,6 +176,8 @@ int stwq_set_option(stwq_ctx* ctx, int option, int value)
         ctx->wait_limit_ms = value;
         return STWQ_OK;
     }
+    if (option == 100) { ctx->force_bn = value; return STWQ_OK; }   // undocumented tuning knobs
+    if (option == 101) { ctx->debug = value; return STWQ_OK; }
     return STWQ_ERR_DIM;
 }
 

@@ -19,6 +19,9 @@ struct stwq_ctx {
     int gemm_path;             // STWQ_OPT_GEMM_PATH
     int wait_limit_ms;         // STWQ_OPT_WAIT_LIMIT_MS
     int64_t launches;
+    int force_bn;              // tuning: 0 = choose, 128 / 256 = force the tile width
+    int debug;                 // tuning: see Gemm2Params::debug
+    int max_pairs;             // CTA pairs of the pair GEMM that can be resident at once (0 = not yet queried)
     uint64_t configured_mask;  // kernels whose shared-memory attribute is already set
     uint32_t* d_status;        // device status word
     int8_t* ws_xq;             // workspace: int8 copy of X for qlinear
@@ -41,6 +44,10 @@ int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int3
 int stwq_launch_qgemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                       int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                       const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
+bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* bias);
+int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
+                       int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
+                       const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);

@@ -1,0 +1,512 @@
+// qgemm2: the main int8 GEMM + dequantize epilogue, as CTA pairs (tcgen05 cta_group::2).
+//
+//   acc[m,n] = sum_k Xq[m,k] * Wq[n,k]                              (Section 3, Y = X W on codes)
+//   Y[m,n]   = act( float(acc) * (s_tok[pos[m]] * s_w[n]) + bias[n] )   (Appendix A.1 dequantizer)
+//
+// A cluster of two CTAs (two SMs) owns a 256 x BN output tile. Each CTA loads its own 128 rows
+// of Xq and its own half (BN/2 rows) of the Wq slice with TMA; one thread of the even CTA issues
+// tcgen05.mma.cta_group::2 (M = 256, N = BN, K = 32), which reads both CTAs' shared memory, so
+// every byte of Wq is staged once per pair instead of once per SM. Each CTA's tensor memory holds
+// the accumulator rows of its own 128 rows, in two buffers of BN columns so that the next tile's
+// main loop runs while this tile drains.
+//
+// Roles per CTA (kThreads = 64 + 32 * EPI threads):
+//   warp 0          TMA producer (one lane): ring of STAGES stages; completion bytes of both CTAs
+//                   land on the even CTA's "full" barrier
+//   warp 1          MMA issuer (one lane, even CTA only); tcgen05.commit multicasts "stage free"
+//                   and "accumulator full" to both CTAs
+//   warps 2..2+EPI  epilogue: tcgen05.ld -> fp32 scale/bias/GELU -> convert -> 128-byte-swizzled
+//                   staging tile in shared memory -> TMA store (full-line writes, clipped at the
+//                   matrix edge by the tensor map). Warp w may read TMEM lanes 32*(w%4)..+31; with
+//                   EPI = 8 two warps share a lane quarter and alternate column chunks.
+// Every mbarrier wait is bounded (limit in ns from the host); on expiry the CTA raises
+// STWQ_DEV_TIMEOUT, all roles leave their loops, loads in flight are awaited with the same
+// bound, both CTAs meet at the cluster barrier, tensor memory is freed and the kernel returns.
+#include "stwq_internal.cuh"
+#include "stwq_ptx.cuh"
+
+using namespace stwq_ptx;
+
+namespace {
+
+constexpr int kBM = 128;      // rows per CTA
+constexpr int kBK = 128;      // bytes of K per stage
+
+struct Gemm2Params {
+    int64_t M;
+    int N, K, P;
+    const int32_t* pos_ids;
+    const float* s_w;
+    const float* s_tok;
+    const float* bias;
+    int tiles_n, num_tiles, num_kb;
+    uint32_t* status;
+    unsigned long long wait_limit_ns;
+    int debug;                 // tuning only: 1 = skip the output stores, 2 = skip the whole epilogue body
+};
+
+__device__ __forceinline__ uint32_t cluster_ctarank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+// TMA load whose completion bytes are credited to a barrier that may live in the peer CTA.
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                                 uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                               uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Arrive (once all MMAs issued so far have completed) on the barrier at this offset in both CTAs.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar)
+{
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int c0, int c1)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_read1() { asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&b);
+}
+
+template <int BN, int STAGES, int EPI>
+struct Smem2 {
+    static constexpr int kABytes = kBM * kBK;               // 16 KB
+    static constexpr int kBBytes = (BN / 2) * kBK;          // this CTA's half of the Wq slice
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kOffB = STAGES * kABytes;
+    static constexpr int kOffStage = STAGES * kStageBytes;  // per epilogue warp: two staging tiles of 32 rows x 128 B
+    static constexpr int kOffScale = kOffStage + EPI * 8192; // per epilogue warp: s_w and bias of its columns
+    static constexpr int kOffBars = kOffScale + 2 * BN * 4 * 4;
+    static constexpr int kNumBars = 2 * STAGES + 4;
+    static constexpr int kOffMisc = kOffBars + kNumBars * 8;
+    static constexpr int kTotal = kOffMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+    static_assert(kDynamic <= 227 * 1024, "shared memory budget");
+};
+
+// ---------------------------------------------------------------------------- kernel
+// OUT: element type of Y (STWQ_OUT_*); ACT: activation. One staging chunk is 32 rows x 128 bytes:
+// 64 bf16 columns or 32 fp32 / int32 columns.
+template <int BN, int STAGES, int EPI, int OUT, int ACT>
+__global__ void __launch_bounds__(64 + 32 * EPI, 1)
+qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const __grid_constant__ CUtensorMap tmY, const Gemm2Params p)
+{
+    using L = Smem2<BN, STAGES, EPI>;
+    constexpr int kChunkCols = (OUT == STWQ_OUT_BF16) ? 64 : 32;
+    constexpr int kChunks = BN / kChunkCols;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+
+    const uint32_t bars = base + L::kOffBars;
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (STAGES + s); };
+    auto bar_tfull = [&](int a) { return bars + 8u * (2 * STAGES + a); };
+    auto bar_tempty = [&](int a) { return bars + 8u * (2 * STAGES + 2 + a); };
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::kOffMisc + 4);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = even CTA = MMA leader
+    const int pair = blockIdx.x >> 1;
+    const int num_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_full(s), 1);                   // leader's producer arrives with expect_tx
+            mbar_init(bar_empty(s), 1);                  // multicast commit
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(bar_tfull(a), 1);                  // multicast commit
+            mbar_init(bar_tempty(a), 2 * EPI);           // every epilogue warp of both CTAs
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(2 * BN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                  // barriers of both CTAs are initialised
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const unsigned long long limit = p.wait_limit_ns;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            const uint32_t full0 = mapa_u32(bar_full(0), 0);     // leader's barriers
+            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+                const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
+                const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
+                    if (rank == 0) mbar_expect_tx(bar_full(s), 2 * L::kStageBytes);
+                    tma_load_2d_pair(base + s * L::kABytes, &tmA, kb * kBK, m0, full0 + 8u * s);
+                    tma_load_2d_pair(base + L::kOffB + s * L::kBBytes, &tmB, kb * kBK, n0, full0 + 8u * s);
+                }
+            }
+            if (!ok && rank == 0) {
+                const uint32_t first = it > (uint32_t)STAGES ? it - STAGES : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar_full(j % STAGES), (j / STAGES) & 1u))
+                        if (globaltimer_ns() - t0 > limit) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(2 * kBM, BN);
+            uint32_t it = 0, t = 0;
+            bool ok = true;
+            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs, ++t) {
+                const int acc = t & 1;
+                const uint32_t aph = (t >> 1) & 1u;
+                if (!mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                    const int s = it % STAGES;
+                    const uint32_t ph = (it / STAGES) & 1u;
+                    if (!mbar_wait(bar_full(s), ph, abort_flag, limit)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t a_desc = make_smem_desc(base + s * L::kABytes);
+                    const uint64_t b_desc = make_smem_desc(base + L::kOffB + s * L::kBBytes);
+#pragma unroll
+                    for (int k = 0; k < kBK / 32; ++k)
+                        tc_mma_i8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc_commit_pair(bar_empty(s));
+                }
+                if (ok) tc_commit_pair(bar_tfull(acc));
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - 2;                          // 0..EPI-1
+        const int q = warp & 3;                           // TMEM lane quarter
+        const int sub = ew >> 2;                          // which of the EPI/4 warps of this quarter
+        constexpr int kSubs = EPI / 4;
+        constexpr int kMyChunks = kChunks / kSubs;        // column chunks this warp owns per tile
+        constexpr int kMyCols = kMyChunks * kChunkCols;
+        static_assert(kChunks % kSubs == 0, "chunks must divide among the warps of a quarter");
+        const uint32_t stage0 = base + L::kOffStage + (uint32_t)ew * 8192u;   // two staging tiles
+        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 2 * kMyCols;
+        float* my_bias = my_sw + kMyCols;
+        const uint32_t tempty0 = mapa_u32(bar_tempty(0), 0);
+        uint32_t t = 0, nstore = 0;
+        bool ok = true;
+        for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++t) {
+            const int acc = t & 1;
+            const uint32_t aph = (t >> 1) & 1u;
+            const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
+            const int n0 = (tile % p.tiles_n) * BN;
+            const int64_t row = (int64_t)m0 + q * 32 + lane;
+            float st = 0.0f;
+            if (OUT != STWQ_OUT_INT32) {
+                // column scales and biases of this warp's chunks -> its private shared copy, and
+                // the row scale, all fetched before the accumulator is waited for
+                __syncwarp();
+                for (int i = lane * 4; i < kMyCols; i += 128) {
+                    const int k = i / kChunkCols;
+                    const int col = n0 + (sub + k * kSubs) * kChunkCols + (i % kChunkCols);
+                    float4 sw = make_float4(0.f, 0.f, 0.f, 0.f), bi = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (col < p.N) {                      // N is a multiple of 4: the float4 is in range
+                        sw = __ldg(reinterpret_cast<const float4*>(p.s_w + col));
+                        if (p.bias != nullptr) bi = __ldg(reinterpret_cast<const float4*>(p.bias + col));
+                    }
+                    *reinterpret_cast<float4*>(my_sw + i) = sw;
+                    *reinterpret_cast<float4*>(my_bias + i) = bi;
+                }
+                if (row < p.M) {
+                    const int pos = p.pos_ids[row];
+                    if (pos >= 0 && pos < p.P) st = p.s_tok[pos];
+                    else atomicOr(p.status, STWQ_DEV_POS_RANGE);
+                }
+                __syncwarp();
+            }
+            if (ok) ok = mbar_wait(bar_tfull(acc), aph, abort_flag, limit);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
+#pragma unroll 1
+            for (int k = 0; k < kMyChunks && p.debug != 2; ++k, ++nstore) {
+                const int c = sub + k * kSubs;
+                const int col0 = n0 + c * kChunkCols;
+                const uint32_t stage_tile = stage0 + (nstore & 1u) * 4096u;
+                const uint32_t my_row_addr = stage_tile + (uint32_t)lane * 128u;
+                const float* csw = my_sw + k * kChunkCols;
+                const float* cbi = my_bias + k * kChunkCols;
+                __syncwarp();                             // lane 0 issued the previous store: reconverge
+                if (OUT == STWQ_OUT_BF16) {
+                    uint32_t r0[32], r1[32];
+                    tmem_ld32(taddr + (uint32_t)(c * 64), r0);
+                    tmem_ld32(taddr + (uint32_t)(c * 64 + 32), r1);
+                    // the store that last used this staging tile (two stores ago) must have been read
+                    if (lane == 0) bulk_wait_read1();
+                    __syncwarp();                         // reconverge: the wait below is warp-aligned
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const uint32_t* r = h == 0 ? r0 : r1;
+                            const float4 sw = *reinterpret_cast<const float4*>(csw + h * 32 + j);
+                            const float4 bi = *reinterpret_cast<const float4*>(cbi + h * 32 + j);
+                            const float v0 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 0], __fmul_rn(st, sw.x), bi.x));
+                            const float v1 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 1], __fmul_rn(st, sw.y), bi.y));
+                            const float v2 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 2], __fmul_rn(st, sw.z), bi.z));
+                            const float v3 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 3], __fmul_rn(st, sw.w), bi.w));
+                            w[j / 2] = pack_bf16(v0, v1);
+                            w[j / 2 + 1] = pack_bf16(v2, v3);
+                        }
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {     // four 16-byte pieces, swizzled by row
+                            const uint32_t piece = (uint32_t)((h * 4 + g) ^ (lane & 7));
+                            st_shared_v4(my_row_addr + piece * 16u, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                        }
+                    }
+                } else {
+                    uint32_t r[32];
+                    tmem_ld32(taddr + (uint32_t)(c * 32), r);
+                    if (lane == 0) bulk_wait_read1();
+                    __syncwarp();                         // reconverge: the wait below is warp-aligned
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        uint32_t o0, o1, o2, o3;
+                        if (OUT == STWQ_OUT_INT32) {
+                            o0 = r[j]; o1 = r[j + 1]; o2 = r[j + 2]; o3 = r[j + 3];
+                        } else {
+                            const float4 sw = *reinterpret_cast<const float4*>(csw + j);
+                            const float4 bi = *reinterpret_cast<const float4*>(cbi + j);
+                            o0 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 0], __fmul_rn(st, sw.x), bi.x)));
+                            o1 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 1], __fmul_rn(st, sw.y), bi.y)));
+                            o2 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 2], __fmul_rn(st, sw.z), bi.z)));
+                            o3 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 3], __fmul_rn(st, sw.w), bi.w)));
+                        }
+                        const uint32_t piece = (uint32_t)((j / 4) ^ (lane & 7));
+                        st_shared_v4(my_row_addr + piece * 16u, o0, o1, o2, o3);
+                    }
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    if (col0 < p.N && (int64_t)m0 + q * 32 < p.M && p.debug == 0)
+                        tma_store_2d(&tmY, stage_tile, col0, m0 + q * 32);
+                    bulk_commit();    // one group per chunk, even an empty one: wait_group.read 1 counts groups
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
+        }
+        if (lane == 0) bulk_wait0();                       // stores complete before the CTA may exit
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, STWQ_DEV_TIMEOUT);
+    cluster_sync_all();                                  // no remote arrive or multicast still to land
+    tc_fence_after();
+    if (warp == 2) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(2 * BN) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+int encode_2d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* ptr,
+              int64_t rows, int64_t cols, int box_cols, int box_rows)
+{
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+    cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    cuuint64_t gstride[1] = {(cuuint64_t)cols * (cuuint64_t)elem_bytes};
+    cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, dt, 2, const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = (int)r;
+        return STWQ_ERR_CUDA;
+    }
+    return STWQ_OK;
+}
+
+template <int BN, int STAGES, int EPI, int OUT, int ACT>
+int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                   const Gemm2Params& p, cudaStream_t st)
+{
+    using L = Smem2<BN, STAGES, EPI>;
+    auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT>;
+    const uint64_t bit = 1ull << (32 + (BN == 256 ? 0 : 12) + OUT * 4 + ACT);
+    if (!(ctx->configured_mask & bit)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->configured_mask |= bit;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.blockDim = dim3(64 + 32 * EPI, 1, 1);
+    cfg.dynamicSmemBytes = L::kDynamic;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    // Persistent kernel with a static tile stride: launch exactly as many CTA pairs as can be
+    // resident at once (pairs must sit in one GPC, so this can be fewer than SMs / 2).
+    if (ctx->max_pairs <= 0) {
+        cfg.gridDim = dim3((unsigned)(ctx->sm_count & ~1), 1, 1);
+        int n = 0;
+        cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kern, &cfg);
+        if (e != cudaSuccess || n <= 0) return stwq_cuda_fail(ctx, e == cudaSuccess ? cudaErrorLaunchOutOfResources : e);
+        ctx->max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
+    }
+    int pairs = ctx->max_pairs;
+    if (p.num_tiles < pairs) pairs = p.num_tiles;
+    cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
+    ctx->launches += 1;
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+template <int BN, int STAGES, int EPI>
+int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+              const Gemm2Params& p, int act, int out_dtype, cudaStream_t st)
+{
+#define STWQ_CASE(O, A) \
+    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A>(ctx, tmA, tmB, tmY, p, st);
+    if (out_dtype == STWQ_OUT_INT32)
+        return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE>(ctx, tmA, tmB, tmY, p, st);
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+#undef STWQ_CASE
+    return STWQ_ERR_BITS;
+}
+
+}  // namespace
+
+// True if the pair kernel can run this problem: TMA needs 16-byte row pitches for Y and the
+// epilogue reads s_w / bias as aligned float4.
+bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* bias)
+{
+    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : 4;
+    if (((int64_t)N * elem) % 16 != 0) return false;
+    if (out_dtype != STWQ_OUT_INT32) {
+        if ((reinterpret_cast<uintptr_t>(s_w) & 15u) != 0) return false;
+        if (bias != nullptr && (reinterpret_cast<uintptr_t>(bias) & 15u) != 0) return false;
+    }
+    return true;
+}
+
+int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+                       const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
+                       int act, int out_dtype, void* Y, cudaStream_t st)
+{
+    // 256-wide tiles whenever N has more than 128 columns: a 128-wide tile needs 1.5x the
+    // L2 -> shared-memory bytes per multiply-accumulate and is bound by that feed.
+    const int tiles_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
+    int bn = N > 128 ? 256 : 128;
+    if (ctx->force_bn == 128 || ctx->force_bn == 256) bn = ctx->force_bn;
+
+    Gemm2Params p;
+    p.debug = ctx->debug;
+    p.M = M; p.N = N; p.K = K; p.P = P;
+    p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
+    p.tiles_n = (N + bn - 1) / bn;
+    p.num_tiles = tiles_m * p.tiles_n;
+    p.num_kb = (K + kBK - 1) / kBK;
+    p.status = ctx->d_status;
+    p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
+
+    CUtensorMap tmA, tmB, tmY;
+    int rc = encode_2d(ctx, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kBK, kBM);
+    if (rc != STWQ_OK) return rc;
+    rc = encode_2d(ctx, &tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, N, K, kBK, bn / 2);
+    if (rc != STWQ_OK) return rc;
+    if (out_dtype == STWQ_OUT_BF16)
+        rc = encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, M, N, 64, 32);
+    else if (out_dtype == STWQ_OUT_F32)
+        rc = encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Y, M, N, 32, 32);
+    else
+        rc = encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
+    if (rc != STWQ_OK) return rc;
+    if (bn == 256) return launch_bn<256, 4, 8>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    return launch_bn<128, 6, 8>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+}

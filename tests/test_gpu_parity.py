@@ -174,7 +174,7 @@ GEMM_SHAPES = [(1, 16, 16), (128, 256, 128), (128, 128, 2048), (129, 257, 16), (
                (256, 512, 384), (640, 1000, 1008), (1000, 136, 8192), (257, 3072, 1024), (2000, 1920, 1920)]
 
 
-@pytest.mark.parametrize("path", [1, 0])
+@pytest.mark.parametrize("path", [1, 3, 0])      # CTA-pair GEMM, single-CTA GEMM, automatic choice
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
 def test_int32_accumulators_bit_exact(gpu, shape, path):
     M, N, K = shape
@@ -229,6 +229,7 @@ def test_qlinear_small_ragged(gpu, bits, act, out):
     acc = _run_qlinear(gpu, L, par, X, pos, "int32")
     np.testing.assert_array_equal(acc, ref["acc"])
     assert_close(_run_qlinear(gpu, L, par, X, pos, out), ref, RTOL[out], f"b{bits} act{act} {out}")
+    assert_close(_run_qlinear(gpu, L, par, X, pos, out, path=3), ref, RTOL[out], "single-CTA kernel")
     # without bias and without channel scale
     par2 = dict(par, bias=None)
     ref2 = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], None, bits, act)
