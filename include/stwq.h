@@ -138,6 +138,33 @@ int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M
               int act, int out_dtype, void* Y, void* stream);
 
 /*
+ * qlinear without any allocation. (The paper has no counterpart to this call; it exists for the
+ * way the library gets embedded.) qlinear needs a context, whose creation allocates, and keeps
+ * the int8 copy of X in workspace that may be (re)allocated during a call. Hosts that cannot
+ * reach an allocator at that point - a loop with a hard latency budget, a process whose device
+ * memory is wholly owned by another runtime's pool, a deployment that forbids allocation after
+ * start-up - call this instead. It takes no context, runs on the CURRENT device, and computes
+ * exactly what qlinear computes (tiled tensor-core GEMM for every M), with the int8 copy of X
+ * held in a fixed array of STWQ_STATIC_MAX_CODES bytes that is part of the library image on
+ * every GPU that loads it (4 MiB + 256 bytes per GPU until the process exits).
+ *  - M * K must not exceed STWQ_STATIC_MAX_CODES; larger problems return STWQ_ERR_DIM and
+ *    nothing is enqueued. All other argument rules are those of qlinear.
+ *  - The first call on each device looks up the array's device address and the driver entry
+ *    point for tensor maps (no allocation, but several runtime queries): make that call once
+ *    during start-up, before any stream capture begins on that device.
+ *  - All calls on a device share the one array, which keeps the codes of the last call. Two
+ *    calls whose kernels can overlap on the GPU (different streams without an ordering between
+ *    them) race on it; order them. Nothing in it needs clearing between calls: each call
+ *    overwrites the M * K bytes it later reads.
+ *  - Device-side conditions (a pos_id outside [0,P) - that row is computed as zeros - or an
+ *    expired device wait) are not reported by this call.
+ */
+#define STWQ_STATIC_MAX_CODES (4 * 1024 * 1024)
+int qlinear_static(const float* X, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
+                   const float* s_w, const float* s_tok, int P, const float* s_ch, const float* bias,
+                   int bits, int act, int out_dtype, void* Y, void* stream);
+
+/*
  * Synchronise `stream`, then return and clear the status recorded by device code since the
  * last call: STWQ_OK, STWQ_ERR_POS_RANGE, STWQ_ERR_NONFINITE or STWQ_ERR_DEVICE_TIMEOUT.
  */

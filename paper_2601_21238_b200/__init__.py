@@ -5,7 +5,7 @@ raises if libstwq.so has not been built (`python -m paper_2601_21238_b200.build`
 sm_100 GPU is present. There is no CPU fallback.
 """
 from .binding import (ACT_GELU_ERF, ACT_GELU_TANH, ACT_NONE, OUT_BF16, OUT_F32, OUT_INT32, Context,
-                      StwqError, exported_symbols, library_path, load_library)
+                      StwqError, exported_symbols, library_path, load_library, qlinear_static)
 
-__all__ = ["Context", "StwqError", "load_library", "library_path", "exported_symbols", "ACT_NONE",
+__all__ = ["Context", "StwqError", "load_library", "library_path", "exported_symbols", "qlinear_static", "ACT_NONE",
            "ACT_GELU_ERF", "ACT_GELU_TANH", "OUT_F32", "OUT_BF16", "OUT_INT32"]

@@ -16,10 +16,11 @@ _LIB_PATH = os.path.join(_HERE, "libstwq.so")
 ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH = 0, 1, 2
 OUT_F32, OUT_BF16, OUT_INT32 = 0, 1, 2
 OPT_GEMM_PATH, OPT_WAIT_LIMIT_MS = 1, 2
+STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
-            "stwq_strerror", "stwq_last_cuda_error"]
+            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static"]
 
 _lib = None
 
@@ -59,6 +60,7 @@ def load_library():
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
+    L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.stwq_device_status.argtypes = [vp, vp]
     L.stwq_set_option.argtypes = [vp, i32, i32]
     L.stwq_launch_count.argtypes = [vp]
@@ -74,6 +76,22 @@ def load_library():
 
 def _p(t):
     return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def qlinear_static(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
+    """The context-free, allocation-free entry point: same arguments as Context.qlinear, runs on
+    the tensors' device (made current for the call), scratch limited to STATIC_MAX_CODES codes."""
+    import torch
+    L = load_library()
+    M, K = X.shape
+    N = Wq.shape[0]
+    with torch.cuda.device(X.device):
+        if stream is None:
+            stream = torch.cuda.current_stream(X.device)
+        rc = L.qlinear_static(_p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok), s_tok.numel(),
+                              _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y), C.c_void_p(stream.cuda_stream))
+    if rc != 0:
+        raise StwqError(rc, "qlinear_static", L.stwq_strerror(rc).decode())
 
 
 class Context:
