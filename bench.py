@@ -57,6 +57,29 @@ def stand_in_channel_scales(layer: wl.Layer) -> np.ndarray:
     return (np.sqrt(wl.outlier_factors(layer)) * np.exp(0.25 * z)).astype(np.float32)
 
 
+def rank_step(rank: int, step: int = 0, world: int = 1) -> int:
+    """Which seeded batch a rank draws: the job's global batch is `world` per-GPU batches, rank r
+    takes the r-th one (weak scaling: rows are independent, parameters are replicated, so no
+    collective touches the data path)."""
+    return step * world + rank
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Slowest rank's time (all-reduce MAX of one scalar; the only collective of the benchmark)."""
+    if world == 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tops(world: int, ops_per_rank_step: float, ms_step: float) -> float:
+    """Aggregate int8 TOPS of the job: every rank performs ops_per_rank_step in the slowest rank's time."""
+    return world * ops_per_rank_step / (ms_step * 1e-3) / 1e12
+
+
 class ClockSampler:
     """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
     Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -105,7 +128,7 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------ GPU arm
-def setup_layers(ctx, torch, dev, layers, calib_samples):
+def setup_layers(ctx, torch, dev, layers, calib_samples, rank=0, world=1):
     """Offline part, on the GPU: fold + quantize weights, calibrate per-position scales; then the
     step's activations (drawn on the device)."""
     T = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev)
@@ -120,7 +143,7 @@ def setup_layers(ctx, torch, dev, layers, calib_samples):
         s_tok = torch.empty(L.P, device=dev)
         Xc_d, pc_d = T(Xc), T(pc)
         ctx.stwq_calibrate(Xc_d, pc_d, L.P, s_ch, L.bits, PCT, s_tok)
-        X, pos = wl.activations_device(L, dev)
+        X, pos = wl.activations_device(L, dev, step=rank_step(rank, 0, world))
         ydt = {"bf16": torch.bfloat16, "fp32": torch.float32}[L.out_dtype]
         Y = torch.empty((L.M, L.N), dtype=ydt, device=dev)
         Xq = torch.empty((L.M, L.K), dtype=torch.int8, device=dev)
@@ -161,20 +184,13 @@ def gpu_arm(args):
         dist.barrier()
     ctx = pk.Context(local)
     layers = wl.config_layers(args.config)
-    S = setup_layers(ctx, torch, dev, layers, args.calib_samples)
+    S = setup_layers(ctx, torch, dev, layers, args.calib_samples, rank, world)
     ops_step = sum(L.ops for L in layers)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
-
-    def max_over_ranks(ms):
-        if world == 1:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
 
     # ---- device-resident timing: K whole steps --------------------------------------------
     for _ in range(args.warmup):
@@ -192,11 +208,11 @@ def gpu_arm(args):
     e1.record()
     barrier()
     launches = ctx.stwq_launch_count() - launches0
-    ms_total = max_over_ranks(e0.elapsed_time(e1))
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     clocks = sampler.stop() if rank == 0 else None
     ctx.check_device_status()
     ms_step = ms_total / args.steps
-    value = world * ops_step / (ms_step * 1e-3) / 1e12
+    value = whole_job_tops(world, ops_step, ms_step)
 
     # ---- per-kernel timing on the same stream: quantize and GEMM+epilogue separately --------
     def time_calls(fn):
@@ -265,8 +281,8 @@ def gpu_arm(args):
         e2e_step()
     e1.record()
     barrier()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1)) / args.steps
-    e2e = {"value": round(world * ops_step / (e2e_ms * 1e-3) / 1e12, 3), "unit": "TOPS",
+    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    e2e = {"value": round(whole_job_tops(world, ops_step, e2e_ms), 3), "unit": "TOPS",
            "ms_per_step": round(e2e_ms, 4), "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
     ctx.check_device_status()
 
