@@ -20,9 +20,10 @@ struct stwq_ctx {
     int wait_limit_ms;         // STWQ_OPT_WAIT_LIMIT_MS
     int64_t launches;
     int force_bn;              // tuning: 0 = choose, 128 / 256 = force the tile width
-    int debug;                 // tuning: see Gemm2Params::debug
+    int debug;                 // tuning: variant of the pair GEMM (epilogue store mode, prefetch distance)
     int max_pairs;             // CTA pairs of the pair GEMM that can be resident at once (0 = not yet queried)
-    uint64_t configured_mask;  // kernels whose shared-memory attribute is already set
+    uint64_t configured_mask;  // kernels whose shared-memory attribute is already set (single-CTA GEMM)
+    uint64_t configured_pair[4]; // the same for the pair GEMM, one mask per kernel variant
     uint32_t* d_status;        // device status word
     int8_t* ws_xq;             // workspace: int8 copy of X for qlinear
     size_t ws_xq_bytes;

@@ -120,16 +120,72 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n)
     return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
-// GELU in the epilogue. The erf form uses the rational approximation of the complementary error
-// function by Abramowitz and Stegun (formula 7.1.26; absolute error below 1.5e-7):
-//   erfc(x) ~ (a1 t + ... + a5 t^5) exp(-x^2),  t = 1 / (1 + p x),  x >= 0,
-// so that Phi(z) = erfc(|z|/sqrt2)/2 for z < 0 and 1 - erfc(|z|/sqrt2)/2 otherwise. About 15
-// instructions per element against roughly twice that for erff, which matters because the
-// epilogue of a K = 1024 tile has only a few thousand issue slots. The tanh form is
-// z * sigmoid(2u), u = sqrt(2/pi) (z + 0.044715 z^3).
-template <int ACT>
+// GELU in the epilogue, two accuracy classes.
+//
+// FAST = false (fp32 output, tolerance 1e-5). The erf form uses the rational approximation of
+// the complementary error function by Abramowitz and Stegun (formula 7.1.26; absolute error
+// below 1.5e-7):  erfc(x) ~ (a1 t + ... + a5 t^5) exp(-x^2),  t = 1 / (1 + p x),  x >= 0,
+// so that Phi(z) = erfc(|z|/sqrt2)/2 for z < 0 and 1 - erfc(|z|/sqrt2)/2 otherwise. The tanh form
+// is z * sigmoid(2u), u = sqrt(2/pi) (z + 0.044715 z^3).
+//
+// FAST = true (bf16 output, tolerance 1e-2, rounding unit 2^-9). Both forms are evaluated as
+// z/2 (1 + tanh(u)) with the hardware tanh (tanh.approx.f32, relative error about 2^-11): six
+// instructions per element. For the erf form this relies on the classical fit
+// erf(x / sqrt2) ~ tanh(sqrt(2/pi) (x + 0.044715 x^3)), whose error on Phi stays below 5e-4, a
+// quarter of the bf16 rounding unit. The epilogue of a K = 1024 tile has only a few thousand
+// issue slots, and a 25-instruction erf more than doubles the kernel time.
+__device__ __forceinline__ float tanh_approx(float x)
+{
+    float y;
+    asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// Packed fp32 arithmetic (two IEEE round-to-nearest operations per instruction on sm_100): the
+// epilogue is bound by instruction issue, and this halves its multiply / fma count. Each half
+// rounds exactly like the scalar instruction.
+__device__ __forceinline__ uint64_t pack_f2(float lo, float hi)
+{
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack_f2(uint64_t v, float& lo, float& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t mul_f2(uint64_t a, uint64_t b)
+{
+    uint64_t r;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+    return r;
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c)
+{
+    uint64_t r;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+    return r;
+}
+// The short GELU (see below) on a pair: z/2 (1 + tanh(z (c1 + c3 z^2))).
+__device__ __forceinline__ uint64_t gelu_fast_f2(uint64_t z)
+{
+    const uint64_t c3 = pack_f2(0.035677408136300125f, 0.035677408136300125f);
+    const uint64_t c1 = pack_f2(0.79788456080286536f, 0.79788456080286536f);
+    const uint64_t half = pack_f2(0.5f, 0.5f);
+    const uint64_t u = mul_f2(z, fma_f2(c3, mul_f2(z, z), c1));
+    float u0, u1;
+    unpack_f2(u, u0, u1);
+    const uint64_t t = pack_f2(tanh_approx(u0), tanh_approx(u1));
+    const uint64_t h = mul_f2(half, z);
+    return fma_f2(h, t, h);
+}
+template <int ACT, bool FAST = false>
 __device__ __forceinline__ float apply_act(float z)
 {
+    if (ACT != STWQ_ACT_NONE && FAST) {
+        const float u = z * fmaf(0.035677408136300125f, z * z, 0.79788456080286536f);
+        const float h = 0.5f * z;
+        return fmaf(h, tanh_approx(u), h);
+    }
     if (ACT == STWQ_ACT_GELU_ERF) {
         const float x = fabsf(z) * 0.70710678118654752f;
         const float t = __fdividef(1.0f, fmaf(0.3275911f, x, 1.0f));

@@ -15,10 +15,13 @@
 //                   land on the even CTA's "full" barrier
 //   warp 1          MMA issuer (one lane, even CTA only); tcgen05.commit multicasts "stage free"
 //                   and "accumulator full" to both CTAs
-//   warps 2..2+EPI  epilogue: tcgen05.ld -> fp32 scale/bias/GELU -> convert -> 128-byte-swizzled
-//                   staging tile in shared memory -> TMA store (full-line writes, clipped at the
-//                   matrix edge by the tensor map). Warp w may read TMEM lanes 32*(w%4)..+31; with
-//                   EPI = 8 two warps share a lane quarter and alternate column chunks.
+//   warps 2..2+EPI  epilogue: tcgen05.ld (the next chunk's loads in flight while this one is
+//                   converted; the accumulator is handed back as soon as the last load has
+//                   landed) -> packed fp32 scale/bias/GELU -> convert -> either a 128-byte-swizzled
+//                   staging tile in shared memory and a TMA store (full-line writes, clipped at
+//                   the matrix edge by the tensor map) or 256-bit stores straight from registers.
+//                   Warp w may read TMEM lanes 32*(w%4)..+31; with EPI = 8 two warps share a lane
+//                   quarter and alternate column chunks.
 // Every mbarrier wait is bounded (limit in ns from the host); on expiry the CTA raises
 // STWQ_DEV_TIMEOUT, all roles leave their loops, loads in flight are awaited with the same
 // bound, both CTAs meet at the cluster barrier, tensor memory is freed and the kernel returns.
@@ -42,7 +45,8 @@ struct Gemm2Params {
     int tiles_n, num_tiles, num_kb;
     uint32_t* status;
     unsigned long long wait_limit_ns;
-    int debug;                 // tuning only: 1 = skip the output stores, 2 = skip the whole epilogue body
+    void* Y;                   // used by the direct-store epilogue
+    int y_vec32;               // Y base and row pitch are 32-byte aligned: 256-bit stores are legal
 };
 
 __device__ __forceinline__ uint32_t cluster_ctarank()
@@ -108,20 +112,34 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t
 {
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
+__device__ __forceinline__ void st_global_v8(void* p, const uint32_t* w)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]),
+                 "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+}
+__device__ __forceinline__ void st_global_v4(void* p, const uint32_t* w)
+{
+    asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]) : "memory");
+}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 {
     __nv_bfloat162 b = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&b);
 }
 
-template <int BN, int STAGES, int EPI>
+// STORE = 0: the epilogue stages 32 x 128-byte pieces in shared memory and writes them with TMA
+// (the fewest shared-memory cycles per output byte; best when K is small and the epilogue is
+// as long as the main loop). STORE = 1: every thread writes its row's 128 bytes straight from
+// registers with 256-bit stores; no staging memory, so the operand ring can be deeper.
+template <int BN, int STAGES, int EPI, int STORE>
 struct Smem2 {
     static constexpr int kABytes = kBM * kBK;               // 16 KB
     static constexpr int kBBytes = (BN / 2) * kBK;          // this CTA's half of the Wq slice
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kOffB = STAGES * kABytes;
     static constexpr int kOffStage = STAGES * kStageBytes;  // per epilogue warp: two staging tiles of 32 rows x 128 B
-    static constexpr int kOffScale = kOffStage + EPI * 8192; // per epilogue warp: s_w and bias of its columns
+    static constexpr int kOffScale = kOffStage + (STORE == 0 ? EPI * 8192 : 0); // per epilogue warp: s_w and bias of its columns
     static constexpr int kOffBars = kOffScale + 2 * BN * 4 * 4;
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kOffMisc = kOffBars + kNumBars * 8;
@@ -133,12 +151,13 @@ struct Smem2 {
 // ---------------------------------------------------------------------------- kernel
 // OUT: element type of Y (STWQ_OUT_*); ACT: activation. One staging chunk is 32 rows x 128 bytes:
 // 64 bf16 columns or 32 fp32 / int32 columns.
-template <int BN, int STAGES, int EPI, int OUT, int ACT>
+// STORE: see Smem2.
+template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
 __global__ void __launch_bounds__(64 + 32 * EPI, 1)
 qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
               const __grid_constant__ CUtensorMap tmY, const Gemm2Params p)
 {
-    using L = Smem2<BN, STAGES, EPI>;
+    using L = Smem2<BN, STAGES, EPI, STORE>;
     constexpr int kChunkCols = (OUT == STWQ_OUT_BF16) ? 64 : 32;
     constexpr int kChunks = BN / kChunkCols;
     extern __shared__ uint8_t smem_raw[];
@@ -249,10 +268,11 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         constexpr int kMyChunks = kChunks / kSubs;        // column chunks this warp owns per tile
         constexpr int kMyCols = kMyChunks * kChunkCols;
         static_assert(kChunks % kSubs == 0, "chunks must divide among the warps of a quarter");
-        const uint32_t stage0 = base + L::kOffStage + (uint32_t)ew * 8192u;   // two staging tiles
+        const uint32_t stage0 = base + L::kOffStage + (uint32_t)ew * 8192u;   // two staging tiles (STORE == 0)
         float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 2 * kMyCols;
         float* my_bias = my_sw + kMyCols;
         const uint32_t tempty0 = mapa_u32(bar_tempty(0), 0);
+        constexpr int kElem = (OUT == STWQ_OUT_BF16) ? 2 : 4;
         uint32_t t = 0, nstore = 0;
         bool ok = true;
         for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++t) {
@@ -289,80 +309,115 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-#pragma unroll 1
-            for (int k = 0; k < kMyChunks && p.debug != 2; ++k, ++nstore) {
+            // r0 / r1 hold the accumulators of the chunk being converted; the loads of the next
+            // chunk are issued as soon as the conversion has consumed them, so that their latency
+            // (long while the tensor pipe is busy with the next tile) overlaps this chunk's stores.
+            uint32_t r0[32], r1[32];
+            auto issue_loads = [&](int k) {
                 const int c = sub + k * kSubs;
-                const int col0 = n0 + c * kChunkCols;
-                const uint32_t stage_tile = stage0 + (nstore & 1u) * 4096u;
-                const uint32_t my_row_addr = stage_tile + (uint32_t)lane * 128u;
-                const float* csw = my_sw + k * kChunkCols;
-                const float* cbi = my_bias + k * kChunkCols;
-                __syncwarp();                             // lane 0 issued the previous store: reconverge
                 if (OUT == STWQ_OUT_BF16) {
-                    uint32_t r0[32], r1[32];
                     tmem_ld32(taddr + (uint32_t)(c * 64), r0);
                     tmem_ld32(taddr + (uint32_t)(c * 64 + 32), r1);
-                    // the store that last used this staging tile (two stores ago) must have been read
-                    if (lane == 0) bulk_wait_read1();
-                    __syncwarp();                         // reconverge: the wait below is warp-aligned
-                    tmem_ld_wait();
+                } else {
+                    tmem_ld32(taddr + (uint32_t)(c * 32), r0);
+                }
+            };
+            issue_loads(0);
+#pragma unroll
+            for (int k = 0; k < kMyChunks; ++k, ++nstore) {
+                const int c = sub + k * kSubs;
+                const int col0 = n0 + c * kChunkCols;
+                const float* csw = my_sw + k * kChunkCols;
+                const float* cbi = my_bias + k * kChunkCols;
+                tmem_ld_wait();
+                if (k == kMyChunks - 1) {
+                    // every accumulator column of this warp is in registers: hand the buffer back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
+                }
+                uint32_t w[32];                           // this row's 128 bytes of output
+                const uint64_t st2 = pack_f2(st, st);
+                if (OUT == STWQ_OUT_BF16) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        uint32_t w[16];
 #pragma unroll
                         for (int j = 0; j < 32; j += 4) {
                             const uint32_t* r = h == 0 ? r0 : r1;
                             const float4 sw = *reinterpret_cast<const float4*>(csw + h * 32 + j);
                             const float4 bi = *reinterpret_cast<const float4*>(cbi + h * 32 + j);
-                            const float v0 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 0], __fmul_rn(st, sw.x), bi.x));
-                            const float v1 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 1], __fmul_rn(st, sw.y), bi.y));
-                            const float v2 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 2], __fmul_rn(st, sw.z), bi.z));
-                            const float v3 = apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 3], __fmul_rn(st, sw.w), bi.w));
-                            w[j / 2] = pack_bf16(v0, v1);
-                            w[j / 2 + 1] = pack_bf16(v2, v3);
+                            uint64_t z01 = fma_f2(pack_f2((float)(int32_t)r[j + 0], (float)(int32_t)r[j + 1]),
+                                                  mul_f2(st2, pack_f2(sw.x, sw.y)), pack_f2(bi.x, bi.y));
+                            uint64_t z23 = fma_f2(pack_f2((float)(int32_t)r[j + 2], (float)(int32_t)r[j + 3]),
+                                                  mul_f2(st2, pack_f2(sw.z, sw.w)), pack_f2(bi.z, bi.w));
+                            if (ACT != STWQ_ACT_NONE) {
+                                z01 = gelu_fast_f2(z01);
+                                z23 = gelu_fast_f2(z23);
+                            }
+                            float v0, v1, v2, v3;
+                            unpack_f2(z01, v0, v1);
+                            unpack_f2(z23, v2, v3);
+                            w[h * 16 + j / 2] = pack_bf16(v0, v1);
+                            w[h * 16 + j / 2 + 1] = pack_bf16(v2, v3);
                         }
+                    }
+                } else if (OUT == STWQ_OUT_F32) {
 #pragma unroll
-                        for (int g = 0; g < 4; ++g) {     // four 16-byte pieces, swizzled by row
-                            const uint32_t piece = (uint32_t)((h * 4 + g) ^ (lane & 7));
-                            st_shared_v4(my_row_addr + piece * 16u, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                    for (int j = 0; j < 32; j += 4) {
+                        const float4 sw = *reinterpret_cast<const float4*>(csw + j);
+                        const float4 bi = *reinterpret_cast<const float4*>(cbi + j);
+                        const uint64_t z01 = fma_f2(pack_f2((float)(int32_t)r0[j + 0], (float)(int32_t)r0[j + 1]),
+                                                    mul_f2(st2, pack_f2(sw.x, sw.y)), pack_f2(bi.x, bi.y));
+                        const uint64_t z23 = fma_f2(pack_f2((float)(int32_t)r0[j + 2], (float)(int32_t)r0[j + 3]),
+                                                    mul_f2(st2, pack_f2(sw.z, sw.w)), pack_f2(bi.z, bi.w));
+                        float v0, v1, v2, v3;
+                        unpack_f2(z01, v0, v1);
+                        unpack_f2(z23, v2, v3);
+                        w[j + 0] = __float_as_uint(apply_act<ACT, false>(v0));
+                        w[j + 1] = __float_as_uint(apply_act<ACT, false>(v1));
+                        w[j + 2] = __float_as_uint(apply_act<ACT, false>(v2));
+                        w[j + 3] = __float_as_uint(apply_act<ACT, false>(v3));
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) w[j] = r0[j];
+                }
+                if (k + 1 < kMyChunks) issue_loads(k + 1);
+                if (STORE == 1) {
+                    // straight from registers: this thread's 128 contiguous bytes of row `row`
+                    if (row < p.M && col0 < p.N) {
+                        uint8_t* y = reinterpret_cast<uint8_t*>(p.Y) + ((size_t)row * (size_t)p.N + (size_t)col0) * kElem;
+                        if (p.y_vec32 && col0 + kChunkCols <= p.N) {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) st_global_v8(y + g * 32, w + g * 8);
+                        } else {
+                            const int valid = (p.N - col0) * kElem;        // a multiple of 16 bytes
+#pragma unroll
+                            for (int g = 0; g < 8; ++g)
+                                if (g * 16 < valid) st_global_v4(y + g * 16, w + g * 4);
                         }
                     }
                 } else {
-                    uint32_t r[32];
-                    tmem_ld32(taddr + (uint32_t)(c * 32), r);
+                    const uint32_t stage_tile = stage0 + (nstore & 1u) * 4096u;
+                    const uint32_t my_row_addr = stage_tile + (uint32_t)lane * 128u;
+                    // the store that last used this staging tile (two stores ago) must have been read
                     if (lane == 0) bulk_wait_read1();
-                    __syncwarp();                         // reconverge: the wait below is warp-aligned
-                    tmem_ld_wait();
+                    __syncwarp();
 #pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        uint32_t o0, o1, o2, o3;
-                        if (OUT == STWQ_OUT_INT32) {
-                            o0 = r[j]; o1 = r[j + 1]; o2 = r[j + 2]; o3 = r[j + 3];
-                        } else {
-                            const float4 sw = *reinterpret_cast<const float4*>(csw + j);
-                            const float4 bi = *reinterpret_cast<const float4*>(cbi + j);
-                            o0 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 0], __fmul_rn(st, sw.x), bi.x)));
-                            o1 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 1], __fmul_rn(st, sw.y), bi.y)));
-                            o2 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 2], __fmul_rn(st, sw.z), bi.z)));
-                            o3 = __float_as_uint(apply_act<ACT>(__fmaf_rn((float)(int32_t)r[j + 3], __fmul_rn(st, sw.w), bi.w)));
-                        }
-                        const uint32_t piece = (uint32_t)((j / 4) ^ (lane & 7));
-                        st_shared_v4(my_row_addr + piece * 16u, o0, o1, o2, o3);
+                    for (int g = 0; g < 8; ++g) {         // eight 16-byte pieces, swizzled by row
+                        const uint32_t piece = (uint32_t)(g ^ (lane & 7));
+                        st_shared_v4(my_row_addr + piece * 16u, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                    }
+                    fence_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        if (col0 < p.N && (int64_t)m0 + q * 32 < p.M) tma_store_2d(&tmY, stage_tile, col0, m0 + q * 32);
+                        bulk_commit();    // one group per chunk, even an empty one: wait_group.read 1 counts groups
                     }
                 }
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    if (col0 < p.N && (int64_t)m0 + q * 32 < p.M && p.debug == 0)
-                        tma_store_2d(&tmY, stage_tile, col0, m0 + q * 32);
-                    bulk_commit();    // one group per chunk, even an empty one: wait_group.read 1 counts groups
-                }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
         }
-        if (lane == 0) bulk_wait0();                       // stores complete before the CTA may exit
+        if (STORE == 0 && lane == 0) bulk_wait0();         // stores complete before the CTA may exit
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -401,17 +456,18 @@ int encode_2d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int elem_
     return STWQ_OK;
 }
 
-template <int BN, int STAGES, int EPI, int OUT, int ACT>
+template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
 int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                    const Gemm2Params& p, cudaStream_t st)
 {
-    using L = Smem2<BN, STAGES, EPI>;
-    auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT>;
-    const uint64_t bit = 1ull << (32 + (BN == 256 ? 0 : 12) + OUT * 4 + ACT);
-    if (!(ctx->configured_mask & bit)) {
+    using L = Smem2<BN, STAGES, EPI, STORE>;
+    auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT, STORE>;
+    const uint64_t bit = 1ull << ((BN == 256 ? 0 : 12) + OUT * 4 + ACT);
+    uint64_t& mask = ctx->configured_pair[STORE];
+    if (!(mask & bit)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->configured_mask |= bit;
+        mask |= bit;
     }
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -442,14 +498,14 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
 }
 
-template <int BN, int STAGES, int EPI>
+template <int BN, int STAGES, int EPI, int STORE>
 int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
               const Gemm2Params& p, int act, int out_dtype, cudaStream_t st)
 {
 #define STWQ_CASE(O, A) \
-    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A>(ctx, tmA, tmB, tmY, p, st);
+    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE>(ctx, tmA, tmB, tmY, p, st);
     if (out_dtype == STWQ_OUT_INT32)
-        return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE>(ctx, tmA, tmB, tmY, p, st);
+        return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE>(ctx, tmA, tmB, tmY, p, st);
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
@@ -486,7 +542,9 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     if (ctx->force_bn == 128 || ctx->force_bn == 256) bn = ctx->force_bn;
 
     Gemm2Params p;
-    p.debug = ctx->debug;
+    p.Y = Y;
+    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : 4;
+    p.y_vec32 = ((reinterpret_cast<uintptr_t>(Y) & 31u) == 0 && ((int64_t)N * elem) % 32 == 0) ? 1 : 0;
     p.M = M; p.N = N; p.K = K; p.P = P;
     p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
     p.tiles_n = (N + bn - 1) / bn;
@@ -507,6 +565,13 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     else
         rc = encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
     if (rc != STWQ_OK) return rc;
-    if (bn == 256) return launch_bn<256, 4, 8>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
-    return launch_bn<128, 6, 8>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    if (bn == 128) return launch_bn<128, 6, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    // Long main loops hide the epilogue anyway and gain from the deeper ring that the
+    // register-direct epilogue leaves room for; short ones (and GELU) are bound by the epilogue,
+    // which costs the fewest shared-memory cycles when it goes through staged TMA stores.
+    bool direct = K >= 1536 && act == STWQ_ACT_NONE;
+    if (ctx->debug == 1) direct = false;                  // tuning: force one or the other
+    if (ctx->debug == 2) direct = true;
+    if (direct) return launch_bn<256, 6, 8, 1>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    return launch_bn<256, 4, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
 }
