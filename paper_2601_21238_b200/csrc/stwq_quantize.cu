@@ -23,6 +23,27 @@ __device__ __forceinline__ float4 ld_stream(const float* p)
     return v;
 }
 
+__device__ __forceinline__ void load_row(const float* xrow, int col0, int K, float4 (&v)[4])
+{
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int c = col0 + j * 128;
+        if (c < K) v[j] = ld_stream(xrow + c);
+    }
+}
+
+// Reciprocal token scale of row m (0 and `ok` false if its position is out of range).
+__device__ __forceinline__ float row_scale(const int32_t* pos_ids, const float* s_tok, int P, int64_t m, bool& ok)
+{
+    const int p = pos_ids[m];
+    ok = (p >= 0) && (p < P);
+    return ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
+}
+
+// The loop is software-pipelined: the loads of the next row (and its position scale) are in
+// flight while the current row is converted, and the first row's loads are issued before the
+// reciprocal channel scales are computed, so that a warp that only sees a few rows (M of a few
+// thousand) does not serialise two memory round trips and sixteen divisions in front of them.
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
                 const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin,
@@ -34,6 +55,12 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
     const int span = (int)(warp % spans);
     int64_t m = warp / spans;
     const int col0 = span * kSpan + lane * 4;
+    if (m >= M) return;
+
+    float4 v[4], vn[4];
+    load_row(X + m * K, col0, K, v);
+    bool ok;
+    float rt = row_scale(pos_ids, s_tok, P, m, ok);
 
     // reciprocal channel scales of this lane's 16 columns (1 where there is no scaling)
     float rc[16];
@@ -45,19 +72,17 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
             rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
     }
 
-    for (; m < M; m += row_stride) {
-        const int p = pos_ids[m];
-        const bool ok = (p >= 0) && (p < P);
-        const float rt = ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
-        if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
-        const float* xrow = X + m * K;
-        int8_t* qrow = Xq + m * K;
-        float4 v[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int c = col0 + j * 128;
-            if (c < K) v[j] = ld_stream(xrow + c);
+    while (true) {
+        const int64_t mn = m + row_stride;
+        const bool more = mn < M;
+        bool okn = false;
+        float rtn = 0.0f;
+        if (more) {
+            load_row(X + mn * K, col0, K, vn);
+            rtn = row_scale(pos_ids, s_tok, P, mn, okn);
         }
+        if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+        int8_t* qrow = Xq + m * K;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int c = col0 + j * 128;
@@ -72,6 +97,12 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
                 *reinterpret_cast<uint32_t*>(qrow + c) = packed;
             }
         }
+        if (!more) break;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = vn[j];
+        m = mn;
+        rt = rtn;
+        ok = okn;
     }
 }
 
@@ -83,11 +114,20 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
 {
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
-    // enough warps for every SM to hold 8 blocks, rounded so that each warp keeps one span
-    int64_t want_warps = (int64_t)ctx->sm_count * 8 * warps_per_block;
-    int64_t rows_in_flight = want_warps / spans;
+    // As many warps as can be resident, then the row stride is shrunk so that every warp sees the
+    // same number of rows (no ragged last pass).
+    if (ctx->quant_blocks_per_sm <= 0) {
+        int n = 0;
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel, kThreads, 0);
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->quant_blocks_per_sm = n > 0 ? n : 1;
+    }
+    const int64_t max_warps = (int64_t)ctx->sm_count * ctx->quant_blocks_per_sm * warps_per_block;
+    int64_t rows_in_flight = max_warps / spans;
     if (rows_in_flight < 1) rows_in_flight = 1;
     if (rows_in_flight > M) rows_in_flight = M;
+    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
+    rows_in_flight = (M + passes - 1) / passes;
     // total warps must be rows_in_flight * spans and a multiple of warps_per_block
     while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
     const int64_t blocks = rows_in_flight * spans / warps_per_block;
