@@ -87,14 +87,15 @@ int check_gemm_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int
 
 int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
              const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
-             int out_dtype, void* Y, cudaStream_t st)
+             int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
 {
     const bool can_decode = M <= 256;
     bool decode = can_decode;
     if (ctx->gemm_path == 1 || ctx->gemm_path == 3) decode = false;
     if (ctx->gemm_path == 2 && !can_decode) return STWQ_ERR_DIM;
     if (decode)
-        return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+        return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
+                                  after_quantize, st);
     if (ctx->gemm_path != 3 && stwq_qgemm2_supported(N, out_dtype, s_w, bias))
         return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
     return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
@@ -150,6 +151,7 @@ void stwq_destroy(stwq_ctx* ctx)
     cudaDeviceSynchronize();
     if (ctx->ws_xq) cudaFree(ctx->ws_xq);
     if (ctx->ws_cal) cudaFree(ctx->ws_cal);
+    if (ctx->ws_dec) cudaFree(ctx->ws_dec);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -178,6 +180,7 @@ int stwq_set_option(stwq_ctx* ctx, int option, int value)
     }
     if (option == 100) { ctx->force_bn = value; return STWQ_OK; }   // undocumented tuning knobs
     if (option == 101) { ctx->debug = value; return STWQ_OK; }
+    if (option == 102) { ctx->force_ksplit = value; return STWQ_OK; }
     return STWQ_ERR_DIM;
 }
 
@@ -224,7 +227,7 @@ int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M
     int rc = check_gemm_args(Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, out_dtype, Y);
     if (rc != STWQ_OK) return rc;
     DeviceGuard g(ctx->device);
-    return run_gemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
+    return run_gemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, false,
                     static_cast<cudaStream_t>(stream));
 }
 
@@ -243,7 +246,7 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
     if (rc != STWQ_OK) return rc;
-    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, true, st);
 }
 
 int stwq_device_status(stwq_ctx* ctx, void* stream)

@@ -1,10 +1,483 @@
-// Few-row (decode-step) variant of the quantized linear. Placeholder routing: until the
-// bandwidth-bound kernel lands, few-row calls use the tiled tensor-core GEMM.
+// Few-row (decode-step) variant of the quantized linear: M <= 256 rows, typically one raster-order
+// decode step in which a whole batch advances one token position (Section 2: "one token at a
+// time"). The arithmetic is that of qgemm2 (int8 x int8 -> int32 on the tensor cores, then the
+// Appendix A.1 dequantizer with bias and activation); what differs is the decomposition. With so
+// few rows the weights dominate the traffic (Wq is read once, 16.8 MB at the decode shapes), so
+// the aim is to have every SM pull its share of Wq from HBM from the first cycle:
+//
+//   * one CTA pair (tcgen05 cta_group::2) per work item; the pair's 256 accumulator rows cover
+//     all of M, so Wq is staged exactly once on the whole GPU;
+//   * a work item is a 128-column slice of N and, when N alone does not give one item per pair,
+//     one of `ksplit` ranges of K (split-K);
+//   * the two operands have separate rings. The Wq ring holds 16 k-blocks (128 KB per pair
+//     member), normally the item's whole slab, and its loads are issued before anything else.
+//     The kernel can be launched as a programmatic dependent of the quantize kernel: it then
+//     starts while that kernel still runs, streams Wq, and only waits for the codes of X
+//     (griddepcontrol.wait) before the first load of Xq, which comes from L2 through a 4-stage ring;
+//   * split-K partials are exact int32 sums. Every epilogue warp writes its 32 x 64 piece of the
+//     pair's partial accumulator to scratch memory (lane-interleaved, so that each instruction
+//     moves 512 contiguous bytes) and then bumps a counter that belongs to that piece; the warp
+//     that arrives last (for that piece, across the K ranges) adds the pieces up and runs the
+//     dequantize epilogue. Nobody waits for anybody: there is no spin on another CTA, the
+//     reduction order does not matter for integers, and the last warp puts the counter back to
+//     zero for the next call;
+//   * the output leaves through shared memory (the Xq ring, idle by then) and TMA stores.
+//
+// Scratch (owned by the context): partials [item][rank][warp][16][32 lanes][4] int32 and one
+// counter per (N slice, rank, warp). Calls that use it must be ordered on the GPU (one stream,
+// or events), like every other use of a context's workspace.
+#include <cuda.h>
+
 #include "stwq_internal.cuh"
+#include "stwq_ptx.cuh"
+
+using namespace stwq_ptx;
+
+namespace {
+
+constexpr int kBM = 128;       // rows per CTA (256 per pair)
+constexpr int kBK = 128;       // bytes of K per k-block
+constexpr int kBN = 128;       // columns per work item
+constexpr int kEpi = 8;        // epilogue warps per CTA: 4 lane quarters x 2 column halves
+constexpr int kStagesA = 4;    // Xq ring
+constexpr int kStagesB = 16;   // Wq ring
+constexpr int kFirstEpiWarp = 3;
+constexpr int kThreads = 32 * (kFirstEpiWarp + kEpi);
+constexpr int kPieceInts = 2 * 32 * 32;   // one warp's piece of a partial: 32 rows x 64 columns
+
+struct DecParams {
+    int64_t M;
+    int N, K, P;
+    const int32_t* pos_ids;
+    const float* s_w;
+    const float* s_tok;
+    const float* bias;
+    int ksplit, kb_per_split, num_kb;
+    int32_t* partial;
+    uint32_t* counters;
+    uint32_t* status;
+    unsigned long long wait_limit_ns;
+};
+
+struct SmemDec {
+    static constexpr int kABytes = kBM * kBK;               // 16 KB
+    static constexpr int kBBytes = (kBN / 2) * kBK;         // 8 KB: this CTA's half of the Wq slice
+    static constexpr int kOffB = kStagesA * kABytes;
+    static constexpr int kOffScale = kOffB + kStagesB * kBBytes; // per epilogue warp: s_w and bias of its 64 columns
+    static constexpr int kOffBars = kOffScale + kEpi * 2 * 64 * 4;
+    static constexpr int kNumBars = 2 * kStagesA + 2 * kStagesB + 1;
+    static constexpr int kOffMisc = kOffBars + kNumBars * 8;
+    static constexpr int kTotal = kOffMisc + 16;
+    static constexpr int kDynamic = kTotal + 1024;
+    static_assert(kDynamic <= 227 * 1024, "shared memory budget");
+    static_assert(kStagesA * kABytes >= kEpi * 8192, "the Xq ring doubles as output staging");
+};
+
+__device__ __forceinline__ uint4 ld_cg_v4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p) : "memory");
+    return v;
+}
+// Let the next kernel in the stream start early / wait for the previous one (programmatic
+// dependent launch). Both are no-ops for a kernel that was launched the ordinary way.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+template <int OUT, int ACT>
+__global__ void __launch_bounds__(kThreads, 1)
+decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+              const __grid_constant__ CUtensorMap tmY, const DecParams p)
+{
+    using L = SmemDec;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 1023u) & ~1023u;
+    uint8_t* smem = smem_raw + (base - raw);
+
+    const uint32_t bars = base + L::kOffBars;
+    auto bar_full_a = [&](int s) { return bars + 8u * s; };
+    auto bar_empty_a = [&](int s) { return bars + 8u * (kStagesA + s); };
+    auto bar_full_b = [&](int s) { return bars + 8u * (2 * kStagesA + s); };
+    auto bar_empty_b = [&](int s) { return bars + 8u * (2 * kStagesA + kStagesB + s); };
+    const uint32_t bar_tfull = bars + 8u * (2 * kStagesA + 2 * kStagesB);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + L::kOffMisc + 4);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();            // 0 = even CTA = MMA leader
+    const int item = blockIdx.x >> 1;
+    const int nt = item / p.ksplit;                     // which 128-column slice of N
+    const int ks = item % p.ksplit;                     // which range of K
+    const int kb0 = ks * p.kb_per_split;
+    const int kb1 = min(kb0 + p.kb_per_split, p.num_kb);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStagesA; ++s) {
+            mbar_init(bar_full_a(s), 1);                 // leader's producer arrives with expect_tx
+            mbar_init(bar_empty_a(s), 1);                // multicast commit
+        }
+        for (int s = 0; s < kStagesB; ++s) {
+            mbar_init(bar_full_b(s), 1);
+            mbar_init(bar_empty_b(s), 1);
+        }
+        mbar_init(bar_tfull, 1);
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    if (warp == 2) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(kBN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                  // barriers of both CTAs are initialised
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    const unsigned long long limit = p.wait_limit_ns;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ Wq producer
+        if (lane == 0) {
+            bool ok = true;
+            const uint32_t full0 = mapa_u32(bar_full_b(0), 0);
+            const int n0 = nt * kBN + (int)rank * (kBN / 2);
+            int it = 0;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int s = it % kStagesB;
+                const uint32_t ph = (uint32_t)(it / kStagesB) & 1u;
+                if (!mbar_wait(bar_empty_b(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
+                if (rank == 0) mbar_expect_tx(bar_full_b(s), 2 * L::kBBytes);
+                tma_load_2d_pair(base + L::kOffB + s * L::kBBytes, &tmB, kb * kBK, n0, full0 + 8u * s);
+            }
+            if (!ok && rank == 0) {
+                const int first = it > kStagesB ? it - kStagesB : 0;
+                for (int j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar_full_b(j % kStagesB), (uint32_t)(j / kStagesB) & 1u))
+                        if (globaltimer_ns() - t0 > limit) break;
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ Xq producer
+        if (lane == 0) {
+            grid_dependency_wait();                      // the codes of X come from the previous kernel
+            bool ok = true;
+            const uint32_t full0 = mapa_u32(bar_full_a(0), 0);
+            const int m0 = (int)rank * kBM;
+            int it = 0;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int s = it % kStagesA;
+                const uint32_t ph = (uint32_t)(it / kStagesA) & 1u;
+                if (!mbar_wait(bar_empty_a(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
+                if (rank == 0) mbar_expect_tx(bar_full_a(s), 2 * L::kABytes);
+                tma_load_2d_pair(base + s * L::kABytes, &tmA, kb * kBK, m0, full0 + 8u * s);
+            }
+            if (!ok && rank == 0) {
+                const int first = it > kStagesA ? it - kStagesA : 0;
+                for (int j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar_full_a(j % kStagesA), (uint32_t)(j / kStagesA) & 1u))
+                        if (globaltimer_ns() - t0 > limit) break;
+                }
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------------ MMA issuer (leader)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc_i8(2 * kBM, kBN);
+            bool ok = true;
+            int it = 0;
+            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                const int sa = it % kStagesA, sb = it % kStagesB;
+                if (!mbar_wait(bar_full_b(sb), (uint32_t)(it / kStagesB) & 1u, abort_flag, limit)) { ok = false; break; }
+                if (!mbar_wait(bar_full_a(sa), (uint32_t)(it / kStagesA) & 1u, abort_flag, limit)) { ok = false; break; }
+                tc_fence_after();
+                const uint64_t a_desc = make_smem_desc(base + sa * L::kABytes);
+                const uint64_t b_desc = make_smem_desc(base + L::kOffB + sb * L::kBBytes);
+#pragma unroll
+                for (int k = 0; k < kBK / 32; ++k)
+                    tc_mma_i8_pair(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, (it | k) != 0 ? 1u : 0u);
+                tc_commit_pair(bar_empty_a(sa));
+                tc_commit_pair(bar_empty_b(sb));
+            }
+            if (ok) tc_commit_pair(bar_tfull);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int ew = warp - kFirstEpiWarp;              // 0..7
+        const int q = warp & 3;                           // TMEM lane quarter
+        const int sub = ew >> 2;                          // column half of the slice
+        const int n0 = nt * kBN + sub * 64;               // first column of this warp's piece
+        const int row0 = (int)rank * kBM + q * 32;
+        const int64_t row = (int64_t)row0 + lane;
+        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 128;
+        float* my_bias = my_sw + 64;
+        float st = 0.0f;
+        if (OUT != STWQ_OUT_INT32) {
+            for (int i = lane; i < 64; i += 32) {
+                const int col = n0 + i;
+                my_sw[i] = col < p.N ? __ldg(p.s_w + col) : 0.0f;
+                my_bias[i] = (p.bias != nullptr && col < p.N) ? __ldg(p.bias + col) : 0.0f;
+            }
+            if (row < p.M) {
+                const int pos = p.pos_ids[row];
+                if (pos >= 0 && pos < p.P) st = p.s_tok[pos];
+                else if (item == 0 && sub == 0) atomicOr(p.status, STWQ_DEV_POS_RANGE);
+            }
+            __syncwarp();
+        }
+        bool ok = mbar_wait(bar_tfull, 0u, abort_flag, limit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(sub * 64);
+            uint32_t r0[32], r1[32];                      // this row's 64 accumulators
+            tmem_ld32(taddr, r0);
+            tmem_ld32(taddr + 32u, r1);
+            tmem_ld_wait();
+            bool finish = true;
+            if (p.ksplit > 1) {
+                // publish this warp's piece of the partial sum, then see who is last
+                int32_t* piece = p.partial + ((((size_t)nt * p.ksplit + ks) * 2 + rank) * kEpi + ew) * kPieceInts;
+#pragma unroll
+                for (int g = 0; g < 8; ++g) {
+                    st_global_v4(piece + ((size_t)g * 32 + lane) * 4, r0 + g * 4);
+                    st_global_v4(piece + ((size_t)(8 + g) * 32 + lane) * 4, r1 + g * 4);
+                }
+                __threadfence();
+                __syncwarp();
+                uint32_t* counter = p.counters + ((size_t)nt * 2 + rank) * kEpi + ew;
+                uint32_t old = 0;
+                if (lane == 0) {
+                    old = atomicAdd(counter, 1u);
+                    if (old == (uint32_t)p.ksplit - 1u) *counter = 0u;    // everyone has arrived: ready for the next call
+                }
+                old = __shfl_sync(0xffffffffu, old, 0);
+                finish = (old == (uint32_t)p.ksplit - 1u);
+                if (finish) {
+                    __threadfence();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) { r0[j] = 0u; r1[j] = 0u; }
+#pragma unroll 2
+                    for (int s2 = 0; s2 < p.ksplit; ++s2) {
+                        const int32_t* src = p.partial + ((((size_t)nt * p.ksplit + s2) * 2 + rank) * kEpi + ew) * kPieceInts;
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint4 a = ld_cg_v4(src + ((size_t)g * 32 + lane) * 4);
+                            const uint4 b = ld_cg_v4(src + ((size_t)(8 + g) * 32 + lane) * 4);
+                            r0[g * 4 + 0] += a.x; r0[g * 4 + 1] += a.y; r0[g * 4 + 2] += a.z; r0[g * 4 + 3] += a.w;
+                            r1[g * 4 + 0] += b.x; r1[g * 4 + 1] += b.y; r1[g * 4 + 2] += b.z; r1[g * 4 + 3] += b.w;
+                        }
+                    }
+                }
+            }
+            if (finish) {
+                // 32 rows x 64 columns -> this warp's staging tiles (8 KB of the idle Xq ring): one
+                // 32 x 128-byte tile for bf16, two for fp32 / int32, 128-byte swizzled as TMA expects
+                const uint32_t stage = base + (uint32_t)ew * 8192u;
+                const uint64_t st2 = pack_f2(st, st);
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {             // two halves of 32 columns
+                    const uint32_t* r = h == 0 ? r0 : r1;
+                    if (OUT == STWQ_OUT_BF16) {
+                        uint32_t w[16];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 2) {
+                            const uint64_t sw = pack_f2(my_sw[h * 32 + j], my_sw[h * 32 + j + 1]);
+                            const uint64_t bi = pack_f2(my_bias[h * 32 + j], my_bias[h * 32 + j + 1]);
+                            uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
+                            if (ACT != STWQ_ACT_NONE) z = gelu_fast_f2(z);
+                            float v0, v1;
+                            unpack_f2(z, v0, v1);
+                            w[j / 2] = pack_bf16(v0, v1);
+                        }
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const uint32_t piece16 = (uint32_t)((h * 4 + g) ^ (lane & 7));
+                            st_shared_v4(stage + (uint32_t)lane * 128u + piece16 * 16u, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
+                        }
+                    } else {
+                        uint32_t w[32];
+                        if (OUT == STWQ_OUT_INT32) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) w[j] = r[j];
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 2) {
+                                const uint64_t sw = pack_f2(my_sw[h * 32 + j], my_sw[h * 32 + j + 1]);
+                                const uint64_t bi = pack_f2(my_bias[h * 32 + j], my_bias[h * 32 + j + 1]);
+                                const uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
+                                float v0, v1;
+                                unpack_f2(z, v0, v1);
+                                w[j] = __float_as_uint(apply_act<ACT, false>(v0));
+                                w[j + 1] = __float_as_uint(apply_act<ACT, false>(v1));
+                            }
+                        }
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint32_t piece16 = (uint32_t)(g ^ (lane & 7));
+                            st_shared_v4(stage + (uint32_t)h * 4096u + (uint32_t)lane * 128u + piece16 * 16u, w[4 * g], w[4 * g + 1],
+                                         w[4 * g + 2], w[4 * g + 3]);
+                        }
+                    }
+                }
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0 && row0 < p.M) {
+                    if (OUT == STWQ_OUT_BF16) {
+                        if (n0 < p.N) tma_store_2d(&tmY, stage, n0, row0);
+                    } else {
+                        if (n0 < p.N) tma_store_2d(&tmY, stage, n0, row0);
+                        if (n0 + 32 < p.N) tma_store_2d(&tmY, stage + 4096u, n0 + 32, row0);
+                    }
+                    bulk_commit();
+                    bulk_wait0();                         // the stores have completed before the CTA may exit
+                }
+            }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, STWQ_DEV_TIMEOUT);
+    cluster_sync_all();                                  // no remote arrive or multicast still to land
+    tc_fence_after();
+    if (warp == 2) {
+        __syncwarp();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kBN) : "memory");
+    }
+}
+
+template <int OUT, int ACT>
+int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
+                   const DecParams& p, int items, bool dependent, cudaStream_t st)
+{
+    auto kern = decode_kernel<OUT, ACT>;
+    const uint64_t bit = 1ull << (OUT * 4 + ACT);
+    if (!(ctx->configured_decode & bit)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SmemDec::kDynamic);
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->configured_decode |= bit;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    // may start while the previous kernel of the stream (the quantize kernel) still runs
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)(2 * items), 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = SmemDec::kDynamic;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
+    ctx->launches += 1;
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+// Scratch for split-K: partial pieces for `items` work items and one counter per piece of an N slice.
+int ensure_scratch(stwq_ctx* ctx, int items, int tiles_n)
+{
+    const size_t partial_bytes = (size_t)items * 2 * kEpi * kPieceInts * sizeof(int32_t);
+    const size_t counter_bytes = (((size_t)tiles_n * 2 * kEpi * sizeof(uint32_t)) + 255) & ~(size_t)255;
+    const size_t need = partial_bytes + counter_bytes;
+    if (ctx->ws_dec_bytes >= need && ctx->ws_dec_counter_bytes >= counter_bytes) return STWQ_OK;
+    if (ctx->ws_dec) {
+        cudaError_t e = cudaFree(ctx->ws_dec);            // synchronises
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->ws_dec = nullptr;
+        ctx->ws_dec_bytes = 0;
+    }
+    void* ptr = nullptr;
+    cudaError_t e = cudaMalloc(&ptr, need);
+    if (e == cudaSuccess) e = cudaMemset(ptr, 0, counter_bytes);   // counters sit first and start at zero
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        if (ptr) cudaFree(ptr);
+        return STWQ_ERR_NOMEM;
+    }
+    ctx->ws_dec = ptr;
+    ctx->ws_dec_bytes = need;
+    ctx->ws_dec_counter_bytes = counter_bytes;
+    return STWQ_OK;
+}
+
+}  // namespace
 
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
-                       int act, int out_dtype, void* Y, cudaStream_t st)
+                       int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
 {
-    return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : 4;
+    // the TMA store of Y needs 16-byte row pitches; otherwise the general tiled kernel runs
+    if (M > 2 * kBM || ((int64_t)N * elem) % 16 != 0)
+        return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+
+    DecParams p;
+    p.M = M; p.N = N; p.K = K; p.P = P;
+    p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
+    p.num_kb = (K + kBK - 1) / kBK;
+    const int tiles_n = (N + kBN - 1) / kBN;
+    // One work item per CTA pair if N allows; otherwise split K so that about sm_count / 2 pairs
+    // have work, keeping at least four k-blocks per item.
+    const int pairs = ctx->sm_count / 2;
+    int ksplit = 1;
+    if (tiles_n * 4 < pairs * 3) {
+        ksplit = pairs / tiles_n;
+        if (ksplit > p.num_kb / 4) ksplit = p.num_kb / 4;
+        if (ksplit > 32) ksplit = 32;
+        if (ksplit < 1) ksplit = 1;
+    }
+    if (ctx->force_ksplit > 0) ksplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
+    p.kb_per_split = (p.num_kb + ksplit - 1) / ksplit;
+    p.ksplit = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;      // every range holds at least one k-block
+    const int items = tiles_n * p.ksplit;
+    p.partial = nullptr;
+    p.counters = nullptr;
+    if (p.ksplit > 1) {
+        int rc = ensure_scratch(ctx, items, tiles_n);
+        if (rc != STWQ_OK) return rc;
+        p.counters = reinterpret_cast<uint32_t*>(ctx->ws_dec);
+        p.partial = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctx->ws_dec) + ctx->ws_dec_counter_bytes);
+    }
+    p.status = ctx->d_status;
+    p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
+
+    CUtensorMap tmA, tmB, tmY;
+    int rc = stwq_encode_2d(ctx, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kBK, kBM);
+    if (rc != STWQ_OK) return rc;
+    rc = stwq_encode_2d(ctx, &tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, N, K, kBK, kBN / 2);
+    if (rc != STWQ_OK) return rc;
+    if (out_dtype == STWQ_OUT_BF16)
+        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, M, N, 64, 32);
+    else if (out_dtype == STWQ_OUT_F32)
+        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Y, M, N, 32, 32);
+    else
+        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
+    if (rc != STWQ_OK) return rc;
+    const bool dependent = after_quantize && ctx->debug != 5;   // tuning: 5 = ordinary launch
+
+#define STWQ_CASE(O, A) \
+    if (out_dtype == O && act == A) return launch_variant<O, A>(ctx, tmA, tmB, tmY, p, items, dependent, st);
+    if (out_dtype == STWQ_OUT_INT32) return launch_variant<STWQ_OUT_INT32, STWQ_ACT_NONE>(ctx, tmA, tmB, tmY, p, items, dependent, st);
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+#undef STWQ_CASE
+    return STWQ_ERR_BITS;
 }

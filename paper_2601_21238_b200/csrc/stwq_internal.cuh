@@ -30,6 +30,11 @@ struct stwq_ctx {
     size_t ws_xq_bytes;
     void* ws_cal;              // workspace: calibration histograms and selection state
     size_t ws_cal_bytes;
+    void* ws_dec;              // workspace of the few-row path: split-K counters, then partial sums
+    size_t ws_dec_bytes;
+    size_t ws_dec_counter_bytes;
+    uint64_t configured_decode;
+    int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
 };
 
@@ -52,7 +57,7 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
                        const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
-                       const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
+                       const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);
 
 static inline int stwq_cuda_fail(stwq_ctx* ctx, cudaError_t e)
 {

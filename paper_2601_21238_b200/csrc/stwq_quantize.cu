@@ -50,6 +50,10 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
                 int qmax, int8_t* __restrict__ Xq, int spans, int64_t row_stride,
                 uint32_t* __restrict__ status)
 {
+    // A kernel launched as a programmatic dependent of this one (the few-row GEMM, which first
+    // streams weights that do not depend on Xq) may start now; it waits for this grid to finish
+    // before it touches Xq. Without such a dependent this does nothing.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
     const int span = (int)(warp % spans);

@@ -331,3 +331,25 @@ def test_decode_rows_with_mixed_positions_and_few_rows(gpu):
         for path in (0, 2):
             np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", act=1, path=path), ref["acc"])
             assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32", act=1, path=path), ref, RTOL["fp32"], "decode")
+
+
+@pytest.mark.parametrize("ksplit", [0, 2, 5])
+@pytest.mark.parametrize("shape", [(256, 2048, 256), (200, 1536, 136), (37, 4096, 128), (1, 512, 1024)])
+def test_decode_split_k_is_exact_and_repeatable(gpu, shape, ksplit):
+    """The few-row path with K split over several CTA pairs: int32 partial sums through scratch
+    memory, added up by whichever warp arrives last. Exact, and the counters return to zero, so a
+    second call gives the same bits."""
+    M, K, N = shape
+    L = wl.scaled(wl.config_layers(4)[0], K=K, N=N, P=16)
+    par = prepare(L, samples=4, gps_n=64)
+    X = wl.activations(wl.scaled(L, batch=256))[:M]
+    pos = rng.integers(0, L.P, M).astype(np.int32)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 2)
+    gpu.ctx.stwq_set_option(102, ksplit)
+    try:
+        for _ in range(2):
+            np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", act=2, path=2), ref["acc"])
+            assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32", act=2, path=2), ref, RTOL["fp32"], "decode fp32")
+            assert_close(_run_qlinear(gpu, L, par, X, pos, "bf16", act=2, path=2), ref, RTOL["bf16"], "decode bf16")
+    finally:
+        gpu.ctx.stwq_set_option(102, 0)
