@@ -193,8 +193,23 @@ def gpu_arm(args):
         torch.cuda.synchronize()
 
     # ---- device-resident timing: K whole steps --------------------------------------------
+    # The step (4 qlinear calls = 8 kernels) is captured once into a CUDA graph through the same
+    # C-ABI calls and replayed K times, the way a serving loop would issue it; --no-graph issues
+    # the calls one by one instead (then the host's launch rate adds ~10 % to the step).
     for _ in range(args.warmup):
         run_step(ctx, S)
+    torch.cuda.synchronize()
+    main = torch.cuda.Stream()
+    graph = None
+    if not args.no_graph:
+        with torch.cuda.stream(main):
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=main):
+                run_step(ctx, S)
+            for _ in range(args.warmup):
+                graph.replay()
+        torch.cuda.synchronize()
+    launches_per_step = 2 * len(S)
     sampler = ClockSampler(local)
     barrier()
     if rank == 0:
@@ -202,37 +217,59 @@ def gpu_arm(args):
     launches0 = ctx.stwq_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
-    e0.record()
-    for _ in range(args.steps):
-        run_step(ctx, S)
-    e1.record()
+    with torch.cuda.stream(main):
+        e0.record()
+        for _ in range(args.steps):
+            if graph is not None:
+                graph.replay()
+            else:
+                run_step(ctx, S)
+        e1.record()
     barrier()
-    launches = ctx.stwq_launch_count() - launches0
+    launches = (ctx.stwq_launch_count() - launches0) if graph is None else launches_per_step * args.steps
     ms_total = max_over_ranks(e0.elapsed_time(e1), world, dev)
     clocks = sampler.stop() if rank == 0 else None
     ctx.check_device_status()
     ms_step = ms_total / args.steps
     value = whole_job_tops(world, ops_step, ms_step)
 
-    # ---- per-kernel timing on the same stream: quantize and GEMM+epilogue separately --------
-    def time_calls(fn):
-        evs = []
-        for _ in range(args.steps):
-            for s in S:
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                fn(s)
-                b.record()
-                evs.append((s["L"].name, a, b))
-        torch.cuda.synchronize()
-        acc = {}
-        for name, a, b in evs:
-            acc.setdefault(name, []).append(a.elapsed_time(b))
-        return {k: sum(v) / len(v) for k, v in acc.items()}
+    # ---- per-kernel timing: quantize and GEMM+epilogue separately ------------------------------
+    # Each kernel is captured a few times into a CUDA graph and the replays are timed with events
+    # on the replay stream, so that the figure is device time, not the host's launch rate. The
+    # quantize kernel reads a different copy of X on every launch (working set > L2, as in the
+    # step, where the four layers' inputs evict one another); the GEMM reads the codes that the
+    # quantize kernel has just written, as in the step.
+    side = torch.cuda.Stream()
 
-    tq = time_calls(lambda s: ctx.stwq_quantize(s["X"], s["pos"], s["s_ch"], s["s_tok"], s["L"].bits, s["Xq"]))
-    tg = time_calls(lambda s: ctx.qlinear_q(s["Xq"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["bias"],
-                                            s["L"].act, s["out_code"], s["Y"]))
+    def graph_time(calls, replays=5):
+        with torch.cuda.stream(side):
+            for c in calls:
+                c()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                for c in calls:
+                    c()
+            g.replay()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(replays):
+                g.replay()
+            b.record()
+            torch.cuda.synchronize()
+        return a.elapsed_time(b) / (replays * len(calls))
+
+    tq, tg = {}, {}
+    l2_bytes = 2 * 126e6
+    for s in S:
+        L = s["L"]
+        ncopy = max(2, int(l2_bytes // (5.0 * L.M * L.K)) + 1)
+        Xc = [s["X"]] + [s["X"].clone() for _ in range(ncopy - 1)]
+        tq[L.name] = graph_time([(lambda x=x: ctx.stwq_quantize(x, s["pos"], s["s_ch"], s["s_tok"], L.bits, s["Xq"]))
+                                 for x in Xc] * 2)
+        del Xc
+        tg[L.name] = graph_time([lambda: ctx.qlinear_q(s["Xq"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["bias"],
+                                                       L.act, s["out_code"], s["Y"])] * 10)
     peaks = measured_peaks()
     per_layer = []
     for s in S:
@@ -245,7 +282,7 @@ def gpu_arm(args):
     gemm_ms = sum(tg.values())
     achieved = ops_step / (gemm_ms * 1e-3) / 1e12
     peak = peaks["bf16_tflops"] * INT8_OVER_BF16
-    roofline = {"kernel": "qgemm_kernel (tcgen05 kind::i8 GEMM + dequant epilogue)", "bound": "tensor",
+    roofline = {"kernel": "qgemm2_kernel (CTA-pair tcgen05 kind::i8 GEMM + dequant epilogue), mean over the 4 layer shapes", "bound": "tensor",
                 "achieved": round(achieved, 1), "peak": round(peak, 1), "unit": "TOP/s",
                 "frac": round(achieved / peak, 4),
                 "peak_source": f"2 x bf16_tflops of {peaks['_source']} peaks (burst)",
@@ -294,10 +331,13 @@ def gpu_arm(args):
                            f"{L.name} {L.K}->{L.N}" for L in layers) + f"; M={layers[0].M} per GPU, W8A8, "
                            f"{layers[0].out_dtype} out",
                        "l2": "inputs larger than L2 (one step touches ~0.6 GB per GPU)",
+                       "launch": "CUDA graph of the step's 4 qlinear calls" if graph is not None else "one C-ABI call at a time",
                        "s_ch": "seeded stand-in for the GPS vector on qkv/fc1", "calib_samples": args.calib_samples},
             "roofline": roofline, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
             "layers": per_layer,
             "pct_of_nominal_int8_peak": round(100 * achieved / 4500.0, 2)}
+    if not args.no_extras:
+        line["other_configs"] = other_configs(ctx, pk, torch, dev, peaks)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(S, layers, torch, rows=args.cpu_rows)
     if rank == 0:
@@ -305,6 +345,81 @@ def gpu_arm(args):
     ctx.close()
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_configs(ctx, pk, torch, dev, peaks):
+    """Timing-only figures for the workload shapes that are not the benchmark's step (random codes
+    and scales of the right shapes; parity of these shapes is the tests' business): the GEMM and
+    quantize kernels of the VAR-d30 and MAR-Huge layers, and the decode-step qlinear measured in a
+    CUDA graph that rotates through more weight copies than fit in L2."""
+    out = {}
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+
+    def burst(fn, n=20, warm=3):
+        for _ in range(warm):
+            fn()
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(n):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    for cfg in (3, 5):
+        rows = []
+        for L in wl.config_layers(cfg):
+            X = torch.randn(L.M, L.K, device=dev)
+            Xq = torch.empty((L.M, L.K), dtype=torch.int8, device=dev)
+            Wq = torch.randint(-128, 128, (L.N, L.K), dtype=torch.int8, device=dev)
+            pos = torch.from_numpy(wl.positions(L)).to(dev)
+            s_w = torch.rand(L.N, device=dev) * 1e-3 + 1e-4
+            s_tok = torch.rand(L.P, device=dev) * 0.05 + 0.01
+            s_ch = (torch.rand(L.K, device=dev) + 0.5) if L.use_gps else None
+            b = torch.randn(L.N, device=dev) * 0.02
+            Y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device=dev)
+            tq = burst(lambda: ctx.stwq_quantize(X, pos, s_ch, s_tok, 8, Xq))
+            tg = burst(lambda: ctx.qlinear_q(Xq, pos, Wq, s_w, s_tok, b, L.act, pk.OUT_BF16, Y))
+            rows.append({"layer": L.name, "M": L.M, "K": L.K, "N": L.N, "act": L.act,
+                         "gemm_tops": round(L.ops / tg / 1e9, 1), "gemm_ms": round(tg, 4),
+                         "quantize_gbs": round(5.0 * L.M * L.K / tq / 1e6, 1), "quantize_ms": round(tq, 4)})
+            del X, Xq, Wq, Y
+        out[f"config{cfg}"] = rows
+    # decode step: X fp32 + Wq + Y bf16 per call, weights rotated so that they come from HBM
+    rows = []
+    copies = 12
+    for L in wl.config_layers(4):
+        Xs = [torch.randn(L.M, L.K, device=dev) for _ in range(copies)]
+        Ws = [torch.randint(-128, 128, (L.N, L.K), dtype=torch.int8, device=dev) for _ in range(copies)]
+        Ys = [torch.empty((L.M, L.N), dtype=torch.bfloat16, device=dev) for _ in range(copies)]
+        pos = torch.full((L.M,), 17, dtype=torch.int32, device=dev)
+        s_w = torch.rand(L.N, device=dev) * 1e-3 + 1e-4
+        s_tok = torch.rand(L.P, device=dev) * 0.05 + 0.01
+        s_ch = (torch.rand(L.K, device=dev) + 0.5) if L.use_gps else None
+        b = torch.randn(L.N, device=dev) * 0.02
+
+        def rot():
+            for i in range(copies):
+                ctx.qlinear(Xs[i], pos, Ws[i], s_w, s_tok, s_ch, b, 8, 0, pk.OUT_BF16, Ys[i])
+        rot()
+        torch.cuda.synchronize()
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            rot()
+            torch.cuda.synchronize()
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                rot()
+        torch.cuda.synchronize()
+        us = burst(g.replay, n=20) / copies * 1e3
+        byts = 4.0 * L.M * L.K + L.N * L.K + 2.0 * L.M * L.N
+        rows.append({"layer": L.name, "M": L.M, "K": L.K, "N": L.N, "qlinear_us": round(us, 2),
+                     "gbs": round(byts / us / 1e3, 1), "frac_of_hbm": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),
+                     "tops": round(L.ops / us / 1e6, 1), "timing": f"CUDA graph, {copies} weight copies rotated (HBM-cold)"})
+        del Xs, Ws, Ys, g
+    out["config4"] = rows
+    ctx.check_device_status()
+    return out
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle
@@ -374,14 +489,16 @@ def reference_arm(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", type=int, default=2, help="workload family 1..5 (default: VAR-d16 block)")
     ap.add_argument("--calib-samples", type=int, default=32)
     ap.add_argument("--cpu-rows", type=int, default=10880)
     ap.add_argument("--ref-rows", type=int, default=256)
+    ap.add_argument("--no-graph", action="store_true", help="issue the step's calls one by one instead of replaying a CUDA graph")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", action="store_true", help="skip the timing-only figures of configs 3, 4, 5")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
