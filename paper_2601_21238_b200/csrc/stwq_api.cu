@@ -97,7 +97,8 @@ int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M,
         return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
                                   after_quantize, st);
     if (ctx->gemm_path != 3 && stwq_qgemm2_supported(N, out_dtype, s_w, bias))
-        return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
+        return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
+                                  after_quantize, st);
     return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
 }
 
@@ -215,7 +216,7 @@ int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t
     if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     if ((K & 15) != 0 || !aligned16(X) || !aligned16(Xq)) return STWQ_ERR_ALIGN;
     DeviceGuard g(ctx->device);
-    return stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, Xq,
+    return stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, Xq, false,
                                 static_cast<cudaStream_t>(stream));
 }
 
@@ -244,9 +245,14 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     rc = ensure_xq(ctx, (size_t)M * (size_t)K);
     if (rc != STWQ_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
+    // Both kernels are launched as programmatic dependents of their predecessor in the stream:
+    // each executes griddepcontrol.wait before it reads or writes anything the predecessor could
+    // have produced, so the order of effects is that of ordinary launches; what overlaps is the
+    // launch itself and the GEMM's prologue.
+    const bool pdl = ctx->debug != 5;                     // tuning: 5 = ordinary launches
+    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, pdl, st);
     if (rc != STWQ_OK) return rc;
-    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, true, st);
+    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, pdl, st);
 }
 
 int stwq_device_status(stwq_ctx* ctx, void* stream)

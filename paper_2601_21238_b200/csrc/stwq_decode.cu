@@ -105,6 +105,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up behind this grid
     const uint32_t rank = cluster_ctarank();            // 0 = even CTA = MMA leader
     const int item = blockIdx.x >> 1;
     const int nt = item / p.ksplit;                     // which 128-column slice of N

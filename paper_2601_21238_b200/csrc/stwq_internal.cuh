@@ -41,7 +41,7 @@ struct stwq_ctx {
 // Launchers (host). Each returns STWQ_OK or STWQ_ERR_CUDA and bumps ctx->launches.
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
-                         cudaStream_t st);
+                         bool dependent, cudaStream_t st);
 int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);
@@ -54,7 +54,8 @@ int stwq_launch_qgemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, i
 bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* bias);
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
-                       const float* bias, int act, int out_dtype, void* Y, cudaStream_t st);
+                       const float* bias, int act, int out_dtype, void* Y, bool after_quantize,
+                       cudaStream_t st);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);

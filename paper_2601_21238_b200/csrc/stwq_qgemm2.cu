@@ -96,6 +96,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next kernel may queue up behind this grid
     const uint32_t rank = cluster_ctarank();            // 0 = even CTA = MMA leader
     const int pair = blockIdx.x >> 1;
     const int num_pairs = gridDim.x >> 1;
@@ -132,6 +133,10 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             uint32_t it = 0;
             bool ok = true;
             const uint32_t full0 = mapa_u32(bar_full(0), 0);     // leader's barriers
+            // launched as a programmatic dependent of the quantize kernel: everything up to here
+            // (barriers, tensor memory, cluster handshake) may have run while that kernel drained;
+            // its codes are read only from here on
+            asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
                 const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
                 const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
@@ -383,7 +388,7 @@ namespace {
 
 template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
 int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
-                   const Gemm2Params& p, cudaStream_t st)
+                   const Gemm2Params& p, bool dependent, cudaStream_t st)
 {
     using L = Smem2<BN, STAGES, EPI, STORE>;
     auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT, STORE>;
@@ -395,11 +400,13 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
         mask |= bit;
     }
     cudaLaunchConfig_t cfg = {};
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.blockDim = dim3(64 + 32 * EPI, 1, 1);
     cfg.dynamicSmemBytes = L::kDynamic;
     cfg.stream = st;
@@ -417,6 +424,7 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
     int pairs = ctx->max_pairs;
     if (p.num_tiles < pairs) pairs = p.num_tiles;
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
+    cfg.numAttrs = dependent ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
     ctx->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
@@ -425,12 +433,12 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
 
 template <int BN, int STAGES, int EPI, int STORE>
 int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
-              const Gemm2Params& p, int act, int out_dtype, cudaStream_t st)
+              const Gemm2Params& p, int act, int out_dtype, bool dependent, cudaStream_t st)
 {
 #define STWQ_CASE(O, A) \
-    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE>(ctx, tmA, tmB, tmY, p, st);
+    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
     if (out_dtype == STWQ_OUT_INT32)
-        return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE>(ctx, tmA, tmB, tmY, p, st);
+        return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
@@ -458,7 +466,7 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
-                       int act, int out_dtype, void* Y, cudaStream_t st)
+                       int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
 {
     // 256-wide tiles whenever N has more than 128 columns: a 128-wide tile needs 1.5x the
     // L2 -> shared-memory bytes per multiply-accumulate and is bound by that feed.
@@ -490,13 +498,13 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     else
         rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
     if (rc != STWQ_OK) return rc;
-    if (bn == 128) return launch_bn<128, 6, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    if (bn == 128) return launch_bn<128, 6, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
     // Long main loops hide the epilogue anyway and gain from the deeper ring that the
     // register-direct epilogue leaves room for; short ones (and GELU) are bound by the epilogue,
     // which costs the fewest shared-memory cycles when it goes through staged TMA stores.
     bool direct = K >= 1536 && act == STWQ_ACT_NONE;
     if (ctx->debug == 1) direct = false;                  // tuning: force one or the other
     if (ctx->debug == 2) direct = true;
-    if (direct) return launch_bn<256, 6, 8, 1>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
-    return launch_bn<256, 4, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, st);
+    if (direct) return launch_bn<256, 6, 8, 1>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
+    return launch_bn<256, 4, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
 }

@@ -50,9 +50,13 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
                 int qmax, int8_t* __restrict__ Xq, int spans, int64_t row_stride,
                 uint32_t* __restrict__ status)
 {
-    // A kernel launched as a programmatic dependent of this one (the few-row GEMM, which first
-    // streams weights that do not depend on Xq) may start now; it waits for this grid to finish
-    // before it touches Xq. Without such a dependent this does nothing.
+    // Programmatic dependent launch, both directions. If this grid was launched as a dependent of
+    // the previous kernel of the stream, its blocks may already be resident while that kernel
+    // drains; nothing is read or written before that kernel has completed (wait). And a kernel
+    // launched as a dependent of this one (the GEMM, which has a prologue, and in the few-row case
+    // weights to stream, that do not depend on Xq) may start now; it waits for this grid to
+    // finish before it touches Xq. Launched the ordinary way, both instructions do nothing.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
@@ -114,7 +118,7 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
 
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
-                         cudaStream_t st)
+                         bool dependent, cudaStream_t st)
 {
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
@@ -136,10 +140,19 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
     const int64_t blocks = rows_in_flight * spans / warps_per_block;
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    quantize_kernel<<<(unsigned)blocks, kThreads, 0, st>>>(X, pos_ids, M, K, s_ch, s_tok, P, qmin,
-                                                           qmax, Xq, spans, rows_in_flight,
-                                                           ctx->d_status);
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)blocks, 1, 1);
+    cfg.blockDim = dim3(kThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quantize_kernel, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
+                                       rows_in_flight, ctx->d_status);
     ctx->launches += 1;
-    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
 }

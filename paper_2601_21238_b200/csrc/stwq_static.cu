@@ -111,11 +111,11 @@ extern "C" int qlinear_static(const float* X, const int32_t* pos_ids, int64_t M,
     if (rc != STWQ_OK) return rc;
     stwq_ctx* ctx = &slot->ctx;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
+    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, false, st);
     if (rc != STWQ_OK) return rc;
     if (stwq_qgemm2_supported(N, out_dtype, s_w, bias))
         return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act,
-                                  out_dtype, Y, st);
+                                  out_dtype, Y, false, st);
     return stwq_launch_qgemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype,
                              Y, st);
 }
