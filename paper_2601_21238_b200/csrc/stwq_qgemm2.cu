@@ -235,33 +235,32 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             if (!ok) break;
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(acc * BN);
-            // r0 / r1 hold the accumulators of the chunk being converted; the loads of the next
-            // chunk are issued as soon as the conversion has consumed them, so that their latency
-            // (long while the tensor pipe is busy with the next tile) overlaps this chunk's stores.
-            uint32_t r0[32], r1[32];
-            auto issue_loads = [&](int k) {
+            // All of this warp's accumulator columns are fetched at once (kLoads x 32 registers) and
+            // the buffer is handed back as soon as they have landed; conversion and stores follow
+            // from registers. tcgen05.ld queues behind the tensor-core instructions already issued,
+            // so one exposed wait per tile is the best that can be had.
+            constexpr int kLoadsPerChunk = (OUT == STWQ_OUT_BF16) ? 2 : 1;
+            constexpr int kLoads = kMyChunks * kLoadsPerChunk;
+            uint32_t racc[kLoads][32];
+#pragma unroll
+            for (int k = 0; k < kMyChunks; ++k) {
                 const int c = sub + k * kSubs;
-                if (OUT == STWQ_OUT_BF16) {
-                    tmem_ld32(taddr + (uint32_t)(c * 64), r0);
-                    tmem_ld32(taddr + (uint32_t)(c * 64 + 32), r1);
-                } else {
-                    tmem_ld32(taddr + (uint32_t)(c * 32), r0);
-                }
-            };
-            issue_loads(0);
+#pragma unroll
+                for (int h = 0; h < kLoadsPerChunk; ++h)
+                    tmem_ld32(taddr + (uint32_t)(c * kChunkCols + h * 32), racc[k * kLoadsPerChunk + h]);
+            }
+            tmem_ld_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
 #pragma unroll
             for (int k = 0; k < kMyChunks; ++k, ++nstore) {
                 const int c = sub + k * kSubs;
                 const int col0 = n0 + c * kChunkCols;
                 const float* csw = my_sw + k * kChunkCols;
                 const float* cbi = my_bias + k * kChunkCols;
-                tmem_ld_wait();
-                if (k == kMyChunks - 1) {
-                    // every accumulator column of this warp is in registers: hand the buffer back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
-                }
+                const uint32_t* r0 = racc[k * kLoadsPerChunk];
+                const uint32_t* r1 = racc[k * kLoadsPerChunk + kLoadsPerChunk - 1];
                 uint32_t w[32];                           // this row's 128 bytes of output
                 const uint64_t st2 = pack_f2(st, st);
                 if (OUT == STWQ_OUT_BF16) {
@@ -308,7 +307,6 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 #pragma unroll
                     for (int j = 0; j < 32; ++j) w[j] = r0[j];
                 }
-                if (k + 1 < kMyChunks) issue_loads(k + 1);
                 if (STORE == 1) {
                     // straight from registers: this thread's 128 contiguous bytes of row `row`
                     if (row < p.M && col0 < p.N) {
