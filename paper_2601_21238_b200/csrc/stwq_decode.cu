@@ -387,35 +387,40 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
 }
 
-// Scratch for split-K: partial pieces for `items` work items and one counter per piece of an N slice.
-int ensure_scratch(stwq_ctx* ctx, int items, int tiles_n)
+}  // namespace
+
+// Scratch for split-K (shared by the few-row kernel and the tail of the tiled GEMM): a fixed
+// region of kSplitCounters arrival counters, zero between calls because the last arriver resets
+// its counter, followed by room for the int32 partial sums.
+int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial)
 {
-    const size_t partial_bytes = (size_t)items * 2 * kEpi * kPieceInts * sizeof(int32_t);
-    const size_t counter_bytes = (((size_t)tiles_n * 2 * kEpi * sizeof(uint32_t)) + 255) & ~(size_t)255;
+    constexpr size_t kSplitCounters = 16384;
+    constexpr size_t counter_bytes = kSplitCounters * sizeof(uint32_t);
+    if (n_counters > kSplitCounters) return STWQ_ERR_DIM;
     const size_t need = partial_bytes + counter_bytes;
-    if (ctx->ws_dec_bytes >= need && ctx->ws_dec_counter_bytes >= counter_bytes) return STWQ_OK;
-    if (ctx->ws_dec) {
-        cudaError_t e = cudaFree(ctx->ws_dec);            // synchronises
-        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->ws_dec = nullptr;
-        ctx->ws_dec_bytes = 0;
+    if (ctx->ws_dec_bytes < need) {
+        if (ctx->ws_dec) {
+            cudaError_t e = cudaFree(ctx->ws_dec);        // synchronises
+            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+            ctx->ws_dec = nullptr;
+            ctx->ws_dec_bytes = 0;
+        }
+        void* ptr = nullptr;
+        cudaError_t e = cudaMalloc(&ptr, need);
+        if (e == cudaSuccess) e = cudaMemset(ptr, 0, counter_bytes);
+        if (e != cudaSuccess) {
+            ctx->last_cuda_error = (int)e;
+            (void)cudaGetLastError();
+            if (ptr) cudaFree(ptr);
+            return STWQ_ERR_NOMEM;
+        }
+        ctx->ws_dec = ptr;
+        ctx->ws_dec_bytes = need;
     }
-    void* ptr = nullptr;
-    cudaError_t e = cudaMalloc(&ptr, need);
-    if (e == cudaSuccess) e = cudaMemset(ptr, 0, counter_bytes);   // counters sit first and start at zero
-    if (e != cudaSuccess) {
-        ctx->last_cuda_error = (int)e;
-        (void)cudaGetLastError();
-        if (ptr) cudaFree(ptr);
-        return STWQ_ERR_NOMEM;
-    }
-    ctx->ws_dec = ptr;
-    ctx->ws_dec_bytes = need;
-    ctx->ws_dec_counter_bytes = counter_bytes;
+    *counters = reinterpret_cast<uint32_t*>(ctx->ws_dec);
+    *partial = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctx->ws_dec) + counter_bytes);
     return STWQ_OK;
 }
-
-}  // namespace
 
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
@@ -448,10 +453,11 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.partial = nullptr;
     p.counters = nullptr;
     if (p.ksplit > 1) {
-        int rc = ensure_scratch(ctx, items, tiles_n);
+        int rc = stwq_split_ws(ctx, (size_t)items * 2 * kEpi * kPieceInts * sizeof(int32_t), (size_t)tiles_n * 2 * kEpi,
+                               &p.counters, &p.partial);
+        if (rc == STWQ_ERR_DIM)                            // more N slices than counters: no split-K path
+            return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
         if (rc != STWQ_OK) return rc;
-        p.counters = reinterpret_cast<uint32_t*>(ctx->ws_dec);
-        p.partial = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctx->ws_dec) + ctx->ws_dec_counter_bytes);
     }
     p.status = ctx->d_status;
     p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;

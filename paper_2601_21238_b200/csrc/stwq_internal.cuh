@@ -30,9 +30,8 @@ struct stwq_ctx {
     size_t ws_xq_bytes;
     void* ws_cal;              // workspace: calibration histograms and selection state
     size_t ws_cal_bytes;
-    void* ws_dec;              // workspace of the few-row path: split-K counters, then partial sums
+    void* ws_dec;              // split-K workspace: arrival counters, then int32 partial sums
     size_t ws_dec_bytes;
-    size_t ws_dec_counter_bytes;
     uint64_t configured_decode;
     int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
@@ -59,6 +58,8 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);
+
+int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial);
 
 static inline int stwq_cuda_fail(stwq_ctx* ctx, cudaError_t e)
 {

@@ -45,6 +45,12 @@ struct Gemm2Params {
     int tiles_n, num_tiles, num_kb;
     uint32_t* status;
     unsigned long long wait_limit_ns;
+    // Work units: the first `full_units` are whole tiles; then the last `tail_tiles` tiles come
+    // as `nsplit` units each, one per range of kb_per_split k-blocks (split-K for the last,
+    // partly filled wave). num_units = full_units + tail_tiles * nsplit.
+    int full_units, num_units, nsplit, kb_per_split;
+    int32_t* partial;          // [tail tile][split][rank][warp][128 x 32 lanes] int32
+    uint32_t* counters;        // [tail tile][rank][warp]
     void* Y;                   // used by the direct-store epilogue
     int y_vec32;               // Y base and row pitch are 32-byte aligned: 256-bit stores are legal
 };
@@ -72,6 +78,31 @@ struct Smem2 {
 // ---------------------------------------------------------------------------- kernel
 // OUT: element type of Y (STWQ_OUT_*); ACT: activation. One staging chunk is 32 rows x 128 bytes:
 // 64 bf16 columns or 32 fp32 / int32 columns.
+struct Unit {
+    int tile, kb0, kb1, split, tail;    // tail = index among the split tiles, -1 for a whole tile
+};
+__device__ __forceinline__ Unit decode_unit(const Gemm2Params& p, int u)
+{
+    Unit w;
+    if (u < p.full_units) {
+        w.tile = u; w.kb0 = 0; w.kb1 = p.num_kb; w.split = 0; w.tail = -1;
+    } else {
+        const int j = u - p.full_units;
+        w.tail = j / p.nsplit;
+        w.split = j % p.nsplit;
+        w.tile = p.full_units + w.tail;
+        w.kb0 = w.split * p.kb_per_split;
+        w.kb1 = min(w.kb0 + p.kb_per_split, p.num_kb);
+    }
+    return w;
+}
+__device__ __forceinline__ uint4 ld_cg_v4(const void* ptr)
+{
+    uint4 v;
+    asm volatile("ld.global.cg.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(ptr) : "memory");
+    return v;
+}
+
 // STORE: see Smem2.
 template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
 __global__ void __launch_bounds__(64 + 32 * EPI, 1)
@@ -137,10 +168,12 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // (barriers, tensor memory, cluster handshake) may have run while that kernel drained;
             // its codes are read only from here on
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs) {
+            for (int u = pair; ok && u < p.num_units; u += num_pairs) {
+                const Unit w = decode_unit(p, u);
+                const int tile = w.tile;
                 const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
                 const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
@@ -164,13 +197,14 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             constexpr uint32_t idesc = make_idesc_i8(2 * kBM, BN);
             uint32_t it = 0, t = 0;
             bool ok = true;
-            for (int tile = pair; ok && tile < p.num_tiles; tile += num_pairs, ++t) {
+            for (int u = pair; ok && u < p.num_units; u += num_pairs, ++t) {
+                const Unit w = decode_unit(p, u);
                 const int acc = t & 1;
                 const uint32_t aph = (t >> 1) & 1u;
                 if (!mbar_wait(bar_tempty(acc), aph ^ 1u, abort_flag, limit)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
-                for (int kb = 0; kb < p.num_kb; ++kb, ++it) {
+                for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(bar_full(s), ph, abort_flag, limit)) { ok = false; break; }
@@ -179,7 +213,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const uint64_t b_desc = make_smem_desc(base + L::kOffB + s * L::kBBytes);
 #pragma unroll
                     for (int k = 0; k < kBK / 32; ++k)
-                        tc_mma_i8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        tc_mma_i8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kb != w.kb0 || k != 0) ? 1u : 0u);
                     tc_commit_pair(bar_empty(s));
                 }
                 if (ok) tc_commit_pair(bar_tfull(acc));
@@ -201,7 +235,9 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         constexpr int kElem = (OUT == STWQ_OUT_BF16) ? 2 : 4;
         uint32_t t = 0, nstore = 0;
         bool ok = true;
-        for (int tile = pair; tile < p.num_tiles; tile += num_pairs, ++t) {
+        for (int u = pair; u < p.num_units; u += num_pairs, ++t) {
+            const Unit wu = decode_unit(p, u);
+            const int tile = wu.tile;
             const int acc = t & 1;
             const uint32_t aph = (t >> 1) & 1u;
             const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
@@ -253,6 +289,42 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(tempty0 + 8u * acc);
+            if (wu.tail >= 0) {
+                // One of nsplit partial sums of a tail tile: publish this warp's piece (lane-interleaved,
+                // 512 contiguous bytes per instruction), then count arrivals; the last warp to arrive for
+                // this piece adds all pieces up and carries on with the epilogue, the others are done.
+                // No CTA waits for another, and the sum of integers does not depend on the order.
+                constexpr int kPieceInts = kLoads * 32 * 32;
+                const size_t piece0 = (((size_t)wu.tail * p.nsplit) * 2 + rank) * EPI + ew;
+                const size_t piece_stride = (size_t)2 * EPI;
+                int32_t* mine = p.partial + (piece0 + (size_t)wu.split * piece_stride) * kPieceInts;
+#pragma unroll
+                for (int l = 0; l < kLoads; ++l)
+#pragma unroll
+                    for (int g = 0; g < 8; ++g) st_global_v4(mine + ((size_t)(l * 8 + g) * 32 + lane) * 4, racc[l] + g * 4);
+                __threadfence();
+                __syncwarp();
+                uint32_t* counter = p.counters + ((size_t)wu.tail * 2 + rank) * EPI + ew;
+                uint32_t old = 0;
+                if (lane == 0) {
+                    old = atomicAdd(counter, 1u);
+                    if (old == (uint32_t)p.nsplit - 1u) *counter = 0u;    // all have arrived: ready for the next call
+                }
+                old = __shfl_sync(0xffffffffu, old, 0);
+                if (old != (uint32_t)p.nsplit - 1u) continue;
+                __threadfence();
+                for (int s2 = 0; s2 < p.nsplit; ++s2) {
+                    if (s2 == wu.split) continue;         // this warp's own piece is still in its registers
+                    const int32_t* src = p.partial + (piece0 + (size_t)s2 * piece_stride) * kPieceInts;
+#pragma unroll
+                    for (int l = 0; l < kLoads; ++l)
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const uint4 a = ld_cg_v4(src + ((size_t)(l * 8 + g) * 32 + lane) * 4);
+                            racc[l][g * 4 + 0] += a.x; racc[l][g * 4 + 1] += a.y; racc[l][g * 4 + 2] += a.z; racc[l][g * 4 + 3] += a.w;
+                        }
+                }
+            }
 #pragma unroll
             for (int k = 0; k < kMyChunks; ++k, ++nstore) {
                 const int c = sub + k * kSubs;
@@ -420,7 +492,7 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
         ctx->max_pairs = n < ctx->sm_count / 2 ? n : ctx->sm_count / 2;
     }
     int pairs = ctx->max_pairs;
-    if (p.num_tiles < pairs) pairs = p.num_tiles;
+    if (p.num_units < pairs) pairs = p.num_units;
     cfg.gridDim = dim3((unsigned)(2 * pairs), 1, 1);
     cfg.numAttrs = dependent ? 2 : 1;
     cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, p);
@@ -483,6 +555,49 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.num_kb = (K + kBK - 1) / kBK;
     p.status = ctx->d_status;
     p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
+
+    // The last wave of a static tile schedule is partly empty unless the tile count divides by
+    // the number of pairs. When at most half the pairs would have work in it, its tiles can be cut
+    // along K into nsplit units each, so that the wave costs 1 / nsplit of a tile time. The price
+    // is the exchange of partial sums through scratch memory: 256 KB written per unit and as much
+    // read back, all at the end of the kernel when nothing overlaps it (measured: about 4 us of
+    // latency plus 0.12 us per unit at ~5 TB/s of L2 traffic), against about 0.38 us per k-block
+    // saved. For the 170-700 tile problems of the VAR / MAR layers this does not pay; it does for
+    // problems of a few tiles with long K.
+    p.full_units = p.num_tiles;
+    p.num_units = p.num_tiles;
+    p.nsplit = 1;
+    p.kb_per_split = p.num_kb;
+    p.partial = nullptr;
+    p.counters = nullptr;
+    const int pairs = ctx->max_pairs > 0 ? ctx->max_pairs : ctx->sm_count / 2;
+    const int tail = p.num_tiles % pairs;
+    if (bn == 256 && tail > 0 && 2 * tail <= pairs && ctx->force_ksplit >= 0) {
+        int nsplit = pairs / tail;
+        if (nsplit > p.num_kb / 4) nsplit = p.num_kb / 4;
+        if (nsplit > 8) nsplit = 8;
+        if (nsplit >= 2) {
+            const double saved_us = (1.0 - 1.0 / nsplit) * p.num_kb * 0.38;
+            const double cost_us = 4.0 + 0.12 * tail * nsplit;
+            if (saved_us < 1.5 * cost_us) nsplit = 1;
+        }
+        if (ctx->force_ksplit > 0) nsplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
+        if (nsplit >= 2) {
+            const int kbps = (p.num_kb + nsplit - 1) / nsplit;
+            nsplit = (p.num_kb + kbps - 1) / kbps;             // every range holds at least one k-block
+            const size_t piece_bytes = (size_t)4 * 32 * 32 * sizeof(int32_t);      // 32 rows x 128 columns
+            int rc = stwq_split_ws(ctx, (size_t)tail * nsplit * 2 * 8 * piece_bytes, (size_t)tail * 2 * 8, &p.counters,
+                                   &p.partial);
+            if (rc == STWQ_OK && nsplit >= 2) {
+                p.full_units = p.num_tiles - tail;
+                p.nsplit = nsplit;
+                p.kb_per_split = kbps;
+                p.num_units = p.full_units + tail * nsplit;
+            } else if (rc != STWQ_ERR_DIM) {
+                return rc;
+            }
+        }
+    }
 
     CUtensorMap tmA, tmB, tmY;
     int rc = stwq_encode_2d(ctx, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kBK, kBM);

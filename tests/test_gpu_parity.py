@@ -353,3 +353,37 @@ def test_decode_split_k_is_exact_and_repeatable(gpu, shape, ksplit):
             assert_close(_run_qlinear(gpu, L, par, X, pos, "bf16", act=2, path=2), ref, RTOL["bf16"], "decode bf16")
     finally:
         gpu.ctx.stwq_set_option(102, 0)
+
+
+@pytest.mark.parametrize("ksplit", [-1, 0, 3, 7])
+@pytest.mark.parametrize("shape", [(600, 520, 2064), (257, 1024, 1024), (1300, 264, 4096)])
+def test_tiled_gemm_split_tail_is_exact_and_repeatable(gpu, shape, ksplit):
+    """The tiled GEMM cuts the tiles of a partly filled last wave along K (here: every tile, the
+    problems being smaller than one wave) and adds the int32 partial sums through scratch memory.
+    -1 switches the split off, 0 lets the library choose, 3 and 7 force the number of K ranges."""
+    M, N, K = shape
+    Xq = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    Wq = rng.integers(-128, 128, (N, K)).astype(np.int8)
+    pos = rng.integers(0, 5, M).astype(np.int32)
+    s_tok = rng.uniform(0.01, 0.1, 5).astype(np.float32)
+    s_w = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = (0.5 * rng.standard_normal(N)).astype(np.float32)
+    acc = oracle.igemm(Xq, Wq)
+    Yref, mag = oracle.epilogue(acc, pos, s_tok, s_w, bias, 1)
+    ref = {"Y": Yref, "mag": mag}
+    d = [gpu.T(a) for a in (Xq, pos, Wq, s_w, s_tok, bias)]
+    gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 1)
+    gpu.ctx.stwq_set_option(102, ksplit)
+    try:
+        for _ in range(2):
+            Yi = _out_tensor(gpu, M, N, "int32")
+            gpu.ctx.qlinear_q(d[0], None, d[2], None, None, None, 0, gpu.B.OUT_INT32, Yi)
+            np.testing.assert_array_equal(Yi.cpu().numpy(), acc)
+            for out in ("bf16", "fp32"):
+                Y = _out_tensor(gpu, M, N, out)
+                gpu.ctx.qlinear_q(d[0], d[1], d[2], d[3], d[4], d[5], 1, _out_code(gpu, out), Y)
+                assert gpu.ctx.stwq_device_status() == 0
+                assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"split tail {out}")
+    finally:
+        gpu.ctx.stwq_set_option(102, 0)
+        gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
