@@ -450,22 +450,39 @@ def reference_arm(args):
         return
     import oracle
     layers = wl.config_layers(args.config)
-    rows = args.ref_rows
-    prepared = []
-    for L in layers:
-        W = wl.weights(L)
-        s_ch = stand_in_channel_scales(L) if L.use_gps else None
-        Wq, s_w = oracle.gps_fold(W, s_ch, L.bits)
-        Xc, pc = wl.calibration(L, 2)
-        s_tok = oracle.stwq_calibrate(Xc, pc, L.P, s_ch, L.bits, PCT)
-        X = wl.activations(L, rows=slice(0, rows))
-        pos = wl.positions(L)[:rows]
-        prepared.append((L, X, pos, Wq, s_w, s_tok, s_ch, wl.bias(L)))
+
+    def prepare(rows):
+        prepared = []
+        for L in layers:
+            W = wl.weights(L)
+            s_ch = stand_in_channel_scales(L) if L.use_gps else None
+            Wq, s_w = oracle.gps_fold(W, s_ch, L.bits)
+            Xc, pc = wl.calibration(L, 2)
+            s_tok = oracle.stwq_calibrate(Xc, pc, L.P, s_ch, L.bits, PCT)
+            X = wl.activations(L, rows=slice(0, rows))
+            pos = wl.positions(L)[:rows]
+            prepared.append((L, X, pos, Wq, s_w, s_tok, s_ch, wl.bias(L)))
+        return prepared
+
+    def run(prepared):
+        for L, X, pos, Wq, s_w, s_tok, s_ch, b in prepared:
+            oracle.qlinear(X, pos, Wq, s_w, s_tok, s_ch, b, L.bits, L.act)
+
+    # The sample per step is sized so that warm-up + steps stay within about two minutes: a probe
+    # at --ref-rows rows gives the oracle's rate on this host, the rows per step follow from it.
+    probe = prepare(args.ref_rows)
+    run(probe)
+    t0 = time.perf_counter()
+    run(probe)
+    t_probe = time.perf_counter() - t0
+    budget_s = 120.0
+    rows = int(args.ref_rows * budget_s / max(1, args.steps + args.warmup) / max(t_probe, 1e-6))
+    rows = max(4, min(rows, args.ref_rows * 8, min(L.M for L in layers)))
+    prepared = probe if rows == args.ref_rows else prepare(rows)
     ops = sum(2.0 * rows * L.N * L.K for L in layers)
 
     def step():
-        for L, X, pos, Wq, s_w, s_tok, s_ch, b in prepared:
-            oracle.qlinear(X, pos, Wq, s_w, s_tok, s_ch, b, L.bits, L.act)
+        run(prepared)
 
     for _ in range(args.warmup):
         step()

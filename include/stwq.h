@@ -123,8 +123,13 @@ int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t
  *     Y[m,n] = act(z)  cast to out_dtype
  * bias == NULL means zero. out_dtype STWQ_OUT_INT32 stores acc itself.
  * Calls with few rows (M <= 256, the raster-order decode step where a batch advances one
- * token position at a time) are routed to a bandwidth-bound variant that streams Wq once
- * across all SMs; the result is the same.
+ * token position at a time) are routed to a variant that streams Wq once across all SMs, split
+ * along K where N alone does not give every SM work; the result is the same. That variant, and
+ * the tiled GEMM when it splits a partly filled last wave along K, keep int32 partial sums in
+ * context workspace that is allocated (synchronously) the first time a shape needs it.
+ * The two kernels of a call are launched as programmatic dependents of their predecessor in the
+ * stream; each waits for that predecessor to complete before its first dependent access, so the
+ * effects are ordered as with ordinary launches.
  * Extra alignment: N a multiple of 8 for bf16 output gives vector stores; other N work but
  * store element by element.
  */
