@@ -7,7 +7,16 @@
 // contiguous 128-byte request. The span of a warp never changes, so the 16 reciprocal channel
 // scales a lane needs stay in registers for the whole kernel; the per-row reciprocal token scale
 // is one IEEE division per row and warp.
+//
+// Large inputs take a second kernel with the same arithmetic (quantize_ring_kernel below): one
+// persistent CTA per SM whose producer thread streams 16-row x 256-column fp32 tiles of X into a
+// ten-stage shared-memory ring with TMA (160 KB in flight per SM, which no register-based scheme
+// reaches), while eight consumer warps convert them; the reciprocal channel and position scales
+// live in shared-memory tables computed once per CTA behind the first loads.
+#include <cuda.h>
+
 #include "stwq_internal.cuh"
+#include "stwq_ptx.cuh"
 
 namespace {
 
@@ -114,12 +123,212 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
     }
 }
 
+// ---------------------------------------------------------------------------- TMA ring variant
+constexpr int kTR = 16;                      // rows per tile
+constexpr int kTC = 256;                     // columns per tile (1 KB of fp32 per row)
+constexpr int kTileBytes = kTR * kTC * 4;    // 16 KB
+constexpr int kRingStages = 10;
+constexpr int kConsumerWarps = 8;            // two rows of a tile each
+constexpr int kRingThreads = 32 * (1 + kConsumerWarps);
+constexpr int kRingMaxK = 8192;              // table of reciprocal channel scales: 32 KB
+constexpr int kRingMaxP = 2048;              // table of reciprocal position scales: 8 KB
+constexpr int kRingOffRc = kRingStages * kTileBytes;
+constexpr int kRingOffRt = kRingOffRc + kRingMaxK * 4;
+constexpr int kRingOffBars = kRingOffRt + kRingMaxP * 4;
+constexpr int kRingSmem = kRingOffBars + 2 * kRingStages * 8 + 16 + 128;
+
+__global__ void __launch_bounds__(kRingThreads, 1)
+quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __restrict__ pos_ids, int64_t M, int K,
+                     const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin, int qmax,
+                     int8_t* __restrict__ Xq, int col_blocks, int num_tiles, int step_rb, int step_cb,
+                     uint32_t* __restrict__ status, unsigned long long limit)
+{
+    using namespace stwq_ptx;
+    asm volatile("griddepcontrol.wait;" ::: "memory");               // see quantize_kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t base = (raw + 127u) & ~127u;
+    uint8_t* smem = smem_raw + (base - raw);
+    float* rc_s = reinterpret_cast<float*>(smem + kRingOffRc);
+    float* rt_s = reinterpret_cast<float*>(smem + kRingOffRt);
+    const uint32_t bars = base + kRingOffBars;
+    auto bar_full = [&](int s) { return bars + 8u * s; };
+    auto bar_empty = [&](int s) { return bars + 8u * (kRingStages + s); };
+    volatile uint32_t* abort_flag = reinterpret_cast<volatile uint32_t*>(smem + kRingOffBars + 2 * kRingStages * 8);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kRingStages; ++s) {
+            mbar_init(bar_full(s), 1);
+            mbar_init(bar_empty(s), kConsumerWarps);
+        }
+        *abort_flag = 0u;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            // (rb, cb) = row block and column block of tile t, advanced without divisions
+            int rb = (int)blockIdx.x / col_blocks, cb = (int)blockIdx.x % col_blocks;
+            for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+                const int s = it % kRingStages;
+                const uint32_t ph = (it / kRingStages) & 1u;
+                if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
+                mbar_expect_tx(bar_full(s), kTileBytes);
+                tma_load_2d(base + s * kTileBytes, &tmX, cb * kTC, rb * kTR, bar_full(s));
+                rb += step_rb;
+                cb += step_cb;
+                if (cb >= col_blocks) { cb -= col_blocks; ++rb; }
+            }
+            if (!ok) {
+                const uint32_t first = it > (uint32_t)kRingStages ? it - kRingStages : 0u;
+                for (uint32_t j = first; j < it; ++j) {
+                    const unsigned long long t0 = globaltimer_ns();
+                    while (!mbar_try_wait(bar_full(j % kRingStages), (j / kRingStages) & 1u))
+                        if (globaltimer_ns() - t0 > limit) break;
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ consumers
+        const int cw = warp - 1;                           // rows 2 cw and 2 cw + 1 of every tile
+        const int ct = threadIdx.x - 32;
+        for (int i = ct; i < K; i += 32 * kConsumerWarps) rc_s[i] = s_ch != nullptr ? __fdiv_rn(1.0f, s_ch[i]) : 1.0f;
+        for (int i = ct; i < P; i += 32 * kConsumerWarps) rt_s[i] = __fdiv_rn(1.0f, s_tok[i]);
+        asm volatile("bar.sync 1, %0;" ::"n"(32 * kConsumerWarps) : "memory");
+        uint32_t it = 0;
+        int t = blockIdx.x;
+        int rb = (int)blockIdx.x / col_blocks, cb = (int)blockIdx.x % col_blocks;
+        int pos_next[2] = {0, 0};
+        if (t < num_tiles) {
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int64_t row = (int64_t)rb * kTR + 2 * cw + rr;
+                pos_next[rr] = row < M ? pos_ids[row] : 0;
+            }
+        }
+        for (; t < num_tiles; t += gridDim.x, ++it) {
+            const int s = it % kRingStages;
+            const uint32_t ph = (it / kRingStages) & 1u;
+            const int64_t row0 = (int64_t)rb * kTR + 2 * cw;
+            const int colb = cb * kTC;
+            const int pos_cur[2] = {pos_next[0], pos_next[1]};
+            rb += step_rb;
+            cb += step_cb;
+            if (cb >= col_blocks) { cb -= col_blocks; ++rb; }
+            if (t + (int)gridDim.x < num_tiles) {          // positions of the next tile's rows, ahead of time
+#pragma unroll
+                for (int rr = 0; rr < 2; ++rr) {
+                    const int64_t row = (int64_t)rb * kTR + 2 * cw + rr;
+                    pos_next[rr] = row < M ? pos_ids[row] : 0;
+                }
+            }
+            bool ok = mbar_wait(bar_full(s), ph, abort_flag, limit);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            const uint8_t* tile = smem + s * kTileBytes;
+#pragma unroll
+            for (int rr = 0; rr < 2; ++rr) {
+                const int64_t row = row0 + rr;
+                if (row >= M) continue;
+                const int p = pos_cur[rr];
+                const bool pok = (p >= 0) && (p < P);
+                const float rt = pok ? rt_s[p] : 0.0f;
+                if (!pok && lane == 0 && colb == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+#pragma unroll
+                for (int j = 0; j < 2; ++j) {
+                    const int cl = 128 * j + 4 * lane;
+                    const int col = colb + cl;
+                    if (col < K) {
+                        const float4 v = *reinterpret_cast<const float4*>(tile + (2 * cw + rr) * (kTC * 4) + cl * 4);
+                        const float4 rc = *reinterpret_cast<const float4*>(rc_s + col);
+                        int q0 = stwq_code(__fmul_rn(__fmul_rn(v.x, rc.x), rt), qmin, qmax);
+                        int q1 = stwq_code(__fmul_rn(__fmul_rn(v.y, rc.y), rt), qmin, qmax);
+                        int q2 = stwq_code(__fmul_rn(__fmul_rn(v.z, rc.z), rt), qmin, qmax);
+                        int q3 = stwq_code(__fmul_rn(__fmul_rn(v.w, rc.w), rt), qmin, qmax);
+                        if (!pok) q0 = q1 = q2 = q3 = 0;
+                        const uint32_t packed = (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) |
+                                                ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
+                        *reinterpret_cast<uint32_t*>(Xq + row * K + col) = packed;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty(s));
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(status, STWQ_DEV_TIMEOUT);
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                const float* s_tok, int P, int qmin, int qmax, int8_t* Xq, bool dependent, cudaStream_t st)
+{
+    CUtensorMap tmX;
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+    cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)M};
+    cuuint64_t gstride[1] = {(cuuint64_t)K * 4};
+    cuuint32_t box[2] = {(cuuint32_t)kTC, (cuuint32_t)kTR};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(&tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = (int)r;
+        return STWQ_ERR_CUDA;
+    }
+    if (!ctx->quant_ring_configured) {
+        cudaError_t e = cudaFuncSetAttribute(quantize_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem);
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->quant_ring_configured = 1;
+    }
+    const int col_blocks = (K + kTC - 1) / kTC;
+    const int num_tiles = (int)(((M + kTR - 1) / kTR) * col_blocks);       // the caller has checked that this fits
+    const int grid = num_tiles < ctx->sm_count ? num_tiles : ctx->sm_count;
+    cudaLaunchConfig_t cfg = {};
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kRingThreads, 1, 1);
+    cfg.dynamicSmemBytes = kRingSmem;
+    cfg.stream = st;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 1 : 0;
+    const unsigned long long limit = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, quantize_ring_kernel, tmX, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq,
+                                       col_blocks, num_tiles, grid / col_blocks, grid % col_blocks, ctx->d_status, limit);
+    ctx->launches += 1;
+    if (e == cudaSuccess) e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
 }  // namespace
 
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
                          bool dependent, cudaStream_t st)
 {
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    // the ring kernel's tables bound K and P; it only wins (by 5-10 %) on inputs of hundreds of MB,
+    // where the output no longer stays in L2 and more bytes in flight help
+    const bool ring_ok = K <= kRingMaxK && P <= kRingMaxP && ctx->encode_tiled != nullptr && M < ((int64_t)1 << 29);
+    bool ring = ring_ok && (int64_t)M * K >= ((int64_t)1 << 27);
+    if (ctx->debug == 7) ring = false;                    // tuning: force one or the other
+    if (ctx->debug == 8) ring = ring_ok;
+    if (ring) return launch_ring(ctx, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, dependent, st);
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
     // As many warps as can be resident, then the row stride is shrunk so that every warp sees the
@@ -139,7 +348,6 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     // total warps must be rows_in_flight * spans and a multiple of warps_per_block
     while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
     const int64_t blocks = rows_in_flight * spans / warps_per_block;
-    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

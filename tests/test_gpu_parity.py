@@ -62,10 +62,15 @@ def test_quantize_codes_bit_exact(gpu, bits, shape):
         X[2] = 1e4                                          # saturating row
     for sc in (s_ch, None):
         ref = oracle.quantize(X, pos, sc, s_tok, bits)
-        Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
-        gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
-        assert gpu.ctx.stwq_device_status() == 0
-        np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
+        for variant in (7, 8):              # the register-streaming kernel, the TMA-ring kernel
+            Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+            gpu.ctx.stwq_set_option(101, variant)
+            try:
+                gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
+                assert gpu.ctx.stwq_device_status() == 0
+            finally:
+                gpu.ctx.stwq_set_option(101, 0)
+            np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
 
 
 def test_quantize_reports_bad_position_and_zeroes_the_row(gpu):
@@ -74,15 +79,20 @@ def test_quantize_reports_bad_position_and_zeroes_the_row(gpu):
     pos = rng.integers(0, P, M).astype(np.int32)
     pos[5], pos[11] = P, -1
     s_tok = rng.uniform(0.01, 0.1, P).astype(np.float32)
-    Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
-    gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), None, gpu.T(s_tok), 8, Xq)
-    assert gpu.ctx.stwq_device_status() == -8               # STWQ_ERR_POS_RANGE
-    assert gpu.ctx.stwq_device_status() == 0                # reading clears it
-    got = Xq.cpu().numpy()
-    assert not got[5].any() and not got[11].any()
-    good = np.ones(M, bool)
-    good[[5, 11]] = False
-    np.testing.assert_array_equal(got[good], oracle.quantize(X[good], pos[good], None, s_tok, 8))
+    for variant in (7, 8):
+        Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+        gpu.ctx.stwq_set_option(101, variant)
+        try:
+            gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), None, gpu.T(s_tok), 8, Xq)
+        finally:
+            gpu.ctx.stwq_set_option(101, 0)
+        assert gpu.ctx.stwq_device_status() == -8               # STWQ_ERR_POS_RANGE
+        assert gpu.ctx.stwq_device_status() == 0                # reading clears it
+        got = Xq.cpu().numpy()
+        assert not got[5].any() and not got[11].any()
+        good = np.ones(M, bool)
+        good[[5, 11]] = False
+        np.testing.assert_array_equal(got[good], oracle.quantize(X[good], pos[good], None, s_tok, 8))
 
 
 def test_host_argument_validation(gpu):
