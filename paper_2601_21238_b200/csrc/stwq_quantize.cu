@@ -32,6 +32,30 @@ __device__ __forceinline__ float4 ld_stream(const float* p)
     return v;
 }
 
+// Four values -> four packed codes. u = (x * rc) * rt in two IEEE multiplies, round to nearest
+// even (cvt.rni: NaN -> 0, +-Inf and huge values -> INT_MIN / INT_MAX), then clamp and pack. With
+// 8 bits the clamp is the saturation of cvt.pack (two instructions for four codes); with fewer
+// bits the integers are clamped first. A row with a bad position gets rt = 0, which makes every
+// finite u zero and every other u NaN, i.e. code 0 throughout.
+template <bool B8>
+__device__ __forceinline__ uint32_t quantize4(const float4 v, const float4 rc, float rt, int qmin, int qmax)
+{
+    int q0 = __float2int_rn(__fmul_rn(__fmul_rn(v.x, rc.x), rt));
+    int q1 = __float2int_rn(__fmul_rn(__fmul_rn(v.y, rc.y), rt));
+    int q2 = __float2int_rn(__fmul_rn(__fmul_rn(v.z, rc.z), rt));
+    int q3 = __float2int_rn(__fmul_rn(__fmul_rn(v.w, rc.w), rt));
+    if (!B8) {
+        q0 = max(min(q0, qmax), qmin);
+        q1 = max(min(q1, qmax), qmin);
+        q2 = max(min(q2, qmax), qmin);
+        q3 = max(min(q3, qmax), qmin);
+    }
+    uint32_t hi, packed;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(packed) : "r"(q1), "r"(q0), "r"(hi));
+    return packed;
+}
+
 __device__ __forceinline__ void load_row(const float* xrow, int col0, int K, float4 (&v)[4])
 {
 #pragma unroll
@@ -53,6 +77,7 @@ __device__ __forceinline__ float row_scale(const int32_t* pos_ids, const float* 
 // flight while the current row is converted, and the first row's loads are issued before the
 // reciprocal channel scales are computed, so that a warp that only sees a few rows (M of a few
 // thousand) does not serialise two memory round trips and sixteen divisions in front of them.
+template <bool B8>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
                 const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin,
@@ -103,16 +128,9 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int c = col0 + j * 128;
-            if (c < K) {
-                int q0 = stwq_code(__fmul_rn(__fmul_rn(v[j].x, rc[j * 4 + 0]), rt), qmin, qmax);
-                int q1 = stwq_code(__fmul_rn(__fmul_rn(v[j].y, rc[j * 4 + 1]), rt), qmin, qmax);
-                int q2 = stwq_code(__fmul_rn(__fmul_rn(v[j].z, rc[j * 4 + 2]), rt), qmin, qmax);
-                int q3 = stwq_code(__fmul_rn(__fmul_rn(v[j].w, rc[j * 4 + 3]), rt), qmin, qmax);
-                if (!ok) q0 = q1 = q2 = q3 = 0;
-                const uint32_t packed = (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) |
-                                        ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
-                *reinterpret_cast<uint32_t*>(qrow + c) = packed;
-            }
+            if (c < K)
+                *reinterpret_cast<uint32_t*>(qrow + c) =
+                    quantize4<B8>(v[j], make_float4(rc[j * 4 + 0], rc[j * 4 + 1], rc[j * 4 + 2], rc[j * 4 + 3]), rt, qmin, qmax);
         }
         if (!more) break;
 #pragma unroll
@@ -128,7 +146,7 @@ constexpr int kTR = 16;                      // rows per tile
 constexpr int kTC = 256;                     // columns per tile (1 KB of fp32 per row)
 constexpr int kTileBytes = kTR * kTC * 4;    // 16 KB
 constexpr int kRingStages = 10;
-constexpr int kConsumerWarps = 8;            // two rows of a tile each
+constexpr int kConsumerWarps = 16;           // one row of a tile each
 constexpr int kRingThreads = 32 * (1 + kConsumerWarps);
 constexpr int kRingMaxK = 8192;              // table of reciprocal channel scales: 32 KB
 constexpr int kRingMaxP = 2048;              // table of reciprocal position scales: 8 KB
@@ -137,6 +155,7 @@ constexpr int kRingOffRt = kRingOffRc + kRingMaxK * 4;
 constexpr int kRingOffBars = kRingOffRt + kRingMaxP * 4;
 constexpr int kRingSmem = kRingOffBars + 2 * kRingStages * 8 + 16 + 128;
 
+template <bool B8>
 __global__ void __launch_bounds__(kRingThreads, 1)
 quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __restrict__ pos_ids, int64_t M, int K,
                      const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin, int qmax,
@@ -198,7 +217,7 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
         }
     } else {
         // ------------------------------------------------------------------ consumers
-        const int cw = warp - 1;                           // rows 2 cw and 2 cw + 1 of every tile
+        const int cw = warp - 1;                           // row cw of every tile
         const int ct = threadIdx.x - 32;
         for (int i = ct; i < K; i += 32 * kConsumerWarps) rc_s[i] = s_ch != nullptr ? __fdiv_rn(1.0f, s_ch[i]) : 1.0f;
         for (int i = ct; i < P; i += 32 * kConsumerWarps) rt_s[i] = __fdiv_rn(1.0f, s_tok[i]);
@@ -206,39 +225,29 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
         uint32_t it = 0;
         int t = blockIdx.x;
         int rb = (int)blockIdx.x / col_blocks, cb = (int)blockIdx.x % col_blocks;
-        int pos_next[2] = {0, 0};
+        int pos_next = 0;
         if (t < num_tiles) {
-#pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                const int64_t row = (int64_t)rb * kTR + 2 * cw + rr;
-                pos_next[rr] = row < M ? pos_ids[row] : 0;
-            }
+            const int64_t row = (int64_t)rb * kTR + cw;
+            pos_next = row < M ? pos_ids[row] : 0;
         }
         for (; t < num_tiles; t += gridDim.x, ++it) {
             const int s = it % kRingStages;
             const uint32_t ph = (it / kRingStages) & 1u;
-            const int64_t row0 = (int64_t)rb * kTR + 2 * cw;
+            const int64_t row = (int64_t)rb * kTR + cw;
             const int colb = cb * kTC;
-            const int pos_cur[2] = {pos_next[0], pos_next[1]};
+            const int p = pos_next;
             rb += step_rb;
             cb += step_cb;
             if (cb >= col_blocks) { cb -= col_blocks; ++rb; }
-            if (t + (int)gridDim.x < num_tiles) {          // positions of the next tile's rows, ahead of time
-#pragma unroll
-                for (int rr = 0; rr < 2; ++rr) {
-                    const int64_t row = (int64_t)rb * kTR + 2 * cw + rr;
-                    pos_next[rr] = row < M ? pos_ids[row] : 0;
-                }
+            if (t + (int)gridDim.x < num_tiles) {          // position of the next tile's row, ahead of time
+                const int64_t rn = (int64_t)rb * kTR + cw;
+                pos_next = rn < M ? pos_ids[rn] : 0;
             }
             bool ok = mbar_wait(bar_full(s), ph, abort_flag, limit);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            const uint8_t* tile = smem + s * kTileBytes;
-#pragma unroll
-            for (int rr = 0; rr < 2; ++rr) {
-                const int64_t row = row0 + rr;
-                if (row >= M) continue;
-                const int p = pos_cur[rr];
+            if (row < M) {
+                const uint8_t* trow = smem + s * kTileBytes + cw * (kTC * 4);
                 const bool pok = (p >= 0) && (p < P);
                 const float rt = pok ? rt_s[p] : 0.0f;
                 if (!pok && lane == 0 && colb == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
@@ -247,16 +256,9 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
                     const int cl = 128 * j + 4 * lane;
                     const int col = colb + cl;
                     if (col < K) {
-                        const float4 v = *reinterpret_cast<const float4*>(tile + (2 * cw + rr) * (kTC * 4) + cl * 4);
+                        const float4 v = *reinterpret_cast<const float4*>(trow + cl * 4);
                         const float4 rc = *reinterpret_cast<const float4*>(rc_s + col);
-                        int q0 = stwq_code(__fmul_rn(__fmul_rn(v.x, rc.x), rt), qmin, qmax);
-                        int q1 = stwq_code(__fmul_rn(__fmul_rn(v.y, rc.y), rt), qmin, qmax);
-                        int q2 = stwq_code(__fmul_rn(__fmul_rn(v.z, rc.z), rt), qmin, qmax);
-                        int q3 = stwq_code(__fmul_rn(__fmul_rn(v.w, rc.w), rt), qmin, qmax);
-                        if (!pok) q0 = q1 = q2 = q3 = 0;
-                        const uint32_t packed = (uint32_t)(q0 & 0xff) | ((uint32_t)(q1 & 0xff) << 8) |
-                                                ((uint32_t)(q2 & 0xff) << 16) | ((uint32_t)(q3 & 0xff) << 24);
-                        *reinterpret_cast<uint32_t*>(Xq + row * K + col) = packed;
+                        *reinterpret_cast<uint32_t*>(Xq + row * K + col) = quantize4<B8>(v, rc, rt, qmin, qmax);
                     }
                 }
             }
@@ -289,10 +291,12 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
         ctx->last_cuda_error = (int)r;
         return STWQ_ERR_CUDA;
     }
-    if (!ctx->quant_ring_configured) {
-        cudaError_t e = cudaFuncSetAttribute(quantize_ring_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem);
+    const bool b8 = (qmin == -128);
+    auto kern = b8 ? quantize_ring_kernel<true> : quantize_ring_kernel<false>;
+    if (!(ctx->quant_ring_configured & (b8 ? 1 : 2))) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, kRingSmem);
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->quant_ring_configured = 1;
+        ctx->quant_ring_configured |= (b8 ? 1 : 2);
     }
     const int col_blocks = (K + kTC - 1) / kTC;
     const int num_tiles = (int)(((M + kTR - 1) / kTR) * col_blocks);       // the caller has checked that this fits
@@ -308,7 +312,7 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
     const unsigned long long limit = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quantize_ring_kernel, tmX, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmX, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq,
                                        col_blocks, num_tiles, grid / col_blocks, grid % col_blocks, ctx->d_status, limit);
     ctx->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
@@ -322,7 +326,7 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
                          bool dependent, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    // the ring kernel's tables bound K and P; it only wins (by 5-10 %) on inputs of hundreds of MB,
+    // the ring kernel's tables bound K and P; it only wins (by 15-20 %) on inputs of hundreds of MB,
     // where the output no longer stays in L2 and more bytes in flight help
     const bool ring_ok = K <= kRingMaxK && P <= kRingMaxP && ctx->encode_tiled != nullptr && M < ((int64_t)1 << 29);
     bool ring = ring_ok && (int64_t)M * K >= ((int64_t)1 << 27);
@@ -335,7 +339,7 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     // same number of rows (no ragged last pass).
     if (ctx->quant_blocks_per_sm <= 0) {
         int n = 0;
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel, kThreads, 0);
+        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel<true>, kThreads, 0);
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
         ctx->quant_blocks_per_sm = n > 0 ? n : 1;
     }
@@ -358,7 +362,7 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, quantize_kernel, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
+    cudaError_t e = cudaLaunchKernelEx(&cfg, bits == 8 ? quantize_kernel<true> : quantize_kernel<false>, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
                                        rows_in_flight, ctx->d_status);
     ctx->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
