@@ -9,9 +9,9 @@
 // is one IEEE division per row and warp.
 //
 // Large inputs take a second kernel with the same arithmetic (quantize_ring_kernel below): one
-// persistent CTA per SM whose producer thread streams 16-row x 256-column fp32 tiles of X into a
+// persistent CTA per SM whose producer thread streams 16 KB runs of the flat array X into a
 // ten-stage shared-memory ring with TMA (160 KB in flight per SM, which no register-based scheme
-// reaches), while eight consumer warps convert them; the reciprocal channel and position scales
+// reaches), while sixteen consumer warps convert them; the reciprocal channel and position scales
 // live in shared-memory tables computed once per CTA behind the first loads.
 #include <cuda.h>
 
@@ -142,11 +142,15 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
 }
 
 // ---------------------------------------------------------------------------- TMA ring variant
-constexpr int kTR = 16;                      // rows per tile
-constexpr int kTC = 256;                     // columns per tile (1 KB of fp32 per row)
-constexpr int kTileBytes = kTR * kTC * 4;    // 16 KB
+// X is dense, so a tile is simply 4096 consecutive floats of the flat array (16 KB of contiguous
+// DRAM, which streams a quarter faster than sixteen 1 KB pieces of sixteen rows: 6.0-6.4 against
+// 4.7-4.8 TB/s of reads with nobody consuming). The tensor map views X as [M K / 256, 256] and a
+// box is 16 of those rows. Every consumer thread owns two float4 slots of the tile and tracks the
+// (row, column) its slots fall on as the tile index advances, without divisions.
+constexpr int kTileFloats = 4096;
+constexpr int kTileBytes = kTileFloats * 4;  // 16 KB
 constexpr int kRingStages = 10;
-constexpr int kConsumerWarps = 16;           // one row of a tile each
+constexpr int kConsumerWarps = 16;           // 256 floats of a tile each
 constexpr int kRingThreads = 32 * (1 + kConsumerWarps);
 constexpr int kRingMaxK = 8192;              // table of reciprocal channel scales: 32 KB
 constexpr int kRingMaxP = 2048;              // table of reciprocal position scales: 8 KB
@@ -157,9 +161,9 @@ constexpr int kRingSmem = kRingOffBars + 2 * kRingStages * 8 + 16 + 128;
 
 template <bool B8>
 __global__ void __launch_bounds__(kRingThreads, 1)
-quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __restrict__ pos_ids, int64_t M, int K,
+quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __restrict__ pos_ids, int64_t total, int K,
                      const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin, int qmax,
-                     int8_t* __restrict__ Xq, int col_blocks, int num_tiles, int step_rb, int step_cb,
+                     int8_t* __restrict__ Xq, int num_tiles, int step_row, int step_col,
                      uint32_t* __restrict__ status, unsigned long long limit)
 {
     using namespace stwq_ptx;
@@ -194,17 +198,12 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
         if (lane == 0) {
             uint32_t it = 0;
             bool ok = true;
-            // (rb, cb) = row block and column block of tile t, advanced without divisions
-            int rb = (int)blockIdx.x / col_blocks, cb = (int)blockIdx.x % col_blocks;
             for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
                 const int s = it % kRingStages;
                 const uint32_t ph = (it / kRingStages) & 1u;
                 if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
                 mbar_expect_tx(bar_full(s), kTileBytes);
-                tma_load_2d(base + s * kTileBytes, &tmX, cb * kTC, rb * kTR, bar_full(s));
-                rb += step_rb;
-                cb += step_cb;
-                if (cb >= col_blocks) { cb -= col_blocks; ++rb; }
+                tma_load_2d(base + s * kTileBytes, &tmX, 0, t * 16, bar_full(s));   // rows past the end are zero-filled
             }
             if (!ok) {
                 const uint32_t first = it > (uint32_t)kRingStages ? it - kRingStages : 0u;
@@ -217,49 +216,69 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
         }
     } else {
         // ------------------------------------------------------------------ consumers
-        const int cw = warp - 1;                           // row cw of every tile
+        const int cw = warp - 1;
         const int ct = threadIdx.x - 32;
         for (int i = ct; i < K; i += 32 * kConsumerWarps) rc_s[i] = s_ch != nullptr ? __fdiv_rn(1.0f, s_ch[i]) : 1.0f;
         for (int i = ct; i < P; i += 32 * kConsumerWarps) rt_s[i] = __fdiv_rn(1.0f, s_tok[i]);
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kConsumerWarps) : "memory");
-        uint32_t it = 0;
-        int t = blockIdx.x;
-        int rb = (int)blockIdx.x / col_blocks, cb = (int)blockIdx.x % col_blocks;
-        int pos_next = 0;
-        if (t < num_tiles) {
-            const int64_t row = (int64_t)rb * kTR + cw;
-            pos_next = row < M ? pos_ids[row] : 0;
+        // slot j of this thread: floats [256 cw + 128 j + 4 lane, +4) of every tile; K is a
+        // multiple of 4, so a slot never straddles two rows
+        // f, col: where the slot falls in the current tile. fa, rowa, cola: the same three tiles
+        // ahead, which is how early the row's position id is fetched (a dependent global load per
+        // tile must not sit on the consumer's critical path); pq holds the ids in flight.
+        constexpr int kAhead = 3;
+        int64_t f[2], fa[2], rowa[2];
+        int col[2], cola[2], pq[2][kAhead];
+        const int64_t stride = (int64_t)gridDim.x * kTileFloats;
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const uint32_t f0 = (uint32_t)blockIdx.x * kTileFloats + 256u * cw + 128u * j + 4u * lane;
+            f[j] = fa[j] = f0;
+            rowa[j] = f0 / (uint32_t)K;
+            col[j] = cola[j] = (int)(f0 % (uint32_t)K);
+#pragma unroll
+            for (int a = 0; a < kAhead; ++a) {
+                pq[j][a] = fa[j] < total ? pos_ids[rowa[j]] : 0;
+                fa[j] += stride;
+                rowa[j] += step_row;
+                cola[j] += step_col;
+                if (cola[j] >= K) { cola[j] -= K; ++rowa[j]; }
+            }
         }
-        for (; t < num_tiles; t += gridDim.x, ++it) {
+        uint32_t it = 0;
+        for (int t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
             const int s = it % kRingStages;
             const uint32_t ph = (it / kRingStages) & 1u;
-            const int64_t row = (int64_t)rb * kTR + cw;
-            const int colb = cb * kTC;
-            const int p = pos_next;
-            rb += step_rb;
-            cb += step_cb;
-            if (cb >= col_blocks) { cb -= col_blocks; ++rb; }
-            if (t + (int)gridDim.x < num_tiles) {          // position of the next tile's row, ahead of time
-                const int64_t rn = (int64_t)rb * kTR + cw;
-                pos_next = rn < M ? pos_ids[rn] : 0;
+            int64_t fc[2];
+            int cc[2], pc[2];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                fc[j] = f[j]; cc[j] = col[j]; pc[j] = pq[j][0];
+                f[j] += stride;
+                col[j] += step_col;
+                if (col[j] >= K) col[j] -= K;
+#pragma unroll
+                for (int a = 0; a + 1 < kAhead; ++a) pq[j][a] = pq[j][a + 1];
+                pq[j][kAhead - 1] = fa[j] < total ? pos_ids[rowa[j]] : 0;
+                fa[j] += stride;
+                rowa[j] += step_row;
+                cola[j] += step_col;
+                if (cola[j] >= K) { cola[j] -= K; ++rowa[j]; }
             }
             bool ok = mbar_wait(bar_full(s), ph, abort_flag, limit);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
-            if (row < M) {
-                const uint8_t* trow = smem + s * kTileBytes + cw * (kTC * 4);
-                const bool pok = (p >= 0) && (p < P);
-                const float rt = pok ? rt_s[p] : 0.0f;
-                if (!pok && lane == 0 && colb == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+            const uint8_t* tile = smem + s * kTileBytes;
 #pragma unroll
-                for (int j = 0; j < 2; ++j) {
-                    const int cl = 128 * j + 4 * lane;
-                    const int col = colb + cl;
-                    if (col < K) {
-                        const float4 v = *reinterpret_cast<const float4*>(trow + cl * 4);
-                        const float4 rc = *reinterpret_cast<const float4*>(rc_s + col);
-                        *reinterpret_cast<uint32_t*>(Xq + row * K + col) = quantize4<B8>(v, rc, rt, qmin, qmax);
-                    }
+            for (int j = 0; j < 2; ++j) {
+                if (fc[j] < total) {
+                    const int p = pc[j];
+                    const bool pok = (p >= 0) && (p < P);
+                    const float rt = pok ? rt_s[p] : 0.0f;
+                    if (!pok && cc[j] == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+                    const float4 v = *reinterpret_cast<const float4*>(tile + (256 * cw + 128 * j + 4 * lane) * 4);
+                    const float4 rc = *reinterpret_cast<const float4*>(rc_s + cc[j]);
+                    *reinterpret_cast<uint32_t*>(Xq + fc[j]) = quantize4<B8>(v, rc, rt, qmin, qmax);
                 }
             }
             __syncwarp();
@@ -275,14 +294,16 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
                                   CUtensorMapFloatOOBfill);
 
+// Requires M * K to be a multiple of 256 (the flat view has whole rows of 256 floats).
 int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
                 const float* s_tok, int P, int qmin, int qmax, int8_t* Xq, bool dependent, cudaStream_t st)
 {
+    const int64_t total = M * (int64_t)K;
     CUtensorMap tmX;
     EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
-    cuuint64_t gdim[2] = {(cuuint64_t)K, (cuuint64_t)M};
-    cuuint64_t gstride[1] = {(cuuint64_t)K * 4};
-    cuuint32_t box[2] = {(cuuint32_t)kTC, (cuuint32_t)kTR};
+    cuuint64_t gdim[2] = {256, (cuuint64_t)(total / 256)};
+    cuuint64_t gstride[1] = {1024};
+    cuuint32_t box[2] = {256, 16};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(&tmX, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<float*>(X), gdim, gstride, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -298,9 +319,9 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
         ctx->quant_ring_configured |= (b8 ? 1 : 2);
     }
-    const int col_blocks = (K + kTC - 1) / kTC;
-    const int num_tiles = (int)(((M + kTR - 1) / kTR) * col_blocks);       // the caller has checked that this fits
+    const int num_tiles = (int)((total + kTileFloats - 1) / kTileFloats);       // the caller has checked that this fits
     const int grid = num_tiles < ctx->sm_count ? num_tiles : ctx->sm_count;
+    const int64_t step = (int64_t)grid * kTileFloats;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -312,8 +333,8 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
     const unsigned long long limit = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmX, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq,
-                                       col_blocks, num_tiles, grid / col_blocks, grid % col_blocks, ctx->d_status, limit);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tmX, pos_ids, total, K, s_ch, s_tok, P, qmin, qmax, Xq, num_tiles,
+                                       (int)(step / K), (int)(step % K), ctx->d_status, limit);
     ctx->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
@@ -326,9 +347,10 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
                          bool dependent, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    // the ring kernel's tables bound K and P; it only wins (by 15-20 %) on inputs of hundreds of MB,
+    // the ring kernel's tables bound K and P; it only wins (by 25-30 %) on inputs of hundreds of MB,
     // where the output no longer stays in L2 and more bytes in flight help
-    const bool ring_ok = K <= kRingMaxK && P <= kRingMaxP && ctx->encode_tiled != nullptr && M < ((int64_t)1 << 29);
+    const bool ring_ok = K <= kRingMaxK && P <= kRingMaxP && ctx->encode_tiled != nullptr && M < ((int64_t)1 << 29) &&
+                         (M * (int64_t)K) % 256 == 0;
     bool ring = ring_ok && (int64_t)M * K >= ((int64_t)1 << 27);
     if (ctx->debug == 7) ring = false;                    // tuning: force one or the other
     if (ctx->debug == 8) ring = ring_ok;

@@ -49,7 +49,7 @@ def _out_code(g, out):
 # ----------------------------------------------------------------------------- quantize
 @pytest.mark.parametrize("bits", [8, 6])
 @pytest.mark.parametrize("shape", [(1, 16, 1), (7, 48, 3), (300, 1040, 11), (64, 1920, 64), (513, 512, 680),
-                                   (40, 5120, 5), (1000, 16, 2)])
+                                   (40, 5120, 5), (1000, 16, 2), (512, 16, 4), (96, 48, 7), (4099, 256, 680)])
 def test_quantize_codes_bit_exact(gpu, bits, shape):
     M, K, P = shape
     X = (rng.standard_normal((M, K)) * 3).astype(np.float32)
