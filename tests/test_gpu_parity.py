@@ -397,3 +397,37 @@ def test_tiled_gemm_split_tail_is_exact_and_repeatable(gpu, shape, ksplit):
     finally:
         gpu.ctx.stwq_set_option(102, 0)
         gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
+
+
+@pytest.mark.parametrize("cfg,idx", [(2, 2), (2, 3), (4, 0), (4, 1)])
+def test_graph_replay_matches_the_oracle(gpu, cfg, idx):
+    """The benchmark replays qlinear from a CUDA graph (with the two kernels of a call chained by
+    programmatic dependent launch). The replayed call must give what the direct call gives."""
+    torch = gpu.torch
+    L = wl.config_layers(cfg)[idx]
+    par = prepare(L, samples=4, gps_n=64)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], L.bits, L.act)
+    d = {k: gpu.T(par[k]) for k in ("Wq", "s_w", "s_tok", "s_ch", "bias")}
+    Xd, pd = gpu.T(X), gpu.T(pos)
+    Y = _out_tensor(gpu, L.M, L.N, "bf16")
+    Yi = _out_tensor(gpu, L.M, L.N, "int32")
+
+    def calls():
+        gpu.ctx.qlinear(Xd, pd, d["Wq"], d["s_w"], d["s_tok"], d["s_ch"], d["bias"], L.bits, L.act, gpu.B.OUT_BF16, Y)
+        gpu.ctx.qlinear(Xd, pd, d["Wq"], d["s_w"], d["s_tok"], d["s_ch"], d["bias"], L.bits, L.act, gpu.B.OUT_INT32, Yi)
+    calls()                                     # workspace is allocated outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            calls()
+        Y.fill_(-3)
+        Yi.fill_(-3)
+        g.replay()
+        g.replay()
+    torch.cuda.synchronize()
+    assert gpu.ctx.stwq_device_status() == 0
+    np.testing.assert_array_equal(Yi.cpu().numpy(), ref["acc"])
+    assert_close(Y.float().cpu().numpy(), ref, RTOL["bf16"], f"graph replay cfg{cfg} {L.name}")
