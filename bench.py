@@ -418,6 +418,50 @@ def other_configs(ctx, pk, torch, dev, peaks):
                      "tops": round(L.ops / us / 1e6, 1), "timing": f"CUDA graph, {copies} weight copies rotated (HBM-cold)"})
         del Xs, Ws, Ys, g
     out["config4"] = rows
+    # static versus dynamic token-wise quantization (Table 5 of the paper prices the dynamic
+    # min-max pass at 473.9 ms against 397.9 ms for whole-model latency on its GPU): the two
+    # quantize kernels and the two whole calls on the benchmark's layer shapes, inputs rotated
+    rows = []
+    for L in wl.config_layers(2):
+        ncopy = max(2, int(2 * 126e6 // (5.0 * L.M * L.K)) + 1)
+        Xs = [torch.randn(L.M, L.K, device=dev) for _ in range(ncopy)]
+        Xq = torch.empty((L.M, L.K), dtype=torch.int8, device=dev)
+        Wq = torch.randint(-128, 128, (L.N, L.K), dtype=torch.int8, device=dev)
+        pos = torch.from_numpy(wl.positions(L)).to(dev)
+        s_w = torch.rand(L.N, device=dev) * 1e-3 + 1e-4
+        s_tok = torch.rand(L.P, device=dev) * 0.05 + 0.01
+        s_row = torch.empty(L.M, device=dev)
+        s_ch = (torch.rand(L.K, device=dev) + 0.5) if L.use_gps else None
+        b = torch.randn(L.N, device=dev) * 0.02
+        Y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device=dev)
+
+        def graph_ms(fn):
+            for x in Xs:
+                fn(x)
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for x in Xs:
+                        fn(x)
+                g.replay()
+                a, e = ev(), ev()
+                a.record()
+                for _ in range(5):
+                    g.replay()
+                e.record()
+                torch.cuda.synchronize()
+            return a.elapsed_time(e) / (5 * len(Xs))
+        t_sq = graph_ms(lambda x: ctx.stwq_quantize(x, pos, s_ch, s_tok, 8, Xq))
+        t_dq = graph_ms(lambda x: ctx.dtwq_quantize(x, s_ch, 8, Xq, s_row))
+        t_sl = graph_ms(lambda x: ctx.qlinear(x, pos, Wq, s_w, s_tok, s_ch, b, 8, L.act, pk.OUT_BF16, Y))
+        t_dl = graph_ms(lambda x: ctx.qlinear_dtwq(x, Wq, s_w, s_ch, b, 8, L.act, pk.OUT_BF16, Y))
+        rows.append({"layer": L.name, "K": L.K, "N": L.N, "stwq_quantize_us": round(t_sq * 1e3, 2),
+                     "dtwq_quantize_us": round(t_dq * 1e3, 2), "stwq_qlinear_us": round(t_sl * 1e3, 2),
+                     "dtwq_qlinear_us": round(t_dl * 1e3, 2), "dtwq_over_stwq_qlinear": round(t_dl / t_sl, 3)})
+        del Xs, Xq, Wq, Y
+    out["static_vs_dynamic_config2"] = rows
     ctx.check_device_status()
     return out
 

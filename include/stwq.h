@@ -143,6 +143,22 @@ int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M
               int act, int out_dtype, void* Y, void* stream);
 
 /*
+ * Dynamic token-wise quantization, the baseline that the static scales replace (Section 1,
+ * Section 4.2, Table 5: the range of every token is found by a min-max pass at run time). Kept
+ * to be timed beside stwq_quantize / qlinear, and for layers without calibrated scales:
+ *     v = X[m,k] * rc[k],  a_m = max_k |v|,  s_row[m] = 2 a_m / D  (1 if a_m == 0),
+ *     Xq[m,k] = clamp(round(v * (1 / s_row[m])), qmin, qmax)
+ * NaN values do not take part in the maximum and give code 0. K <= 8192.
+ * X [M,K] fp32, s_ch [K] or NULL, Xq [M,K] int8 out, s_row [M] fp32 out.
+ * qlinear_dtwq is qlinear with this quantizer: the dequantizer uses s_row[m] in place of
+ * s_tok[pos_ids[m]]; codes, scales and row ids live in context workspace.
+ */
+int dtwq_quantize(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
+                  float* s_row, void* stream);
+int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const int8_t* Wq, const float* s_w,
+                 const float* s_ch, const float* bias, int bits, int act, int out_dtype, void* Y, void* stream);
+
+/*
  * qlinear without any allocation. (The paper has no counterpart to this call; it exists for the
  * way the library gets embedded.) qlinear needs a context, whose creation allocates, and keeps
  * the int8 copy of X in workspace that may be (re)allocated during a call. Hosts that cannot

@@ -63,6 +63,7 @@ def lib():
             for f in (L.orc_quantize, L.orc_quantize_exact_div):
                 f.restype = C.c_int
                 f.argtypes = [fp, ip, C.c_int64, C.c_int, fp, fp, C.c_int, C.c_int, bp]
+            L.orc_dtwq_quantize.argtypes = [fp, C.c_int64, C.c_int, fp, C.c_int, bp, fp]
             L.orc_igemm.argtypes = [bp, bp, C.c_int64, C.c_int, C.c_int, ip]
             L.orc_epilogue.restype = C.c_int
             L.orc_epilogue.argtypes = [ip, ip, C.c_int64, C.c_int, fp, C.c_int, fp, fp, C.c_int, dp, dp]
@@ -155,6 +156,18 @@ def quantize(X, pos_ids, s_ch, s_tok, bits, exact_div=False):
     if st != 0:
         raise ValueError("pos_ids outside [0, P)")
     return Xq
+
+
+def dtwq_quantize(X, s_ch, bits):
+    """Dynamic token-wise quantization (per-row min-max at run time). Returns (Xq int8 [M,K], s_row [M])."""
+    X = _f32(X)
+    s_ch = _f32(s_ch)
+    M, K = X.shape
+    Xq = np.empty((M, K), np.int8)
+    s_row = np.empty(M, np.float32)
+    lib().orc_dtwq_quantize(_ptr(X, C.c_float), M, K, _ptr(s_ch, C.c_float), bits, _ptr(Xq, C.c_int8),
+                            _ptr(s_row, C.c_float))
+    return Xq, s_row
 
 
 def igemm(Xq, Wq):

@@ -232,6 +232,43 @@ int orc_quantize(const float* X, const int32_t* pos_ids, int64_t M, int K,
 }
 
 /*
+ * Dynamic token-wise quantization, the baseline that the static scheme replaces
+ * (Section 1 and Section 4.2: the quantization range of every token is found at
+ * run time by a min-max pass over that token; Table 5 prices it at 473.9 ms
+ * against 397.9 ms for the static scales). Per row m:
+ *   v[k]  = X[m,k] * rc[k]                       (rc = 1 / s_ch, or 1)
+ *   a_m   = max_k |v[k]|                         (NaN entries do not take part)
+ *   s_m   = delta(a_m) = 2 a_m / (2^b - 1)       (the symmetric quantizer above)
+ *   Xq    = clamp(round(v[k] * (1 / s_m)))       (reciprocal form, as on the static path)
+ * s_row[m] = s_m is returned so that the dequantizer can use it in place of the
+ * static s_tok[pos[m]].
+ */
+void orc_dtwq_quantize(const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
+                       float* s_row)
+{
+    float* rc = (float*)malloc(sizeof(float) * (size_t)K);
+    for (int k = 0; k < K; ++k) rc[k] = s_ch ? 1.0f / s_ch[k] : 1.0f;
+    for (int64_t m = 0; m < M; ++m) {
+        float a = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            const float x = X[m * K + k];
+            const float v = s_ch ? x * rc[k] : x;
+            const float av = fabsf(v);
+            if (av > a) a = av;                       /* false for NaN */
+        }
+        const float s = orc_delta(a, bits);
+        const float rt = 1.0f / s;
+        s_row[m] = s;
+        for (int k = 0; k < K; ++k) {
+            const float x = X[m * K + k];
+            const float v = s_ch ? x * rc[k] : x;
+            Xq[m * K + k] = (int8_t)orc_code(v * rt, bits);
+        }
+    }
+    free(rc);
+}
+
+/*
  * The same step with two true divisions per element, (x / s_ch[k]) / s_tok[p]:
  * the literal reading of Eq. 1 and Eq. 2. Information only (how many codes the
  * reciprocal form moves); not the parity definition.

@@ -20,7 +20,7 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
-            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static"]
+            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq"]
 
 _lib = None
 
@@ -61,6 +61,8 @@ def load_library():
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
     L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.dtwq_quantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, vp]
+    L.qlinear_dtwq.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, vp]
     L.stwq_device_status.argtypes = [vp, vp]
     L.stwq_set_option.argtypes = [vp, i32, i32]
     L.stwq_launch_count.argtypes = [vp]
@@ -165,6 +167,17 @@ class Context:
         self._check(self._L.qlinear_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
                                       P, _p(bias), act, out_dtype, _p(Y), self._stream(stream)),
                     "qlinear_q")
+
+    def dtwq_quantize(self, X, s_ch, bits, Xq, s_row, stream=None):
+        M, K = X.shape
+        self._check(self._L.dtwq_quantize(self._h, _p(X), M, K, _p(s_ch), bits, _p(Xq), _p(s_row),
+                                          self._stream(stream)), "dtwq_quantize")
+
+    def qlinear_dtwq(self, X, Wq, s_w, s_ch, bias, bits, act, out_dtype, Y, stream=None):
+        M, K = X.shape
+        N = Wq.shape[0]
+        self._check(self._L.qlinear_dtwq(self._h, _p(X), M, K, N, _p(Wq), _p(s_w), _p(s_ch), _p(bias), bits, act,
+                                         out_dtype, _p(Y), self._stream(stream)), "qlinear_dtwq")
 
     def stwq_device_status(self, stream=None) -> int:
         return int(self._L.stwq_device_status(self._h, self._stream(stream)))

@@ -153,6 +153,7 @@ void stwq_destroy(stwq_ctx* ctx)
     if (ctx->ws_xq) cudaFree(ctx->ws_xq);
     if (ctx->ws_cal) cudaFree(ctx->ws_cal);
     if (ctx->ws_dec) cudaFree(ctx->ws_dec);
+    if (ctx->ws_dyn) cudaFree(ctx->ws_dyn);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -253,6 +254,55 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, pdl, st);
     if (rc != STWQ_OK) return rc;
     return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, pdl, st);
+}
+
+int dtwq_quantize(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
+                  float* s_row, void* stream)
+{
+    if (!ctx || !X || !Xq || !s_row) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || K > 8192) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if ((K & 15) != 0 || !aligned16(X) || !aligned16(Xq)) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_dtwq(ctx, X, M, K, s_ch, bits, Xq, s_row, nullptr, static_cast<cudaStream_t>(stream));
+}
+
+int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const int8_t* Wq, const float* s_w,
+                 const float* s_ch, const float* bias, int bits, int act, int out_dtype, void* Y, void* stream)
+{
+    if (!ctx || !s_w) return STWQ_ERR_NULL;
+    static const int32_t dummy_pos = 0;
+    static const float dummy_tok = 1.0f;
+    int rc = check_gemm_args(X, &dummy_pos, M, K, N, Wq, s_w, &dummy_tok, 1, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if (K > 8192 || M > (int64_t)0x7fffffff) return STWQ_ERR_DIM;
+    DeviceGuard g(ctx->device);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc != STWQ_OK) return rc;
+    const size_t need = (size_t)M * 8;
+    if (ctx->ws_dyn_bytes < need) {
+        if (ctx->ws_dyn) {
+            cudaError_t e = cudaFree(ctx->ws_dyn);
+            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+            ctx->ws_dyn = nullptr;
+            ctx->ws_dyn_bytes = 0;
+        }
+        void* ptr = nullptr;
+        if (cudaMalloc(&ptr, need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return STWQ_ERR_NOMEM;
+        }
+        ctx->ws_dyn = ptr;
+        ctx->ws_dyn_bytes = need;
+    }
+    float* s_row = static_cast<float*>(ctx->ws_dyn);
+    int32_t* row_ids = reinterpret_cast<int32_t*>(s_row + M);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = stwq_launch_dtwq(ctx, X, M, K, s_ch, bits, ctx->ws_xq, s_row, row_ids, st);
+    if (rc != STWQ_OK) return rc;
+    // the dequantizer takes the row's own scale: position id = row index, table = the scales just computed
+    return run_gemm(ctx, ctx->ws_xq, row_ids, M, K, N, Wq, s_w, s_row, (int)M, bias, act, out_dtype, Y, false, st);
 }
 
 int stwq_device_status(stwq_ctx* ctx, void* stream)

@@ -29,6 +29,8 @@ struct stwq_ctx {
     uint32_t* d_status;        // device status word
     int8_t* ws_xq;             // workspace: int8 copy of X for qlinear
     size_t ws_xq_bytes;
+    void* ws_dyn;              // workspace of qlinear_dtwq: per-row scales [M] and row ids [M]
+    size_t ws_dyn_bytes;
     void* ws_cal;              // workspace: calibration histograms and selection state
     size_t ws_cal_bytes;
     void* ws_dec;              // split-K workspace: arrival counters, then int32 partial sums
@@ -60,6 +62,8 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);
 
+int stwq_launch_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
+                     float* s_row, int32_t* row_ids, cudaStream_t st);
 int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial);
 
 static inline int stwq_cuda_fail(stwq_ctx* ctx, cudaError_t e)

@@ -431,3 +431,45 @@ def test_graph_replay_matches_the_oracle(gpu, cfg, idx):
     assert gpu.ctx.stwq_device_status() == 0
     np.testing.assert_array_equal(Yi.cpu().numpy(), ref["acc"])
     assert_close(Y.float().cpu().numpy(), ref, RTOL["bf16"], f"graph replay cfg{cfg} {L.name}")
+
+
+# ----------------------------------------------------------------------------- dynamic token-wise baseline
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(1, 16), (37, 1040), (300, 2048), (64, 5120), (9, 8192)])
+def test_dtwq_codes_and_scales_bit_exact(gpu, bits, shape):
+    M, K = shape
+    X = (rng.standard_normal((M, K)) * rng.uniform(0.1, 30, (M, 1))).astype(np.float32)
+    X.flat[:2] = [np.nan, 1e30]
+    if M > 2:
+        X[1] = 0.0
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    for sc in (s_ch, None):
+        ref_q, ref_s = oracle.dtwq_quantize(X, sc, bits)
+        Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+        sr = gpu.torch.zeros(M, device=gpu.dev)
+        gpu.ctx.dtwq_quantize(gpu.T(X), gpu.T(sc), bits, Xq, sr)
+        np.testing.assert_array_equal(sr.cpu().numpy(), ref_s)
+        np.testing.assert_array_equal(Xq.cpu().numpy(), ref_q)
+
+
+@pytest.mark.parametrize("M", [200, 1500])
+def test_qlinear_dtwq_matches_the_oracle(gpu, M):
+    """qlinear with run-time per-row scales: codes from the dynamic quantizer, dequantizer fed
+    with the row's own scale. M = 200 takes the few-row kernel, M = 1500 the tiled GEMM."""
+    L = wl.scaled(wl.config_layers(2)[2], batch=3, K=1024, N=768)
+    par = prepare(L, samples=4, gps_n=64)
+    X = wl.activations(L)[:M]
+    Xq, s_row = oracle.dtwq_quantize(X, par["s_ch"], 8)
+    acc = oracle.igemm(Xq, par["Wq"])
+    ids = np.arange(M, dtype=np.int32)
+    Yref, mag = oracle.epilogue(acc, ids, s_row, par["s_w"], par["bias"], 1)
+    ref = {"Y": Yref, "mag": mag}
+    d = {k: gpu.T(par[k]) for k in ("Wq", "s_w", "s_ch", "bias")}
+    Yi = _out_tensor(gpu, M, L.N, "int32")
+    gpu.ctx.qlinear_dtwq(gpu.T(X), d["Wq"], d["s_w"], d["s_ch"], d["bias"], 8, 1, gpu.B.OUT_INT32, Yi)
+    np.testing.assert_array_equal(Yi.cpu().numpy(), acc)
+    for out in ("fp32", "bf16"):
+        Y = _out_tensor(gpu, M, L.N, out)
+        gpu.ctx.qlinear_dtwq(gpu.T(X), d["Wq"], d["s_w"], d["s_ch"], d["bias"], 8, 1, _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+        assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"qlinear_dtwq {out}")

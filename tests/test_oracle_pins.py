@@ -417,3 +417,40 @@ def test_gps_and_stwq_reduce_output_error_on_outlier_data():
     e_none, e_stwq, e_both = err(None, False), err(None, True), err(s_gps, True)
     assert e_stwq < e_none
     assert e_both < e_stwq
+
+
+# ----------------------------------------------------------------------------- dynamic token-wise (the baseline)
+@pytest.mark.parametrize("bits", [8, 6])
+def test_dtwq_is_per_row_minmax(bits):
+    """Section 4.2 / Table 5 baseline: every row gets the min-max scale of that row alone. Pinned
+    by numpy's own max, by the extreme code every non-zero row must reach, by the round-trip
+    bound with the row's scale, and by the static quantizer fed with the same scales."""
+    rng = np.random.default_rng(5)
+    M, K = 37, 96
+    X = (rng.standard_normal((M, K)) * rng.uniform(0.1, 30, (M, 1))).astype(np.float32)
+    X[3] = 0.0
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    qmax, qmin, D = 2 ** (bits - 1) - 1, -2 ** (bits - 1), 2 ** bits - 1
+    for sc in (s_ch, None):
+        Xq, s_row = oracle.dtwq_quantize(X, sc, bits)
+        V = X * (np.float32(1) / sc) if sc is not None else X
+        a = np.abs(V).max(axis=1)
+        want = np.where(a > 0, (a + a) / np.float32(D), np.float32(1)).astype(np.float32)
+        np.testing.assert_array_equal(s_row, want)
+        nz = a > 0
+        assert (np.abs(Xq[nz].astype(np.int32)).max(axis=1) >= qmax).all()     # a / delta = D / 2 rounds past qmax
+        assert not Xq[3].any() and s_row[3] == 1.0
+        assert Xq.min() >= qmin and Xq.max() <= qmax
+        # round trip with the row's own scale: inside the range the error is at most delta / 2
+        err = np.abs(Xq.astype(np.float64) * s_row[:, None] - V.astype(np.float64))
+        inside = np.abs(V) <= (qmax * s_row)[:, None]
+        assert (err[inside] <= 0.5000001 * np.broadcast_to(s_row[:, None], V.shape)[inside]).all()
+        # the static quantizer with these scales and position = row index gives the same codes
+        same = oracle.quantize(X, np.arange(M, dtype=np.int32), sc, s_row, bits)
+        np.testing.assert_array_equal(Xq, same)
+    # a single huge element sets the scale of its own row only
+    X2 = X.copy()
+    X2[5, 7] = 1e6
+    _, s2 = oracle.dtwq_quantize(X2, None, bits)
+    _, s1 = oracle.dtwq_quantize(X, None, bits)
+    assert s2[5] > 1000 * s1[5] and np.array_equal(np.delete(s2, 5), np.delete(s1, 5))
