@@ -462,6 +462,56 @@ def other_configs(ctx, pk, torch, dev, peaks):
                      "dtwq_qlinear_us": round(t_dl * 1e3, 2), "dtwq_over_stwq_qlinear": round(t_dl / t_sl, 3)})
         del Xs, Xq, Wq, Y
     out["static_vs_dynamic_config2"] = rows
+    # fc1 -> fc2 of a block, unfused (fc1 writes fp32 activations, fc2's call quantizes them) and
+    # chained (fc1's epilogue emits fc2's codes; fc2 runs from codes)
+    rows = []
+    for cfg in (2, 5):
+        fc1, fc2 = [L for L in wl.config_layers(cfg) if L.name in ("fc1", "fc2")]
+        X = torch.randn(fc1.M, fc1.K, device=dev)
+        pos = torch.from_numpy(wl.positions(fc1)).to(dev)
+        W1 = torch.randint(-128, 128, (fc1.N, fc1.K), dtype=torch.int8, device=dev)
+        W2 = torch.randint(-128, 128, (fc2.N, fc2.K), dtype=torch.int8, device=dev)
+        sw1 = torch.rand(fc1.N, device=dev) * 1e-4 + 1e-5
+        sw2 = torch.rand(fc2.N, device=dev) * 1e-3 + 1e-4
+        st1 = torch.rand(fc1.P, device=dev) * 0.05 + 0.01
+        st2 = torch.rand(fc1.P, device=dev) * 0.05 + 0.01
+        sc1 = torch.rand(fc1.K, device=dev) + 0.5
+        b1 = torch.randn(fc1.N, device=dev) * 0.02
+        b2 = torch.randn(fc2.N, device=dev) * 0.02
+        H = torch.empty((fc1.M, fc1.N), dtype=torch.float32, device=dev)
+        Hq = torch.empty((fc1.M, fc1.N), dtype=torch.int8, device=dev)
+        Y = torch.empty((fc2.M, fc2.N), dtype=torch.bfloat16, device=dev)
+
+        def unfused():
+            ctx.qlinear(X, pos, W1, sw1, st1, sc1, b1, 8, fc1.act, pk.OUT_F32, H)
+            ctx.qlinear(H, pos, W2, sw2, st2, None, b2, 8, 0, pk.OUT_BF16, Y)
+
+        def chained():
+            ctx.qlinear_chain(X, pos, W1, sw1, st1, sc1, b1, 8, fc1.act, None, st2, 8, Hq)
+            ctx.qlinear_q(Hq, pos, W2, sw2, st2, b2, 0, pk.OUT_BF16, Y)
+        res = {}
+        for name, fn in (("unfused", unfused), ("chained", chained)):
+            fn()
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    fn()
+                g.replay()
+                a, e = ev(), ev()
+                a.record()
+                for _ in range(10):
+                    g.replay()
+                e.record()
+                torch.cuda.synchronize()
+            res[name] = a.elapsed_time(e) / 10
+        ops = fc1.ops + fc2.ops
+        rows.append({"config": cfg, "M": fc1.M, "hidden": fc1.K, "ffn": fc1.N,
+                     "unfused_us": round(res["unfused"] * 1e3, 1), "chained_us": round(res["chained"] * 1e3, 1),
+                     "unfused_tops": round(ops / res["unfused"] / 1e9, 1), "chained_tops": round(ops / res["chained"] / 1e9, 1)})
+        del X, W1, W2, H, Hq, Y
+    out["ffn_fc1_fc2_chained"] = rows
     ctx.check_device_status()
     return out
 

@@ -143,6 +143,29 @@ int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M
               int act, int out_dtype, void* Y, void* stream);
 
 /*
+ * Chained layers (Section 5 quantizes every linear of a block, so one quantized linear feeds
+ * the next one's quantizer): qlinear whose epilogue applies the NEXT layer's static activation
+ * quantizer instead of storing Y, so that the activation never makes the round trip through
+ * memory in floating point:
+ *     z = float(acc) * (s_tok[pos] * s_w[n]) + bias[n],  y = act(z)                 (fp32)
+ *     Xq_next[m,n] = clamp(round((y * rc_next[n]) * rt_next[pos_ids[m]]), qmin, qmax)
+ * rc_next = 1 / s_ch_next (1 if NULL), rt_next = 1 / s_tok_next, bits_next in {8, 6}; positions
+ * are those of this layer (a linear keeps the token order). Xq_next [M,N] int8 is what
+ * stwq_quantize would give on Y kept in fp32; feed it to qlinear_q / qlinear_chain_q of the next
+ * layer. GELU is evaluated in the short form used for bf16 output (error on y below 6e-4 |z|),
+ * so a code can differ by one from the exact activation's where u lies that close to a tie.
+ * Always runs the tiled CTA-pair GEMM: N a multiple of 16, s_w / bias / s_ch_next 16-byte aligned
+ * (STWQ_ERR_ALIGN otherwise).
+ */
+int qlinear_chain(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
+                  const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+                  const float* bias, int bits, int act, const float* s_ch_next, const float* s_tok_next,
+                  int bits_next, int8_t* Xq_next, void* stream);
+int qlinear_chain_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+                    const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
+                    const float* s_ch_next, const float* s_tok_next, int bits_next, int8_t* Xq_next, void* stream);
+
+/*
  * Dynamic token-wise quantization, the baseline that the static scales replace (Section 1,
  * Section 4.2, Table 5: the range of every token is found by a min-max pass at run time). Kept
  * to be timed beside stwq_quantize / qlinear, and for layers without calibrated scales:

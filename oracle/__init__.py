@@ -67,6 +67,9 @@ def lib():
             L.orc_igemm.argtypes = [bp, bp, C.c_int64, C.c_int, C.c_int, ip]
             L.orc_epilogue.restype = C.c_int
             L.orc_epilogue.argtypes = [ip, ip, C.c_int64, C.c_int, fp, C.c_int, fp, fp, C.c_int, dp, dp]
+            L.orc_chain_codes.restype = C.c_int
+            L.orc_chain_codes.argtypes = [ip, ip, C.c_int64, C.c_int, fp, C.c_int, fp, fp, C.c_int, fp, fp, C.c_int,
+                                          bp, fp, fp]
             L.orc_qlinear.restype = C.c_int
             L.orc_qlinear.argtypes = [fp, ip, C.c_int64, C.c_int, C.c_int, bp, fp, fp, C.c_int, fp, fp,
                                       C.c_int, C.c_int, dp, bp, ip, dp]
@@ -196,6 +199,26 @@ def epilogue(acc, pos_ids, s_tok, s_w, bias, act):
     if st != 0:
         raise ValueError("pos_ids outside [0, P)")
     return Y, mag
+
+
+def chain_codes(acc, pos_ids, s_tok, s_w, bias, act, s_ch_next, s_tok_next, bits_next):
+    """Dequantize + bias + activation in fp32, then the next layer's static quantizer.
+    Returns dict(codes int8 [M,N], u float32 (value before rounding), zmag float32)."""
+    acc = np.ascontiguousarray(acc, np.int32)
+    pos_ids = np.ascontiguousarray(pos_ids, np.int32)
+    s_tok, s_w, bias = _f32(s_tok), _f32(s_w), _f32(bias)
+    s_ch_next, s_tok_next = _f32(s_ch_next), _f32(s_tok_next)
+    M, N = acc.shape
+    codes = np.empty((M, N), np.int8)
+    u = np.empty((M, N), np.float32)
+    zmag = np.empty((M, N), np.float32)
+    st = lib().orc_chain_codes(_ptr(acc, C.c_int32), _ptr(pos_ids, C.c_int32), M, N, _ptr(s_tok, C.c_float),
+                               s_tok.size, _ptr(s_w, C.c_float), _ptr(bias, C.c_float), act,
+                               _ptr(s_ch_next, C.c_float), _ptr(s_tok_next, C.c_float), bits_next,
+                               _ptr(codes, C.c_int8), _ptr(u, C.c_float), _ptr(zmag, C.c_float))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return {"codes": codes, "u": u, "zmag": zmag}
 
 
 def qlinear(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act=0):

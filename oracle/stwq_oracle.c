@@ -344,6 +344,48 @@ int orc_epilogue(const int32_t* acc, const int32_t* pos_ids, int64_t M, int N,
 }
 
 /*
+ * Chained layers: the paper quantizes every linear of a block (Section 5), so the
+ * output of one quantized linear is the input of the next one's static
+ * quantizer. This is Step 3 followed at once by Step 1 of the next layer:
+ *   z = fmaf(float(acc), s_tok[pos] * s_w[n], bias[n])        in fp32, this order
+ *   y = act(z)         (the activation itself evaluated in double, rounded to fp32)
+ *   u = (y * rc_next[n]) * rt_next[pos]                       two fp32 multiplies
+ *   code = clamp(round(u))
+ * A code is an integer decided by floating point, so the decision is taken in the
+ * precision of the deployed path (fp32), not in double. u_out (optional) receives
+ * u and zmag_out (optional) |z * rc_next * rt_next|, which bounds how far an
+ * approximate activation can move u.
+ */
+int orc_chain_codes(const int32_t* acc, const int32_t* pos_ids, int64_t M, int N,
+                    const float* s_tok, int P, const float* s_w, const float* bias, int act,
+                    const float* s_ch_next, const float* s_tok_next, int bits_next,
+                    int8_t* codes, float* u_out, float* zmag_out)
+{
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) return -1;
+        const float st = s_tok[p];
+        const float rt = 1.0f / s_tok_next[p];
+        for (int n = 0; n < N; ++n) {
+            const float scale = st * s_w[n];
+            const float z = fmaf((float)acc[m * N + n], scale, bias ? bias[n] : 0.0f);
+            float y = z;
+            const double zd = (double)z;
+            if (act == 1) y = (float)(zd * 0.5 * (1.0 + erf(zd / sqrt(2.0))));
+            else if (act == 2)
+                y = (float)(zd * 0.5 * (1.0 + tanh(sqrt(2.0 / M_PI) * (zd + 0.044715 * zd * zd * zd))));
+            const float rc = s_ch_next ? 1.0f / s_ch_next[n] : 1.0f;
+            const float t = y * rc;
+            const float u = t * rt;
+            codes[m * N + n] = (int8_t)orc_code(u, bits_next);
+            if (u_out) u_out[m * N + n] = u;
+            if (zmag_out) zmag_out[m * N + n] = fabsf((z * rc) * rt);
+        }
+    }
+    return 0;
+}
+
+/*
  * The whole quantized linear: quantize -> integer GEMM -> dequantize.
  * Xq_out, acc_out and mag may be NULL. Returns 0 or -1 (bad pos_id).
  */

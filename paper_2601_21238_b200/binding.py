@@ -20,7 +20,7 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
-            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq"]
+            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q"]
 
 _lib = None
 
@@ -61,6 +61,8 @@ def load_library():
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
     L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.qlinear_chain.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp]
+    L.qlinear_chain_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, vp, vp, i32, vp, vp]
     L.dtwq_quantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, vp]
     L.qlinear_dtwq.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, vp, i32, i32, i32, vp, vp]
     L.stwq_device_status.argtypes = [vp, vp]
@@ -167,6 +169,23 @@ class Context:
         self._check(self._L.qlinear_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
                                       P, _p(bias), act, out_dtype, _p(Y), self._stream(stream)),
                     "qlinear_q")
+
+    def qlinear_chain(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, s_ch_next, s_tok_next, bits_next,
+                      Xq_next, stream=None):
+        M, K = X.shape
+        N = Wq.shape[0]
+        self._check(self._L.qlinear_chain(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
+                                          s_tok.numel(), _p(s_ch), _p(bias), bits, act, _p(s_ch_next),
+                                          _p(s_tok_next), bits_next, _p(Xq_next), self._stream(stream)),
+                    "qlinear_chain")
+
+    def qlinear_chain_q(self, Xq, pos_ids, Wq, s_w, s_tok, bias, act, s_ch_next, s_tok_next, bits_next, Xq_next,
+                        stream=None):
+        M, K = Xq.shape
+        N = Wq.shape[0]
+        self._check(self._L.qlinear_chain_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
+                                            s_tok.numel(), _p(bias), act, _p(s_ch_next), _p(s_tok_next),
+                                            bits_next, _p(Xq_next), self._stream(stream)), "qlinear_chain_q")
 
     def dtwq_quantize(self, X, s_ch, bits, Xq, s_row, stream=None):
         M, K = X.shape

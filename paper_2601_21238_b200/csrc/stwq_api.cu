@@ -98,7 +98,7 @@ int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M,
                                   after_quantize, st);
     if (ctx->gemm_path != 3 && stwq_qgemm2_supported(N, out_dtype, s_w, bias))
         return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
-                                  after_quantize, st);
+                                  after_quantize, nullptr, st);
     return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
 }
 
@@ -254,6 +254,53 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, pdl, st);
     if (rc != STWQ_OK) return rc;
     return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, pdl, st);
+}
+
+static int chain_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
+                      const float* s_w, const float* s_tok, int P, const float* bias, int act,
+                      const float* s_ch_next, const float* s_tok_next, int bits_next, const int8_t* Xq_next)
+{
+    if (!pos_ids || !s_tok || !s_w || !s_tok_next) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(A, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, STWQ_OUT_F32, Xq_next);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits_next) != STWQ_OK) return STWQ_ERR_BITS;
+    // the fused epilogue lives in the CTA-pair kernel only: 16-byte rows of codes, aligned vectors
+    if ((N & 15) != 0 || !stwq_qgemm2_supported(N, 3, s_w, bias)) return STWQ_ERR_ALIGN;
+    if (s_ch_next != nullptr && (reinterpret_cast<uintptr_t>(s_ch_next) & 15u) != 0) return STWQ_ERR_ALIGN;
+    return STWQ_OK;
+}
+
+int qlinear_chain_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
+                    const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
+                    const float* s_ch_next, const float* s_tok_next, int bits_next, int8_t* Xq_next, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    int rc = chain_args(Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, s_ch_next, s_tok_next, bits_next, Xq_next);
+    if (rc != STWQ_OK) return rc;
+    DeviceGuard g(ctx->device);
+    const stwq_chain chain = {s_ch_next, s_tok_next, bits_next};
+    return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, 3, Xq_next, false, &chain,
+                              static_cast<cudaStream_t>(stream));
+}
+
+int qlinear_chain(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
+                  const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+                  const float* bias, int bits, int act, const float* s_ch_next, const float* s_tok_next,
+                  int bits_next, int8_t* Xq_next, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    int rc = chain_args(X, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, s_ch_next, s_tok_next, bits_next, Xq_next);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc != STWQ_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool pdl = ctx->debug != 5;
+    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, pdl, st);
+    if (rc != STWQ_OK) return rc;
+    const stwq_chain chain = {s_ch_next, s_tok_next, bits_next};
+    return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, 3, Xq_next, pdl, &chain, st);
 }
 
 int dtwq_quantize(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,

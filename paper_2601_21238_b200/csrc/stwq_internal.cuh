@@ -40,6 +40,14 @@ struct stwq_ctx {
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
 };
 
+// The next layer's static quantizer, applied by the GEMM epilogue when the output type is 3
+// (int8 codes for the next linear instead of Y): s_ch_next [N] or NULL, s_tok_next [P].
+struct stwq_chain {
+    const float* s_ch_next;
+    const float* s_tok_next;
+    int bits_next;
+};
+
 // Launchers (host). Each returns STWQ_OK or STWQ_ERR_CUDA and bumps ctx->launches.
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
@@ -57,7 +65,7 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize,
-                       cudaStream_t st);
+                       const struct stwq_chain* chain, cudaStream_t st);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);

@@ -34,6 +34,7 @@ namespace {
 
 constexpr int kBM = 128;      // rows per CTA
 constexpr int kBK = 128;      // bytes of K per stage
+constexpr int kOutCodes = 3;  // internal output type: int8 codes for the next layer (see stwq_chain)
 
 struct Gemm2Params {
     int64_t M;
@@ -51,6 +52,10 @@ struct Gemm2Params {
     int full_units, num_units, nsplit, kb_per_split;
     int32_t* partial;          // [tail tile][split][rank][warp][128 x 32 lanes] int32
     uint32_t* counters;        // [tail tile][rank][warp]
+    // chained output (OUT == kOutCodes): the next layer's static quantizer applied to act(z)
+    const float* s_ch_next;    // [N] or NULL
+    const float* s_tok_next;   // [P]
+    int qmin_next, qmax_next;
     void* Y;                   // used by the direct-store epilogue
     int y_vec32;               // Y base and row pitch are 32-byte aligned: 256-bit stores are legal
 };
@@ -67,7 +72,7 @@ struct Smem2 {
     static constexpr int kOffB = STAGES * kABytes;
     static constexpr int kOffStage = STAGES * kStageBytes;  // per epilogue warp: two staging tiles of 32 rows x 128 B
     static constexpr int kOffScale = kOffStage + (STORE == 0 ? EPI * 8192 : 0); // per epilogue warp: s_w and bias of its columns
-    static constexpr int kOffBars = kOffScale + 2 * BN * 4 * 4;
+    static constexpr int kOffBars = kOffScale + 3 * BN * 4 * 4;   // s_w, bias and (chained output) the next layer's 1 / s_ch
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kOffMisc = kOffBars + kNumBars * 8;
     static constexpr int kTotal = kOffMisc + 16;
@@ -110,7 +115,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
               const __grid_constant__ CUtensorMap tmY, const Gemm2Params p)
 {
     using L = Smem2<BN, STAGES, EPI, STORE>;
-    constexpr int kChunkCols = (OUT == STWQ_OUT_BF16) ? 64 : 32;
+    constexpr int kChunkCols = (OUT == STWQ_OUT_BF16) ? 64 : (OUT == kOutCodes ? 128 : 32);
     constexpr int kChunks = BN / kChunkCols;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -229,10 +234,11 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         constexpr int kMyCols = kMyChunks * kChunkCols;
         static_assert(kChunks % kSubs == 0, "chunks must divide among the warps of a quarter");
         const uint32_t stage0 = base + L::kOffStage + (uint32_t)ew * 8192u;   // two staging tiles (STORE == 0)
-        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 2 * kMyCols;
+        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 3 * kMyCols;
         float* my_bias = my_sw + kMyCols;
+        float* my_rcn = my_bias + kMyCols;
         const uint32_t tempty0 = mapa_u32(bar_tempty(0), 0);
-        constexpr int kElem = (OUT == STWQ_OUT_BF16) ? 2 : 4;
+        constexpr int kElem = (OUT == STWQ_OUT_BF16) ? 2 : (OUT == kOutCodes ? 1 : 4);
         uint32_t t = 0, nstore = 0;
         bool ok = true;
         for (int u = pair; u < p.num_units; u += num_pairs, ++t) {
@@ -243,7 +249,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
             const int n0 = (tile % p.tiles_n) * BN;
             const int64_t row = (int64_t)m0 + q * 32 + lane;
-            float st = 0.0f;
+            float st = 0.0f, rtn = 0.0f;
             if (OUT != STWQ_OUT_INT32) {
                 // column scales and biases of this warp's chunks -> its private shared copy, and
                 // the row scale, all fetched before the accumulator is waited for
@@ -258,11 +264,23 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     }
                     *reinterpret_cast<float4*>(my_sw + i) = sw;
                     *reinterpret_cast<float4*>(my_bias + i) = bi;
+                    if (OUT == kOutCodes) {
+                        float4 rn = make_float4(1.f, 1.f, 1.f, 1.f);
+                        if (col < p.N && p.s_ch_next != nullptr) {
+                            const float4 sn = __ldg(reinterpret_cast<const float4*>(p.s_ch_next + col));
+                            rn = make_float4(__fdiv_rn(1.0f, sn.x), __fdiv_rn(1.0f, sn.y), __fdiv_rn(1.0f, sn.z), __fdiv_rn(1.0f, sn.w));
+                        }
+                        *reinterpret_cast<float4*>(my_rcn + i) = rn;
+                    }
                 }
                 if (row < p.M) {
                     const int pos = p.pos_ids[row];
-                    if (pos >= 0 && pos < p.P) st = p.s_tok[pos];
-                    else atomicOr(p.status, STWQ_DEV_POS_RANGE);
+                    if (pos >= 0 && pos < p.P) {
+                        st = p.s_tok[pos];
+                        if (OUT == kOutCodes) rtn = __fdiv_rn(1.0f, p.s_tok_next[pos]);
+                    } else {
+                        atomicOr(p.status, STWQ_DEV_POS_RANGE);
+                    }
                 }
                 __syncwarp();
             }
@@ -275,7 +293,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             // the buffer is handed back as soon as they have landed; conversion and stores follow
             // from registers. tcgen05.ld queues behind the tensor-core instructions already issued,
             // so one exposed wait per tile is the best that can be had.
-            constexpr int kLoadsPerChunk = (OUT == STWQ_OUT_BF16) ? 2 : 1;
+            constexpr int kLoadsPerChunk = (OUT == STWQ_OUT_BF16) ? 2 : (OUT == kOutCodes ? 4 : 1);
             constexpr int kLoads = kMyChunks * kLoadsPerChunk;
             uint32_t racc[kLoads][32];
 #pragma unroll
@@ -335,7 +353,46 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint32_t* r1 = racc[k * kLoadsPerChunk + kLoadsPerChunk - 1];
                 uint32_t w[32];                           // this row's 128 bytes of output
                 const uint64_t st2 = pack_f2(st, st);
-                if (OUT == STWQ_OUT_BF16) {
+                if (OUT == kOutCodes) {
+                    // y = act(z) stays in fp32 registers and goes straight through the next layer's
+                    // static quantizer: (y * rc_next[n]) * rt_next[pos], round to nearest even, clamp, pack
+                    const float* crn = my_rcn + k * kChunkCols;
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const uint32_t* r = racc[k * kLoadsPerChunk + h];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const float4 sw = *reinterpret_cast<const float4*>(csw + h * 32 + j);
+                            const float4 bi = *reinterpret_cast<const float4*>(cbi + h * 32 + j);
+                            const float4 rn = *reinterpret_cast<const float4*>(crn + h * 32 + j);
+                            uint64_t z01 = fma_f2(pack_f2((float)(int32_t)r[j + 0], (float)(int32_t)r[j + 1]),
+                                                  mul_f2(st2, pack_f2(sw.x, sw.y)), pack_f2(bi.x, bi.y));
+                            uint64_t z23 = fma_f2(pack_f2((float)(int32_t)r[j + 2], (float)(int32_t)r[j + 3]),
+                                                  mul_f2(st2, pack_f2(sw.z, sw.w)), pack_f2(bi.z, bi.w));
+                            if (ACT != STWQ_ACT_NONE) {
+                                z01 = gelu_fast_f2(z01);
+                                z23 = gelu_fast_f2(z23);
+                            }
+                            float v0, v1, v2, v3;
+                            unpack_f2(z01, v0, v1);
+                            unpack_f2(z23, v2, v3);
+                            int q0 = __float2int_rn(__fmul_rn(__fmul_rn(v0, rn.x), rtn));
+                            int q1 = __float2int_rn(__fmul_rn(__fmul_rn(v1, rn.y), rtn));
+                            int q2 = __float2int_rn(__fmul_rn(__fmul_rn(v2, rn.z), rtn));
+                            int q3 = __float2int_rn(__fmul_rn(__fmul_rn(v3, rn.w), rtn));
+                            if (p.qmax_next != 127) {
+                                q0 = max(min(q0, p.qmax_next), p.qmin_next);
+                                q1 = max(min(q1, p.qmax_next), p.qmin_next);
+                                q2 = max(min(q2, p.qmax_next), p.qmin_next);
+                                q3 = max(min(q3, p.qmax_next), p.qmin_next);
+                            }
+                            uint32_t hi, packed;
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+                            asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(packed) : "r"(q1), "r"(q0), "r"(hi));
+                            w[h * 8 + j / 4] = packed;
+                        }
+                    }
+                } else if (OUT == STWQ_OUT_BF16) {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
 #pragma unroll
@@ -462,7 +519,7 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
 {
     using L = Smem2<BN, STAGES, EPI, STORE>;
     auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT, STORE>;
-    const uint64_t bit = 1ull << ((BN == 256 ? 0 : 12) + OUT * 4 + ACT);
+    const uint64_t bit = 1ull << ((BN == 256 ? 0 : 16) + OUT * 4 + ACT);
     uint64_t& mask = ctx->configured_pair[STORE];
     if (!(mask & bit)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
@@ -509,6 +566,14 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
     if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
     if (out_dtype == STWQ_OUT_INT32)
         return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
+    if (out_dtype == kOutCodes) {                         // 128-column chunks: 256-wide tiles only
+        if constexpr (BN == 256) {
+            STWQ_CASE(kOutCodes, STWQ_ACT_NONE)
+            STWQ_CASE(kOutCodes, STWQ_ACT_GELU_ERF)
+            STWQ_CASE(kOutCodes, STWQ_ACT_GELU_TANH)
+        }
+        return STWQ_ERR_DIM;
+    }
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
@@ -525,7 +590,7 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
 // epilogue reads s_w / bias as aligned float4.
 bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* bias)
 {
-    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : 4;
+    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : (out_dtype == kOutCodes ? 1 : 4);
     if (((int64_t)N * elem) % 16 != 0) return false;
     if (out_dtype != STWQ_OUT_INT32) {
         if ((reinterpret_cast<uintptr_t>(s_w) & 15u) != 0) return false;
@@ -536,17 +601,22 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
-                       int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
+                       int act, int out_dtype, void* Y, bool after_quantize, const stwq_chain* chain, cudaStream_t st)
 {
     // 256-wide tiles whenever N has more than 128 columns: a 128-wide tile needs 1.5x the
     // L2 -> shared-memory bytes per multiply-accumulate and is bound by that feed.
     const int tiles_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
-    int bn = N > 128 ? 256 : 128;
+    int bn = (N > 128 || out_dtype == kOutCodes) ? 256 : 128;
     if (ctx->force_bn == 128 || ctx->force_bn == 256) bn = ctx->force_bn;
 
     Gemm2Params p;
     p.Y = Y;
-    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : 4;
+    p.s_ch_next = chain ? chain->s_ch_next : nullptr;
+    p.s_tok_next = chain ? chain->s_tok_next : nullptr;
+    p.qmax_next = chain ? (1 << (chain->bits_next - 1)) - 1 : 127;
+    p.qmin_next = -p.qmax_next - 1;
+    if (out_dtype == kOutCodes && (!chain || !chain->s_tok_next)) return STWQ_ERR_NULL;
+    const int elem = out_dtype == STWQ_OUT_BF16 ? 2 : (out_dtype == kOutCodes ? 1 : 4);
     p.y_vec32 = ((reinterpret_cast<uintptr_t>(Y) & 31u) == 0 && ((int64_t)N * elem) % 32 == 0) ? 1 : 0;
     p.M = M; p.N = N; p.K = K; p.P = P;
     p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
@@ -608,6 +678,8 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
         rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, M, N, 64, 32);
     else if (out_dtype == STWQ_OUT_F32)
         rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Y, M, N, 32, 32);
+    else if (out_dtype == kOutCodes)
+        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Y, M, N, 128, 32);
     else
         rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
     if (rc != STWQ_OK) return rc;

@@ -115,7 +115,7 @@ extern "C" int qlinear_static(const float* X, const int32_t* pos_ids, int64_t M,
     if (rc != STWQ_OK) return rc;
     if (stwq_qgemm2_supported(N, out_dtype, s_w, bias))
         return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act,
-                                  out_dtype, Y, false, st);
+                                  out_dtype, Y, false, nullptr, st);
     return stwq_launch_qgemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype,
                              Y, st);
 }

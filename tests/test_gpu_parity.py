@@ -473,3 +473,48 @@ def test_qlinear_dtwq_matches_the_oracle(gpu, M):
         gpu.ctx.qlinear_dtwq(gpu.T(X), d["Wq"], d["s_w"], d["s_ch"], d["bias"], 8, 1, _out_code(gpu, out), Y)
         assert gpu.ctx.stwq_device_status() == 0
         assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"qlinear_dtwq {out}")
+
+
+# ----------------------------------------------------------------------------- chained layers
+@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("bits_next", [8, 6])
+@pytest.mark.parametrize("shape", [(333, 400, 336), (1500, 1024, 1024)])
+def test_chained_output_codes(gpu, shape, bits_next, act):
+    """qlinear_chain: the epilogue applies the next layer's static quantizer. Without activation
+    the codes are bit-exact. With GELU the kernel's short form moves y by at most 6e-4 |z|, so a
+    code may differ by one, and only where the oracle's pre-round value lies that close to a tie."""
+    M0, K, N = shape
+    L = wl.scaled(wl.config_layers(2)[2], batch=3, P=680, K=K, N=N, act=act)
+    par = prepare(L, samples=4, gps_n=64)
+    X, pos = wl.activations(L)[:M0], wl.positions(L)[:M0]
+    first = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, act)
+    s_chn = rng.uniform(0.5, 2, N).astype(np.float32)
+    # next-layer scales sized so that the codes use the range: y / (s_ch s_tok) of order 30
+    typical = np.maximum(np.abs(first["Y"]).mean(axis=1), 1e-3)
+    s_tokn = np.zeros(L.P, np.float32)
+    for p_ in range(L.P):
+        sel = pos == p_
+        s_tokn[p_] = np.float32(typical[sel].mean() / 20) if sel.any() else np.float32(1)
+    ref = oracle.chain_codes(first["acc"], pos, par["s_tok"], par["s_w"], par["bias"], act, s_chn, s_tokn, bits_next)
+    d = {k: gpu.T(par[k]) for k in ("Wq", "s_w", "s_tok", "s_ch", "bias")}
+    out = gpu.torch.full((M0, N), 99, dtype=gpu.torch.int8, device=gpu.dev)
+    gpu.ctx.qlinear_chain(gpu.T(X), gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["s_ch"], d["bias"], 8, act,
+                          gpu.T(s_chn), gpu.T(s_tokn), bits_next, out)
+    assert gpu.ctx.stwq_device_status() == 0
+    got = out.cpu().numpy().astype(np.int32)
+    want = ref["codes"].astype(np.int32)
+    if act == 0:
+        np.testing.assert_array_equal(got, want)
+    else:
+        diff = got != want
+        assert np.abs(got - want).max() <= 1
+        u = ref["u"].astype(np.float64)
+        slack = 1e-3 * ref["zmag"].astype(np.float64) + 1e-3
+        assert (np.abs(u - np.floor(u) - 0.5)[diff] <= slack[diff]).all()
+        assert diff.mean() < 0.05
+    assert np.abs(got).max() > 2 ** (bits_next - 1) // 2       # the range is really used
+    # the same from codes already held
+    out2 = gpu.torch.full((M0, N), 99, dtype=gpu.torch.int8, device=gpu.dev)
+    gpu.ctx.qlinear_chain_q(gpu.T(first["Xq"]), gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["bias"], act,
+                            gpu.T(s_chn), gpu.T(s_tokn), bits_next, out2)
+    assert gpu.torch.equal(out, out2)

@@ -454,3 +454,34 @@ def test_dtwq_is_per_row_minmax(bits):
     _, s2 = oracle.dtwq_quantize(X2, None, bits)
     _, s1 = oracle.dtwq_quantize(X, None, bits)
     assert s2[5] > 1000 * s1[5] and np.array_equal(np.delete(s2, 5), np.delete(s1, 5))
+
+
+# ----------------------------------------------------------------------------- chained layers
+def test_chain_codes_are_the_next_quantizer_applied_to_the_dequantized_output():
+    """The chained output is Step 3 followed by the next layer's Step 1. Pinned against the two
+    oracle steps it composes (double epilogue -> quantize): the pre-round value agrees to fp32
+    accuracy and the codes agree except where that value sits within rounding noise of a tie;
+    with unit scales and no activation the codes are the clamped accumulators themselves."""
+    rng = np.random.default_rng(11)
+    M, N, P = 40, 24, 6
+    acc = rng.integers(-60000, 60000, (M, N)).astype(np.int32)
+    pos = rng.integers(0, P, M).astype(np.int32)
+    s_tok = rng.uniform(0.01, 0.05, P).astype(np.float32)
+    s_w = rng.uniform(1e-4, 1e-3, N).astype(np.float32)
+    bias = (0.3 * rng.standard_normal(N)).astype(np.float32)
+    s_chn = rng.uniform(0.5, 2, N).astype(np.float32)
+    s_tokn = rng.uniform(0.005, 0.02, P).astype(np.float32)
+    for act in (0, 1, 2):
+        for bits in (8, 6):
+            got = oracle.chain_codes(acc, pos, s_tok, s_w, bias, act, s_chn, s_tokn, bits)
+            Y, _ = oracle.epilogue(acc, pos, s_tok, s_w, bias, act)
+            u = (Y / s_chn[None, :].astype(np.float64)) / s_tokn[pos][:, None].astype(np.float64)
+            assert np.allclose(got["u"], u, rtol=3e-6, atol=1e-6)
+            qmax, qmin = 2 ** (bits - 1) - 1, -2 ** (bits - 1)
+            want = np.clip(np.rint(u), qmin, qmax)
+            near_tie = np.abs(u - np.floor(u) - 0.5) < 8e-6 * np.maximum(1.0, np.abs(u)) + 1e-6
+            assert ((got["codes"] == want) | near_tie).all() and near_tie.mean() < 0.02
+            assert np.abs(got["codes"].astype(np.int64) - want).max() <= 1
+    ident = oracle.chain_codes(acc // 500, pos, np.ones(P, np.float32), np.ones(N, np.float32), None, 0, None,
+                               np.ones(P, np.float32), 8)
+    np.testing.assert_array_equal(ident["codes"], np.clip(acc // 500, -128, 127))
