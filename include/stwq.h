@@ -115,6 +115,11 @@ int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int
 int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                   const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream);
 
+/* stwq_quantize for activations held in bf16 (X [M,K] bf16): every bf16 value is an fp32 value,
+ * and the codes are those stwq_quantize gives on the widened input. */
+int stwq_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
+                       const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream);
+
 /*
  * The quantized linear layer: stwq_quantize into context workspace, then
  *     acc[m,n] = sum_k Xq[m,k] * Wq[n,k]                          (int32, exact)

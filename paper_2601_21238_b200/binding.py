@@ -20,7 +20,7 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
-            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q"]
+            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16"]
 
 _lib = None
 
@@ -61,6 +61,7 @@ def load_library():
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
     L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.stwq_quantize_bf16.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear_chain.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp]
     L.qlinear_chain_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, vp, vp, i32, vp, vp]
     L.dtwq_quantize.argtypes = [vp, vp, i64, i32, vp, i32, vp, vp, vp]
@@ -154,6 +155,12 @@ class Context:
         self._check(self._L.stwq_quantize(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok),
                                           s_tok.numel(), bits, _p(Xq), self._stream(stream)),
                     "stwq_quantize")
+
+    def stwq_quantize_bf16(self, X, pos_ids, s_ch, s_tok, bits, Xq, stream=None):
+        M, K = X.shape
+        self._check(self._L.stwq_quantize_bf16(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok),
+                                               s_tok.numel(), bits, _p(Xq), self._stream(stream)),
+                    "stwq_quantize_bf16")
 
     def qlinear(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
         M, K = X.shape

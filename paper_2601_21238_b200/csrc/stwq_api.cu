@@ -221,6 +221,17 @@ int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t
                                 static_cast<cudaStream_t>(stream));
 }
 
+int stwq_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
+                       const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream)
+{
+    if (!ctx || !X || !pos_ids || !s_tok || !Xq) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || P <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if ((K & 15) != 0 || !aligned16(X) || !aligned16(Xq)) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_quantize_bf16(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, Xq, static_cast<cudaStream_t>(stream));
+}
+
 int qlinear_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
               const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
               int out_dtype, void* Y, void* stream)

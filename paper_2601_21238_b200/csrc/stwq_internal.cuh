@@ -52,6 +52,8 @@ struct stwq_chain {
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
                          bool dependent, cudaStream_t st);
+int stwq_launch_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
+                              const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, cudaStream_t st);
 int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);

@@ -141,6 +141,84 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
     }
 }
 
+// ---------------------------------------------------------------------------- bf16 input
+// The same quantizer for activations held in bf16 (a bf16 value is an fp32 value, so the
+// arithmetic and the result are those of quantize_kernel on the widened input). A warp owns a
+// 512-column span; a lane owns two runs of 8 consecutive columns (one 16-byte load each) and
+// stores 8 codes per run.
+__device__ __forceinline__ uint4 ld_stream_u4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <bool B8>
+__global__ void __launch_bounds__(kThreads)
+quantize_bf16_kernel(const uint16_t* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
+                     const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin, int qmax,
+                     int8_t* __restrict__ Xq, int spans, int64_t row_stride, uint32_t* __restrict__ status)
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");               // see quantize_kernel
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int span = (int)(warp % spans);
+    int64_t m = warp / spans;
+    const int col0 = span * kSpan + lane * 8;
+    if (m >= M) return;
+    uint4 v[2], vn[2];
+    auto load = [&](int64_t r, uint4 (&d)[2]) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int c = col0 + j * 256;
+            if (c < K) d[j] = ld_stream_u4(X + r * K + c);
+        }
+    };
+    load(m, v);
+    bool ok;
+    float rt = row_scale(pos_ids, s_tok, P, m, ok);
+    float rc[16];
+#pragma unroll
+    for (int j = 0; j < 2; ++j)
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int c = col0 + j * 256 + e;
+            rc[j * 8 + e] = (s_ch != nullptr && c < K) ? __fdiv_rn(1.0f, s_ch[c]) : 1.0f;
+        }
+    while (true) {
+        const int64_t mn = m + row_stride;
+        const bool more = mn < M;
+        bool okn = false;
+        float rtn = 0.0f;
+        if (more) {
+            load(mn, vn);
+            rtn = row_scale(pos_ids, s_tok, P, mn, okn);
+        }
+        if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int c = col0 + j * 256;
+            if (c < K) {
+                const float4 a = make_float4(bf16_lo(v[j].x), bf16_hi(v[j].x), bf16_lo(v[j].y), bf16_hi(v[j].y));
+                const float4 b = make_float4(bf16_lo(v[j].z), bf16_hi(v[j].z), bf16_lo(v[j].w), bf16_hi(v[j].w));
+                uint2 o;
+                o.x = quantize4<B8>(a, make_float4(rc[j * 8 + 0], rc[j * 8 + 1], rc[j * 8 + 2], rc[j * 8 + 3]), rt, qmin, qmax);
+                o.y = quantize4<B8>(b, make_float4(rc[j * 8 + 4], rc[j * 8 + 5], rc[j * 8 + 6], rc[j * 8 + 7]), rt, qmin, qmax);
+                *reinterpret_cast<uint2*>(Xq + m * K + c) = o;
+            }
+        }
+        if (!more) break;
+        v[0] = vn[0];
+        v[1] = vn[1];
+        m = mn;
+        rt = rtn;
+        ok = okn;
+    }
+}
+
 // ---------------------------------------------------------------------------- TMA ring variant
 // X is dense, so a tile is simply 4096 consecutive floats of the flat array (16 KB of contiguous
 // DRAM, which streams a quarter faster than sixteen 1 KB pieces of sixteen rows: 6.0-6.4 against
@@ -341,6 +419,32 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
 }
 
 }  // namespace
+
+int stwq_launch_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
+                              const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, cudaStream_t st)
+{
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    const int spans = (K + kSpan - 1) / kSpan;
+    const int warps_per_block = kThreads / 32;
+    const int64_t max_warps = (int64_t)ctx->sm_count * 4 * warps_per_block;
+    int64_t rows_in_flight = max_warps / spans;
+    if (rows_in_flight < 1) rows_in_flight = 1;
+    if (rows_in_flight > M) rows_in_flight = M;
+    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
+    rows_in_flight = (M + passes - 1) / passes;
+    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    const unsigned blocks = (unsigned)(rows_in_flight * spans / warps_per_block);
+    const uint16_t* x = static_cast<const uint16_t*>(X);
+    if (bits == 8)
+        quantize_bf16_kernel<true><<<blocks, kThreads, 0, st>>>(x, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
+                                                                rows_in_flight, ctx->d_status);
+    else
+        quantize_bf16_kernel<false><<<blocks, kThreads, 0, st>>>(x, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
+                                                                 rows_in_flight, ctx->d_status);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
 
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,

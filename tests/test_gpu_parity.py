@@ -518,3 +518,22 @@ def test_chained_output_codes(gpu, shape, bits_next, act):
     gpu.ctx.qlinear_chain_q(gpu.T(first["Xq"]), gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["bias"], act,
                             gpu.T(s_chn), gpu.T(s_tokn), bits_next, out2)
     assert gpu.torch.equal(out, out2)
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(1, 16, 1), (7, 48, 3), (300, 1040, 11), (513, 512, 680), (40, 5120, 5)])
+def test_quantize_bf16_input_bit_exact(gpu, bits, shape):
+    """bf16 activations: the codes are those of the quantizer on the same values widened to fp32."""
+    M, K, P = shape
+    Xb = gpu.torch.from_numpy((rng.standard_normal((M, K)) * 3).astype(np.float32)).to(gpu.dev).to(gpu.torch.bfloat16)
+    Xb.view(-1)[:3] = gpu.torch.tensor([float("nan"), float("inf"), 1e30], dtype=gpu.torch.bfloat16)
+    X = Xb.float().cpu().numpy()
+    pos = rng.integers(0, P, M).astype(np.int32)
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    s_tok = rng.uniform(0.01, 0.1, P).astype(np.float32)
+    for sc in (s_ch, None):
+        ref = oracle.quantize(X, pos, sc, s_tok, bits)
+        Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
+        gpu.ctx.stwq_quantize_bf16(Xb, gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
+        assert gpu.ctx.stwq_device_status() == 0
+        np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
