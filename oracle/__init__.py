@@ -63,6 +63,15 @@ def lib():
             for f in (L.orc_quantize, L.orc_quantize_exact_div):
                 f.restype = C.c_int
                 f.argtypes = [fp, ip, C.c_int64, C.c_int, fp, fp, C.c_int, C.c_int, bp]
+            L.orc_asym_params.argtypes = [C.c_float, C.c_float, C.c_int, fp, ip]
+            L.orc_gps_fold_asym.argtypes = [fp, C.c_int, C.c_int, fp, C.c_int, bp, fp, ip, ip]
+            L.orc_stwq_calibrate_asym.restype = C.c_int
+            L.orc_stwq_calibrate_asym.argtypes = [fp, ip, C.c_int64, C.c_int, C.c_int, fp, C.c_int, C.c_uint32, fp, ip]
+            L.orc_quantize_asym.restype = C.c_int
+            L.orc_quantize_asym.argtypes = [fp, ip, C.c_int64, C.c_int, fp, fp, ip, C.c_int, C.c_int, bp, ip]
+            L.orc_epilogue_asym.restype = C.c_int
+            L.orc_epilogue_asym.argtypes = [ip, ip, C.c_int64, C.c_int, fp, ip, C.c_int, fp, ip, ip, ip, fp, C.c_int,
+                                            dp, dp, ip]
             L.orc_dtwq_quantize.argtypes = [fp, C.c_int64, C.c_int, fp, C.c_int, bp, fp]
             L.orc_igemm.argtypes = [bp, bp, C.c_int64, C.c_int, C.c_int, ip]
             L.orc_epilogue.restype = C.c_int
@@ -159,6 +168,88 @@ def quantize(X, pos_ids, s_ch, s_tok, bits, exact_div=False):
     if st != 0:
         raise ValueError("pos_ids outside [0, P)")
     return Xq
+
+
+def _i32(a):
+    return None if a is None else np.ascontiguousarray(a, dtype=np.int32)
+
+
+def asym_params(x_down, x_up, bits):
+    """Eq. 1 parameters for the range [x_down, x_up] widened to contain 0: (delta, signed zero point)."""
+    d = C.c_float()
+    z = C.c_int32()
+    lib().orc_asym_params(np.float32(x_down), np.float32(x_up), bits, C.byref(d), C.byref(z))
+    return float(d.value), int(z.value)
+
+
+def gps_fold_asym(W, s_ch, bits):
+    """Asymmetric per-output-channel weights. Returns (Wq int8, s_w, z_w int32, colsum int32)."""
+    W, s_ch = _f32(W), _f32(s_ch)
+    N, K = W.shape
+    Wq = np.empty((N, K), np.int8)
+    s_w = np.empty(N, np.float32)
+    z_w = np.empty(N, np.int32)
+    cs = np.empty(N, np.int32)
+    lib().orc_gps_fold_asym(_ptr(W, C.c_float), N, K, _ptr(s_ch, C.c_float), bits, _ptr(Wq, C.c_int8),
+                            _ptr(s_w, C.c_float), _ptr(z_w, C.c_int32), _ptr(cs, C.c_int32))
+    return Wq, s_w, z_w, cs
+
+
+def stwq_calibrate_asym(X, pos_ids, P, s_ch, bits, pct_ppm):
+    """Asymmetric per-position calibration. Returns (s_tok [P], z_tok int32 [P])."""
+    X, pos_ids, s_ch = _f32(X), _i32(pos_ids), _f32(s_ch)
+    rows, K = X.shape
+    s_tok = np.empty(P, np.float32)
+    z_tok = np.empty(P, np.int32)
+    st = lib().orc_stwq_calibrate_asym(_ptr(X, C.c_float), _ptr(pos_ids, C.c_int32), rows, K, P,
+                                       _ptr(s_ch, C.c_float), bits, int(pct_ppm), _ptr(s_tok, C.c_float),
+                                       _ptr(z_tok, C.c_int32))
+    if st == -1:
+        raise ValueError("pos_ids outside [0, P)")
+    if st == -2:
+        raise ValueError("non-finite calibration value")
+    return s_tok, z_tok
+
+
+def quantize_asym(X, pos_ids, s_ch, s_tok, z_tok, bits):
+    """Asymmetric static activation quantization. Returns (Xq int8 [M,K], rowcorr int32 [M])."""
+    X, pos_ids, s_ch, s_tok, z_tok = _f32(X), _i32(pos_ids), _f32(s_ch), _f32(s_tok), _i32(z_tok)
+    M, K = X.shape
+    Xq = np.empty((M, K), np.int8)
+    rc = np.empty(M, np.int32)
+    st = lib().orc_quantize_asym(_ptr(X, C.c_float), _ptr(pos_ids, C.c_int32), M, K, _ptr(s_ch, C.c_float),
+                                 _ptr(s_tok, C.c_float), _ptr(z_tok, C.c_int32), s_tok.size, bits,
+                                 _ptr(Xq, C.c_int8), _ptr(rc, C.c_int32))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return Xq, rc
+
+
+def epilogue_asym(acc, pos_ids, s_tok, z_tok, s_w, z_w, colsum, rowcorr, bias, act):
+    """Zero-point correction, dequantize, bias, activation. Returns dict(Y, mag, acc_corr)."""
+    acc, pos_ids = _i32(acc), _i32(pos_ids)
+    M, N = acc.shape
+    s_tok, s_w, bias = _f32(s_tok), _f32(s_w), _f32(bias)
+    z_tok, z_w, colsum, rowcorr = _i32(z_tok), _i32(z_w), _i32(colsum), _i32(rowcorr)
+    Y = np.empty((M, N), np.float64)
+    mag = np.empty((M, N), np.float64)
+    ac = np.empty((M, N), np.int32)
+    st = lib().orc_epilogue_asym(_ptr(acc, C.c_int32), _ptr(pos_ids, C.c_int32), M, N, _ptr(s_tok, C.c_float),
+                                 _ptr(z_tok, C.c_int32), s_tok.size, _ptr(s_w, C.c_float), _ptr(z_w, C.c_int32),
+                                 _ptr(colsum, C.c_int32), _ptr(rowcorr, C.c_int32), _ptr(bias, C.c_float), act,
+                                 _ptr(Y, C.c_double), _ptr(mag, C.c_double), _ptr(ac, C.c_int32))
+    if st != 0:
+        raise ValueError("pos_ids outside [0, P)")
+    return {"Y": Y, "mag": mag, "acc": ac}
+
+
+def qlinear_asym(X, pos_ids, Wq, s_w, z_w, colsum, s_tok, z_tok, s_ch, bias, bits, act=0):
+    """The whole asymmetric quantized linear. Returns dict(Y, mag, acc (corrected), Xq, rowcorr)."""
+    Xq, rowcorr = quantize_asym(X, pos_ids, s_ch, s_tok, z_tok, bits)
+    raw = igemm(Xq, Wq)
+    out = epilogue_asym(raw, pos_ids, s_tok, z_tok, s_w, z_w, colsum, rowcorr, bias, act)
+    out.update(Xq=Xq, rowcorr=rowcorr, raw=raw)
+    return out
 
 
 def dtwq_quantize(X, s_ch, bits):

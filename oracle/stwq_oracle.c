@@ -408,6 +408,186 @@ int orc_qlinear(const float* X, const int32_t* pos_ids, int64_t M, int K, int N,
 
 /* ------------------------------------------------------------------------- */
 /*
+ * The asymmetric quantizer, Eq. 1 as printed (Appendix B deploys "channel-wise
+ * asymmetric" weights and asymmetric activations), in the form the integer
+ * pipeline needs.
+ *   delta = (x_up - x_down) / (2^b - 1),  z = round(-x_down / delta),
+ *   c = clamp(round(x / delta) + z, 0, 2^b - 1),  x_hat = delta (c - z).
+ * Readings: the range is widened to contain 0 (x_down <= 0 <= x_up), which keeps
+ * z inside [0, 2^b - 1] and zero exactly representable; a degenerate range gives
+ * delta = 1; delta is floored at 2^-64. Codes are stored in signed containers by
+ * subtracting h = 2^(b-1): cs = c - h in [-h, h-1], with the signed zero point
+ * zs = z - h, so that x_hat = delta (cs - zs). orc_asym_params gives (delta, zs).
+ */
+void orc_asym_params(float x_down, float x_up, int bits, float* delta_out, int32_t* zs_out)
+{
+    const float levels = (float)((1 << bits) - 1);
+    if (x_down > 0.0f) x_down = 0.0f;
+    if (x_up < 0.0f) x_up = 0.0f;
+    float delta = (x_up - x_down) / levels;
+    if (!(delta > 0.0f)) delta = 1.0f;
+    const float floor_ = 5.421010862427522e-20f;
+    if (delta < floor_) delta = floor_;
+    float z = nearbyintf(-x_down / delta);
+    if (z < 0.0f) z = 0.0f;
+    if (z > levels) z = levels;
+    *delta_out = delta;
+    *zs_out = (int32_t)z - (1 << (bits - 1));
+}
+
+/* cs = clamp(round(u) + zs, -h, h-1); NaN gives round(u) = 0; huge u saturates first. */
+static int32_t orc_code_asym(float u, int32_t zs, int bits)
+{
+    float r = (u != u) ? 0.0f : nearbyintf(u);
+    if (r > 1048576.0f) r = 1048576.0f;
+    if (r < -1048576.0f) r = -1048576.0f;
+    int32_t c = (int32_t)r + zs;
+    if (c < orc_qmin(bits)) c = orc_qmin(bits);
+    if (c > orc_qmax(bits)) c = orc_qmax(bits);
+    return c;
+}
+
+/*
+ * Weights, asymmetric per output channel (Eq. 2 weight side, then Eq. 1 with the
+ * min-max range of the scaled row): Wq signed codes, s_w = delta_n, z_w = zs_n,
+ * and colsum[n] = sum_k Wq[n,k], which the zero-point correction of the
+ * integer product needs.
+ */
+void orc_gps_fold_asym(const float* W, int N, int K, const float* s_ch, int bits,
+                       int8_t* Wq, float* s_w, int32_t* z_w, int32_t* colsum)
+{
+    for (int n = 0; n < N; ++n) {
+        const float* w = W + (int64_t)n * K;
+        float lo = 0.0f, hi = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            const float v = s_ch ? w[k] * s_ch[k] : w[k];
+            if (v < lo) lo = v;
+            if (v > hi) hi = v;
+        }
+        float d; int32_t zs;
+        orc_asym_params(lo, hi, bits, &d, &zs);
+        s_w[n] = d;
+        z_w[n] = zs;
+        int32_t sum = 0;
+        for (int k = 0; k < K; ++k) {
+            const float v = s_ch ? w[k] * s_ch[k] : w[k];
+            const int32_t c = orc_code_asym(v / d, zs, bits);
+            Wq[(int64_t)n * K + k] = (int8_t)c;
+            sum += c;
+        }
+        colsum[n] = sum;
+    }
+}
+
+/*
+ * Static token-wise calibration, asymmetric: per position the range is
+ * [x_down, x_up] with x_up the nearest-rank percentile of the signed values
+ * (rank r = ceil(pct n), ascending) and x_down the mirrored one (rank n + 1 - r);
+ * pct = 100 % is min-max. s_tok[p] = delta_p, z_tok[p] = zs_p. A position with
+ * no rows gets (1, -h + 0) from the degenerate range [0, 0].
+ */
+int orc_stwq_calibrate_asym(const float* X, const int32_t* pos_ids, int64_t rows, int K, int P,
+                            const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok)
+{
+    int64_t* count = (int64_t*)calloc((size_t)P, sizeof(int64_t));
+    for (int64_t r = 0; r < rows; ++r) {
+        if (pos_ids[r] < 0 || pos_ids[r] >= P) { free(count); return -1; }
+        count[pos_ids[r]] += 1;
+    }
+    float* rc = (float*)malloc(sizeof(float) * (size_t)K);
+    for (int k = 0; k < K; ++k) rc[k] = s_ch ? 1.0f / s_ch[k] : 1.0f;
+    int status = 0;
+    for (int p = 0; p < P; ++p) {
+        const int64_t n_p = count[p] * (int64_t)K;
+        if (n_p == 0) { orc_asym_params(0.0f, 0.0f, bits, &s_tok[p], &z_tok[p]); continue; }
+        float* v = (float*)malloc(sizeof(float) * (size_t)n_p);
+        int64_t j = 0;
+        for (int64_t r = 0; r < rows; ++r) {
+            if (pos_ids[r] != p) continue;
+            for (int k = 0; k < K; ++k) {
+                const float x = X[r * K + k];
+                const float t = s_ch ? x * rc[k] : x;
+                if (!isfinite(t)) status = -2;
+                v[j++] = t;
+            }
+        }
+        qsort(v, (size_t)n_p, sizeof(float), orc_cmp_float);
+        uint64_t rank = ((uint64_t)pct_ppm * (uint64_t)n_p + 999999ull) / 1000000ull;
+        if (rank < 1) rank = 1;
+        if (rank > (uint64_t)n_p) rank = (uint64_t)n_p;
+        orc_asym_params(v[(uint64_t)n_p - rank], v[rank - 1], bits, &s_tok[p], &z_tok[p]);
+        free(v);
+    }
+    free(rc);
+    free(count);
+    return status;
+}
+
+/*
+ * Activation quantization, asymmetric static per position, reciprocal form as on
+ * the symmetric path: u = (X * rc) * rt, cs = clamp(round(u) + zs[pos], -h, h-1).
+ * rowcorr[m] = sum_k cs[m,k] - K zs[pos[m]] is returned for the correction below.
+ */
+int orc_quantize_asym(const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                      const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr)
+{
+    float* rc = (float*)malloc(sizeof(float) * (size_t)K);
+    for (int k = 0; k < K; ++k) rc[k] = s_ch ? 1.0f / s_ch[k] : 1.0f;
+    int status = 0;
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) { status = -1; break; }
+        const float rt = 1.0f / s_tok[p];
+        int32_t sum = 0;
+        for (int k = 0; k < K; ++k) {
+            const float x = X[m * K + k];
+            const float t = s_ch ? x * rc[k] : x;
+            const int32_t c = orc_code_asym(t * rt, z_tok[p], bits);
+            Xq[m * K + k] = (int8_t)c;
+            sum += c;
+        }
+        rowcorr[m] = sum - K * z_tok[p];
+    }
+    free(rc);
+    return status;
+}
+
+/*
+ * The integer product of two asymmetric factors. With x_hat = dx (cs - zx) and
+ * w_hat = dw (ws - zw):
+ *   sum_k x_hat w_hat = dx dw [ acc - zw (sum_k cs - K zx) - zx sum_k ws ]
+ *                     = dx dw [ acc - zw[n] rowcorr[m] - zx[pos[m]] colsum[n] ]
+ * acc_corr (optional) receives the bracket (an exact integer); then bias and
+ * activation as in orc_epilogue, in double.
+ */
+int orc_epilogue_asym(const int32_t* acc, const int32_t* pos_ids, int64_t M, int N, const float* s_tok,
+                      const int32_t* z_tok, int P, const float* s_w, const int32_t* z_w, const int32_t* colsum,
+                      const int32_t* rowcorr, const float* bias, int act, double* Y, double* mag,
+                      int32_t* acc_corr)
+{
+    for (int64_t m = 0; m < M; ++m) {
+        const int32_t p = pos_ids[m];
+        if (p < 0 || p >= P) return -1;
+        const double st = (double)s_tok[p];
+        for (int n = 0; n < N; ++n) {
+            const int64_t a = (int64_t)acc[m * N + n] - (int64_t)z_w[n] * rowcorr[m] - (int64_t)z_tok[p] * colsum[n];
+            if (acc_corr) acc_corr[m * N + n] = (int32_t)a;
+            const double prod = (double)a * (st * (double)s_w[n]);
+            const double b = bias ? (double)bias[n] : 0.0;
+            const double z = prod + b;
+            double y = z;
+            if (act == 1) y = z * 0.5 * (1.0 + erf(z / sqrt(2.0)));
+            else if (act == 2)
+                y = z * 0.5 * (1.0 + tanh(sqrt(2.0 / M_PI) * (z + 0.044715 * z * z * z)));
+            Y[m * N + n] = y;
+            if (mag) mag[m * N + n] = fabs(prod) + fabs(b);
+        }
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
+/*
  * Gain-Projected Scaling, Algorithm 1 (Appendix F), with Eq. 13-16 of Section 4.1.
  * Inputs: calibration activations X [T, K], weights W [N, K] (paper: n x m,
  * transposed here), bit width, percentile for the activation range.

@@ -485,3 +485,94 @@ def test_chain_codes_are_the_next_quantizer_applied_to_the_dequantized_output():
     ident = oracle.chain_codes(acc // 500, pos, np.ones(P, np.float32), np.ones(N, np.float32), None, 0, None,
                                np.ones(P, np.float32), 8)
     np.testing.assert_array_equal(ident["codes"], np.clip(acc // 500, -128, 127))
+
+
+# ----------------------------------------------------------------------------- asymmetric quantizer (Eq. 1 as printed)
+@pytest.mark.parametrize("bits", [8, 6])
+def test_asym_weights_are_eq1_per_output_channel(bits):
+    """Per-output-channel asymmetric weights: the codes are Eq. 1's unsigned codes (the function
+    pinned by the hand-worked values) minus 2^(b-1), the zero point likewise, colsum is the code
+    sum, and the round trip stays within delta / 2."""
+    rng = np.random.default_rng(3)
+    N, K = 9, 80
+    W = (0.02 * rng.standard_normal((N, K)) + 0.01 * rng.standard_normal((N, 1))).astype(np.float32)
+    W[4] = np.abs(W[4]) + 0.01                       # an all-positive channel: the range is widened to 0
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    h, D = 2 ** (bits - 1), 2 ** bits - 1
+    for sc in (s_ch, None):
+        Wq, s_w, z_w, cs = oracle.gps_fold_asym(W, sc, bits)
+        Ws = W * sc if sc is not None else W
+        for n in range(N):
+            lo, hi = min(Ws[n].min(), 0.0), max(Ws[n].max(), 0.0)
+            code, delta, z = oracle.eq1_quantize(Ws[n], lo, hi, bits)
+            assert s_w[n] == np.float32(delta) and z_w[n] == z - h
+            np.testing.assert_array_equal(Wq[n].astype(np.int32), code - h)
+            assert cs[n] == int(Wq[n].astype(np.int64).sum())
+            back = s_w[n].astype(np.float64) * (Wq[n].astype(np.float64) - z_w[n])
+            assert np.abs(back - Ws[n]).max() <= 0.5000001 * s_w[n]
+        assert z_w[4] == -h and Wq.min() >= -h and Wq.max() <= h - 1
+        assert 0 <= z_w.min() + h and z_w.max() + h <= D
+
+
+def test_asym_zero_point_correction_is_the_exact_integer_product():
+    """sum_k (cs - zx)(ws - zw) by brute force in int64 equals acc - zw rowcorr - zx colsum."""
+    rng = np.random.default_rng(4)
+    M, N, K, P = 13, 7, 48, 3
+    X = (rng.standard_normal((M, K)) + 0.7).astype(np.float32)
+    W = (0.05 * rng.standard_normal((N, K)) - 0.02).astype(np.float32)
+    pos = rng.integers(0, P, M).astype(np.int32)
+    s_tok, z_tok = oracle.stwq_calibrate_asym(X, pos, P, None, 8, 1000000)
+    Wq, s_w, z_w, cs = oracle.gps_fold_asym(W, None, 8)
+    out = oracle.qlinear_asym(X, pos, Wq, s_w, z_w, cs, s_tok, z_tok, None, None, 8, 0)
+    Xc = out["Xq"].astype(np.int64) - z_tok[pos][:, None].astype(np.int64)
+    Wc = Wq.astype(np.int64) - z_w[:, None].astype(np.int64)
+    np.testing.assert_array_equal(out["acc"].astype(np.int64), Xc @ Wc.T)
+    # and the dequantized product is close to the real one: both factors within delta / 2
+    Y = (Xc * s_tok[pos][:, None].astype(np.float64)) @ (Wc * s_w[:, None].astype(np.float64)).T
+    np.testing.assert_allclose(out["Y"], Y, rtol=1e-12, atol=1e-12)
+    assert np.abs(out["Y"] - X.astype(np.float64) @ W.astype(np.float64).T).max() < 0.05
+
+
+@pytest.mark.parametrize("pct", [1000000, 990000, 600000])
+def test_asym_calibration_against_a_full_sort(pct):
+    rng = np.random.default_rng(6)
+    S, P, K = 5, 4, 60
+    pos = np.tile(np.arange(P, dtype=np.int32), S)
+    X = (rng.standard_normal((S * P, K)) * (1 + pos[:, None]) + 0.5 * pos[:, None]).astype(np.float32)
+    X[pos == 3] = np.abs(X[pos == 3])                # a position with only non-negative values
+    s_tok, z_tok = oracle.stwq_calibrate_asym(X, pos, P + 1, None, 8, pct)
+    for p in range(P):
+        v = np.sort(X[pos == p].ravel())
+        r = min(max(-(-pct * v.size // 1000000), 1), v.size)
+        d, z = oracle.asym_params(v[v.size - r], v[r - 1], 8)
+        assert s_tok[p] == np.float32(d) and z_tok[p] == z
+    assert z_tok[3] == -128                          # range [0, up]: zero point at the bottom code
+    assert s_tok[P] == 1.0                           # a position that never occurs
+    if pct == 1000000:
+        v = X[pos == 1]
+        assert s_tok[1] == np.float32((np.float32(v.max()) - np.float32(v.min())) / np.float32(255))
+
+
+def test_asym_activation_codes_and_its_advantage_on_one_sided_data():
+    """Codes follow Eq. 1 (reciprocal form): inside the range the round trip is within delta / 2,
+    outside it saturates; on one-sided data (what follows a GELU) the asymmetric range wastes no
+    codes, so its error is about half the symmetric one's."""
+    rng = np.random.default_rng(8)
+    M, K, P = 64, 96, 4
+    pos = rng.integers(0, P, M).astype(np.int32)
+    X = np.abs(rng.standard_normal((M, K))).astype(np.float32) * (1 + pos[:, None])
+    s_tok, z_tok = oracle.stwq_calibrate_asym(X, pos, P, None, 8, 1000000)
+    Xq, rowcorr = oracle.quantize_asym(X, pos, None, s_tok, z_tok, 8)
+    np.testing.assert_array_equal(rowcorr, Xq.astype(np.int64).sum(axis=1) - K * z_tok[pos])
+    back = s_tok[pos][:, None].astype(np.float64) * (Xq.astype(np.float64) - z_tok[pos][:, None])
+    err_a = np.abs(back - X)
+    assert (err_a <= 0.5001 * s_tok[pos][:, None]).all()
+    s_sym = oracle.stwq_calibrate(X, pos, P, None, 8, 1000000)
+    Xs = oracle.quantize(X, pos, None, s_sym, 8)
+    err_s = np.abs(s_sym[pos][:, None].astype(np.float64) * Xs - X)
+    assert err_a.mean() < 0.6 * err_s.mean()
+    big = X.copy()
+    big[0, 0] = 1e9
+    big[1, 1] = -1e9
+    q2, _ = oracle.quantize_asym(big, pos, None, s_tok, z_tok, 8)
+    assert q2[0, 0] == 127 and q2[1, 1] == -128
