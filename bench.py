@@ -512,6 +512,44 @@ def other_configs(ctx, pk, torch, dev, peaks):
                      "unfused_tops": round(ops / res["unfused"] / 1e9, 1), "chained_tops": round(ops / res["chained"] / 1e9, 1)})
         del X, W1, W2, H, Hq, Y
     out["ffn_fc1_fc2_chained"] = rows
+    # the asymmetric quantizer (Eq. 1 with zero points) beside the symmetric one, whole calls
+    rows = []
+    for L in wl.config_layers(2):
+        X = torch.randn(L.M, L.K, device=dev) + 0.5
+        Wq = torch.randint(-128, 128, (L.N, L.K), dtype=torch.int8, device=dev)
+        pos = torch.from_numpy(wl.positions(L)).to(dev)
+        s_w = torch.rand(L.N, device=dev) * 1e-3 + 1e-4
+        z_w = torch.randint(-40, 40, (L.N,), dtype=torch.int32, device=dev)
+        cs = Wq.to(torch.int32).sum(dim=1).to(torch.int32)
+        s_tok = torch.rand(L.P, device=dev) * 0.05 + 0.01
+        z_tok = torch.randint(-40, 40, (L.P,), dtype=torch.int32, device=dev)
+        s_ch = (torch.rand(L.K, device=dev) + 0.5) if L.use_gps else None
+        b = torch.randn(L.N, device=dev) * 0.02
+        Y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device=dev)
+        res = {}
+        for name, fn in (("sym", lambda: ctx.qlinear(X, pos, Wq, s_w, s_tok, s_ch, b, 8, L.act, pk.OUT_BF16, Y)),
+                         ("asym", lambda: ctx.qlinear_asym(X, pos, Wq, s_w, z_w, cs, s_tok, z_tok, s_ch, b, 8, L.act,
+                                                           pk.OUT_BF16, Y))):
+            fn()
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for _ in range(4):
+                        fn()
+                g.replay()
+                a, e = ev(), ev()
+                a.record()
+                for _ in range(5):
+                    g.replay()
+                e.record()
+                torch.cuda.synchronize()
+            res[name] = a.elapsed_time(e) / 20
+        rows.append({"layer": L.name, "K": L.K, "N": L.N, "sym_qlinear_us": round(res["sym"] * 1e3, 2),
+                     "asym_qlinear_us": round(res["asym"] * 1e3, 2), "asym_tops": round(L.ops / res["asym"] / 1e9, 1)})
+        del X, Wq, Y
+    out["asymmetric_config2"] = rows
     ctx.check_device_status()
     return out
 

@@ -171,6 +171,34 @@ int qlinear_chain_q(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int
                     const float* s_ch_next, const float* s_tok_next, int bits_next, int8_t* Xq_next, void* stream);
 
 /*
+ * The asymmetric quantizer, Eq. 1 as printed (Appendix B: channel-wise asymmetric weights,
+ * asymmetric activations), next to the symmetric one that the calls above use:
+ *     delta = (x_up - x_down) / D,  z = round(-x_down / delta),  c = clamp(round(x / delta) + z, 0, D)
+ * with the range widened to contain 0 (so 0 <= z <= D). Codes live in the same signed containers,
+ * cs = c - 2^(b-1), together with the signed zero point zs = z - 2^(b-1): x_hat = delta (cs - zs).
+ *  - stwq_calibrate_asym: per position, x_up = the value of rank ceil(pct n) among the signed
+ *    values X / s_ch, x_down = the value of rank n + 1 - ceil(pct n); s_tok[p] = delta, z_tok[p] = zs.
+ *  - gps_fold_asym: per output channel the min-max range of W * s_ch; also colsum[n] = sum_k Wq[n,k].
+ *  - stwq_quantize_asym: cs = clamp(round((X * rc) * rt) + z_tok[pos], qmin, qmax) and
+ *    rowcorr[m] = sum_k cs[m,k] - K z_tok[pos[m]].
+ *  - qlinear_asym: quantize, integer GEMM, then the exact zero-point correction
+ *        acc' = acc - z_w[n] rowcorr[m] - z_tok[pos[m]] colsum[n]     (= sum_k (cs - zx)(ws - zw))
+ *    and z = float(acc') * (s_tok[pos] * s_w[n]) + bias[n], activation, cast. STWQ_OUT_INT32 stores acc'.
+ *    Runs the tiled CTA-pair GEMM for every M: N a multiple of 4 (8 for bf16), s_w / bias / z_w /
+ *    colsum 16-byte aligned, K <= 32768 (STWQ_ERR_ALIGN / STWQ_ERR_DIM otherwise).
+ */
+int stwq_calibrate_asym(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K, int P,
+                        const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok, void* stream);
+int gps_fold_asym(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq, float* s_w,
+                  int32_t* z_w, int32_t* colsum, void* stream);
+int stwq_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                       const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr,
+                       void* stream);
+int qlinear_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
+                 const float* s_w, const int32_t* z_w, const int32_t* colsum, const float* s_tok, const int32_t* z_tok,
+                 int P, const float* s_ch, const float* bias, int bits, int act, int out_dtype, void* Y, void* stream);
+
+/*
  * Dynamic token-wise quantization, the baseline that the static scales replace (Section 1,
  * Section 4.2, Table 5: the range of every token is found by a min-max pass at run time). Kept
  * to be timed beside stwq_quantize / qlinear, and for layers without calibrated scales:

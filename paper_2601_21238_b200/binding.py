@@ -20,7 +20,8 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
-            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16"]
+            "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
+            "stwq_quantize_asym", "qlinear_asym"]
 
 _lib = None
 
@@ -61,6 +62,10 @@ def load_library():
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
     L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.stwq_calibrate_asym.argtypes = [vp, vp, vp, i64, i32, i32, vp, i32, u32, vp, vp, vp]
+    L.gps_fold_asym.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, vp, vp, vp]
+    L.stwq_quantize_asym.argtypes = [vp, vp, vp, i64, i32, vp, vp, vp, i32, i32, vp, vp, vp]
+    L.qlinear_asym.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.stwq_quantize_bf16.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear_chain.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, vp, vp, i32, vp, vp]
     L.qlinear_chain_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, vp, vp, i32, vp, vp]
@@ -193,6 +198,30 @@ class Context:
         self._check(self._L.qlinear_chain_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
                                             s_tok.numel(), _p(bias), act, _p(s_ch_next), _p(s_tok_next),
                                             bits_next, _p(Xq_next), self._stream(stream)), "qlinear_chain_q")
+
+    def stwq_calibrate_asym(self, Xcal, pos_ids, P, s_ch, bits, pct_ppm, s_tok, z_tok, stream=None):
+        rows, K = Xcal.shape
+        self._check(self._L.stwq_calibrate_asym(self._h, _p(Xcal), _p(pos_ids), rows, K, P, _p(s_ch), bits, pct_ppm,
+                                                _p(s_tok), _p(z_tok), self._stream(stream)), "stwq_calibrate_asym")
+
+    def gps_fold_asym(self, W, s_ch, bits, Wq, s_w, z_w, colsum, stream=None):
+        N, K = W.shape
+        self._check(self._L.gps_fold_asym(self._h, _p(W), N, K, _p(s_ch), bits, _p(Wq), _p(s_w), _p(z_w), _p(colsum),
+                                          self._stream(stream)), "gps_fold_asym")
+
+    def stwq_quantize_asym(self, X, pos_ids, s_ch, s_tok, z_tok, bits, Xq, rowcorr, stream=None):
+        M, K = X.shape
+        self._check(self._L.stwq_quantize_asym(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok), _p(z_tok),
+                                               s_tok.numel(), bits, _p(Xq), _p(rowcorr), self._stream(stream)),
+                    "stwq_quantize_asym")
+
+    def qlinear_asym(self, X, pos_ids, Wq, s_w, z_w, colsum, s_tok, z_tok, s_ch, bias, bits, act, out_dtype, Y,
+                     stream=None):
+        M, K = X.shape
+        N = Wq.shape[0]
+        self._check(self._L.qlinear_asym(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(z_w), _p(colsum),
+                                         _p(s_tok), _p(z_tok), s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype,
+                                         _p(Y), self._stream(stream)), "qlinear_asym")
 
     def dtwq_quantize(self, X, s_ch, bits, Xq, s_row, stream=None):
         M, K = X.shape

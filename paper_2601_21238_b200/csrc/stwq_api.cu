@@ -314,6 +314,83 @@ int qlinear_chain(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t
     return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, 3, Xq_next, pdl, &chain, st);
 }
 
+// ---- asymmetric quantizer (Eq. 1 as printed)
+int stwq_calibrate_asym(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K, int P,
+                        const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok, void* stream)
+{
+    if (!ctx || !Xcal || !pos_ids || !s_tok || !z_tok) return STWQ_ERR_NULL;
+    if (rows <= 0 || K <= 0 || P <= 0 || P > (1 << 20)) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    int rc = ensure_cal(ctx, P);
+    if (rc != STWQ_OK) return rc;
+    return stwq_launch_calibrate_asym(ctx, ctx->ws_cal, Xcal, pos_ids, rows, K, P, s_ch, bits, pct_ppm, s_tok, z_tok,
+                                      static_cast<cudaStream_t>(stream));
+}
+
+int gps_fold_asym(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq, float* s_w,
+                  int32_t* z_w, int32_t* colsum, void* stream)
+{
+    if (!ctx || !W || !Wq || !s_w || !z_w || !colsum) return STWQ_ERR_NULL;
+    if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_fold_asym(ctx, W, N, K, s_ch, bits, Wq, s_w, z_w, colsum, static_cast<cudaStream_t>(stream));
+}
+
+int stwq_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                       const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr,
+                       void* stream)
+{
+    if (!ctx || !X || !pos_ids || !s_tok || !z_tok || !Xq || !rowcorr) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || P <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if ((K & 15) != 0 || !aligned16(X) || !aligned16(Xq)) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_quantize_asym(ctx, X, pos_ids, M, K, s_ch, s_tok, z_tok, P, bits, Xq, rowcorr,
+                                     static_cast<cudaStream_t>(stream));
+}
+
+int qlinear_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
+                 const float* s_w, const int32_t* z_w, const int32_t* colsum, const float* s_tok, const int32_t* z_tok,
+                 int P, const float* s_ch, const float* bias, int bits, int act, int out_dtype, void* Y, void* stream)
+{
+    if (!ctx || !pos_ids || !s_tok || !s_w || !z_w || !colsum || !z_tok) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(X, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if (K > 32768 || M > (int64_t)0x7fffffff) return STWQ_ERR_DIM;     // the corrections stay inside int32
+    // the corrected epilogue lives in the CTA-pair kernel: 16-byte rows of Y, aligned per-column vectors
+    if (!stwq_qgemm2_supported(N, out_dtype, s_w, bias) || (N & 3) != 0 || !aligned16(z_w) || !aligned16(colsum))
+        return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc != STWQ_OK) return rc;
+    const size_t need = (size_t)M * 8;
+    if (ctx->ws_dyn_bytes < need) {
+        if (ctx->ws_dyn) {
+            cudaError_t e = cudaFree(ctx->ws_dyn);
+            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+            ctx->ws_dyn = nullptr;
+            ctx->ws_dyn_bytes = 0;
+        }
+        void* ptr = nullptr;
+        if (cudaMalloc(&ptr, need) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return STWQ_ERR_NOMEM;
+        }
+        ctx->ws_dyn = ptr;
+        ctx->ws_dyn_bytes = need;
+    }
+    int32_t* rowcorr = static_cast<int32_t*>(ctx->ws_dyn);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = stwq_launch_quantize_asym(ctx, X, pos_ids, M, K, s_ch, s_tok, z_tok, P, bits, ctx->ws_xq, rowcorr, st);
+    if (rc != STWQ_OK) return rc;
+    const stwq_asym asym = {z_tok, z_w, colsum, rowcorr};
+    return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, false, nullptr,
+                              st, &asym);
+}
+
 int dtwq_quantize(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
                   float* s_row, void* stream)
 {

@@ -47,7 +47,7 @@ __global__ void cal_clear_kernel(void* base, int P)
 // One block per row (grid-stride). pass 0..3 histograms byte (3 - pass) of the bit pattern.
 __global__ void __launch_bounds__(kThreads)
 cal_hist_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t rows,
-                int K, int P, const float* __restrict__ s_ch, void* base, int pass,
+                int K, int P, const float* __restrict__ s_ch, void* base, int pass, int signed_keys,
                 uint32_t* __restrict__ status)
 {
     __shared__ uint32_t bins[256];
@@ -67,8 +67,11 @@ cal_hist_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
         bool bad = false;
         for (int k = threadIdx.x; k < K; k += kThreads) {
             const float t = s_ch ? __fmul_rn(x[k], __fdiv_rn(1.0f, s_ch[k])) : x[k];
-            const uint32_t b = __float_as_uint(t) & 0x7fffffffu;
-            if (b >= 0x7f800000u) bad = true;
+            const uint32_t raw = __float_as_uint(t);
+            if ((raw & 0x7fffffffu) >= 0x7f800000u) bad = true;
+            // key that sorts like the value: |t| for the symmetric range, or the usual
+            // order-preserving map of a signed float for the two-sided one
+            const uint32_t b = signed_keys ? (raw ^ ((raw >> 31) ? 0xffffffffu : 0x80000000u)) : (raw & 0x7fffffffu);
             const bool match = (pass == 0) || ((b >> (shift + 8)) == (prefix >> (shift + 8)));
             if (match) atomicAdd(&bins[(b >> shift) & 255u], 1u);
         }
@@ -81,8 +84,11 @@ cal_hist_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
 }
 
 // One thread per position: locate the bin that holds the rank, extend the prefix, clear bins.
+// raw_out == nullptr: s_tok[p] = delta of the selected |value|. Otherwise the selected signed value
+// itself goes to raw_out[p] (0 for a position without rows), and with `mirror` the rank counts from
+// the top (rank n + 1 - r), which selects the lower end of a two-sided range.
 __global__ void cal_select_kernel(void* base, int P, int pass, uint32_t pct_ppm, int bits,
-                                  float* __restrict__ s_tok)
+                                  float* __restrict__ s_tok, float* __restrict__ raw_out, int mirror)
 {
     CalWs w = cal_ws(base, P);
     const int p = blockIdx.x * blockDim.x + threadIdx.x;
@@ -94,12 +100,14 @@ __global__ void cal_select_kernel(void* base, int P, int pass, uint32_t pct_ppm,
         for (int i = 0; i < 256; ++i) n += h[i];
         if (n == 0ull) {
             w.rank[p] = 0ull;
-            s_tok[p] = 1.0f;
+            if (raw_out) raw_out[p] = 0.0f;
+            else s_tok[p] = 1.0f;
             return;
         }
         rank = ((unsigned long long)pct_ppm * n + 999999ull) / 1000000ull;
         if (rank < 1ull) rank = 1ull;
         if (rank > n) rank = n;
+        if (mirror) rank = n + 1ull - rank;
     } else if (rank == 0ull) {
         return;
     }
@@ -115,14 +123,30 @@ __global__ void cal_select_kernel(void* base, int P, int pass, uint32_t pct_ppm,
     const uint32_t prefix = w.prefix[p] | ((uint32_t)bin << shift);
     w.prefix[p] = prefix;
     w.rank[p] = rank - cum;
-    if (pass == 3) s_tok[p] = stwq_delta(__uint_as_float(prefix), bits);
+    if (pass == 3) {
+        if (raw_out) raw_out[p] = __uint_as_float((prefix & 0x80000000u) ? (prefix ^ 0x80000000u) : ~prefix);
+        else s_tok[p] = stwq_delta(__uint_as_float(prefix), bits);
+    }
+}
+
+__global__ void cal_asym_finalize_kernel(const float* __restrict__ up, const float* __restrict__ down, int P, int bits,
+                                         float* __restrict__ s_tok, int32_t* __restrict__ z_tok)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= P) return;
+    float d;
+    int zs;
+    stwq_asym_params(down[p], up[p], bits, d, zs);
+    s_tok[p] = d;
+    z_tok[p] = zs;
 }
 
 }  // namespace
 
 size_t stwq_calibrate_ws_bytes(int P)
 {
-    return (size_t)P * 256 * 8 + (size_t)P * 8 + (size_t)P * 4 + 16;
+    // histograms, ranks, prefixes, then two float vectors for the two-sided (asymmetric) range
+    return (size_t)P * 256 * 8 + (size_t)P * 8 + (size_t)P * 4 + 16 + (size_t)P * 8;
 }
 
 int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids,
@@ -136,10 +160,37 @@ int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int3
     int64_t hist_blocks = rows < (int64_t)ctx->sm_count * 16 ? rows : (int64_t)ctx->sm_count * 16;
     for (int pass = 0; pass < 4; ++pass) {
         cal_hist_kernel<<<(unsigned)hist_blocks, kThreads, 0, st>>>(Xcal, pos_ids, rows, K, P, s_ch,
-                                                                    ws, pass, ctx->d_status);
-        cal_select_kernel<<<(P + 127) / 128, 128, 0, st>>>(ws, P, pass, pct_ppm, bits, s_tok);
+                                                                    ws, pass, 0, ctx->d_status);
+        cal_select_kernel<<<(P + 127) / 128, 128, 0, st>>>(ws, P, pass, pct_ppm, bits, s_tok, nullptr, 0);
         ctx->launches += 2;
     }
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+// Two-sided calibration (asymmetric quantizer): the same radix selection on order-preserving keys
+// of the signed values, once for the upper end (rank r) and once for the lower (rank n + 1 - r).
+int stwq_launch_calibrate_asym(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K,
+                               int P, const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok,
+                               cudaStream_t st)
+{
+    float* up = reinterpret_cast<float*>(reinterpret_cast<uint8_t*>(ws) + (((size_t)P * 256 * 8 + (size_t)P * 8 + (size_t)P * 4 + 15) & ~(size_t)15));
+    float* down = up + P;
+    const int clear_blocks = (int)(((size_t)P * 256 + 255) / 256 < 1024 ? ((size_t)P * 256 + 255) / 256 : 1024);
+    const int64_t hist_blocks = rows < (int64_t)ctx->sm_count * 16 ? rows : (int64_t)ctx->sm_count * 16;
+    for (int side = 0; side < 2; ++side) {
+        cal_clear_kernel<<<clear_blocks, 256, 0, st>>>(ws, P);
+        ctx->launches += 1;
+        for (int pass = 0; pass < 4; ++pass) {
+            cal_hist_kernel<<<(unsigned)hist_blocks, kThreads, 0, st>>>(Xcal, pos_ids, rows, K, P, s_ch, ws, pass, 1,
+                                                                        ctx->d_status);
+            cal_select_kernel<<<(P + 127) / 128, 128, 0, st>>>(ws, P, pass, pct_ppm, bits, nullptr, side == 0 ? up : down,
+                                                               side);
+            ctx->launches += 2;
+        }
+    }
+    cal_asym_finalize_kernel<<<(P + 127) / 128, 128, 0, st>>>(up, down, P, bits, s_tok, z_tok);
+    ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
 }

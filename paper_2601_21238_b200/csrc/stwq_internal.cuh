@@ -48,12 +48,28 @@ struct stwq_chain {
     int bits_next;
 };
 
+// Zero points of the asymmetric quantizer (Eq. 1 as printed) and the sums its correction needs.
+struct stwq_asym {
+    const int32_t* z_tok;      // [P] signed zero point per position
+    const int32_t* z_w;        // [N] signed zero point per output channel
+    const int32_t* colsum;     // [N] sum_k Wq[n,k]
+    const int32_t* rowcorr;    // [M] sum_k Xq[m,k] - K z_tok[pos[m]]
+};
+
 // Launchers (host). Each returns STWQ_OK or STWQ_ERR_CUDA and bumps ctx->launches.
 int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,
                          const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq,
                          bool dependent, cudaStream_t st);
 int stwq_launch_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
                               const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, cudaStream_t st);
+int stwq_launch_fold_asym(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
+                          float* s_w, int32_t* z_w, int32_t* colsum, cudaStream_t st);
+int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                              const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr,
+                              cudaStream_t st);
+int stwq_launch_calibrate_asym(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K,
+                               int P, const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok,
+                               cudaStream_t st);
 int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);
@@ -67,7 +83,7 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize,
-                       const struct stwq_chain* chain, cudaStream_t st);
+                       const struct stwq_chain* chain, cudaStream_t st, const struct stwq_asym* asym = nullptr);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);
@@ -91,6 +107,29 @@ __device__ __forceinline__ float stwq_delta(float a, int bits)
     const float levels = (float)((1 << bits) - 1);
     float d = __fdiv_rn(__fadd_rn(a, a), levels);
     return fmaxf(d, 5.421010862427522e-20f);
+}
+
+// Eq. 1 as printed, for a range widened to contain 0: delta = (up - down) / (2^b - 1), z =
+// round(-down / delta) clamped to [0, 2^b - 1]; returned as the signed zero point z - 2^(b-1)
+// that goes with codes stored in signed containers.
+__device__ __forceinline__ void stwq_asym_params(float lo, float hi, int bits, float& delta, int& zs)
+{
+    const float levels = (float)((1 << bits) - 1);
+    if (lo > 0.0f) lo = 0.0f;
+    if (hi < 0.0f) hi = 0.0f;
+    float d = __fdiv_rn(__fsub_rn(hi, lo), levels);
+    if (!(d > 0.0f)) d = 1.0f;
+    d = fmaxf(d, 5.421010862427522e-20f);
+    float z = rintf(__fdiv_rn(-lo, d));
+    z = fminf(fmaxf(z, 0.0f), levels);
+    delta = d;
+    zs = (int)z - (1 << (bits - 1));
+}
+// signed asymmetric code: clamp(round(u) + zs) (NaN -> round 0; the rounded value saturates at +-2^20 first)
+__device__ __forceinline__ int stwq_code_asym(float u, int zs, int qmin, int qmax)
+{
+    const int r = max(min(__float2int_rn(u), 1048576), -1048576);
+    return max(min(r + zs, qmax), qmin);
 }
 
 // round to nearest even (NaN -> 0, +-Inf and large values saturate), clamp to the b-bit range.

@@ -52,6 +52,11 @@ struct Gemm2Params {
     int full_units, num_units, nsplit, kb_per_split;
     int32_t* partial;          // [tail tile][split][rank][warp][128 x 32 lanes] int32
     uint32_t* counters;        // [tail tile][rank][warp]
+    // asymmetric quantizer (ASYM): acc - z_w[n] rowcorr[m] - z_tok[pos] colsum[n] replaces acc
+    const int32_t* z_tok;      // [P]
+    const int32_t* z_w;        // [N]
+    const int32_t* colsum;     // [N]
+    const int32_t* rowcorr;    // [M]
     // chained output (OUT == kOutCodes): the next layer's static quantizer applied to act(z)
     const float* s_ch_next;    // [N] or NULL
     const float* s_tok_next;   // [P]
@@ -72,7 +77,8 @@ struct Smem2 {
     static constexpr int kOffB = STAGES * kABytes;
     static constexpr int kOffStage = STAGES * kStageBytes;  // per epilogue warp: two staging tiles of 32 rows x 128 B
     static constexpr int kOffScale = kOffStage + (STORE == 0 ? EPI * 8192 : 0); // per epilogue warp: s_w and bias of its columns
-    static constexpr int kOffBars = kOffScale + 3 * BN * 4 * 4;   // s_w, bias and (chained output) the next layer's 1 / s_ch
+    static constexpr int kOffBars = kOffScale + 4 * BN * 4 * 4;   // s_w, bias, and either the next layer's 1 / s_ch (chained
+                                                                  // output) or the weights' zero points and code sums (asymmetric)
     static constexpr int kNumBars = 2 * STAGES + 4;
     static constexpr int kOffMisc = kOffBars + kNumBars * 8;
     static constexpr int kTotal = kOffMisc + 16;
@@ -108,8 +114,8 @@ __device__ __forceinline__ uint4 ld_cg_v4(const void* ptr)
     return v;
 }
 
-// STORE: see Smem2.
-template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
+// STORE: see Smem2. ASYM: zero-point correction of the accumulators (Eq. 1 with zero points).
+template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE, bool ASYM>
 __global__ void __launch_bounds__(64 + 32 * EPI, 1)
 qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
               const __grid_constant__ CUtensorMap tmY, const Gemm2Params p)
@@ -234,9 +240,11 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         constexpr int kMyCols = kMyChunks * kChunkCols;
         static_assert(kChunks % kSubs == 0, "chunks must divide among the warps of a quarter");
         const uint32_t stage0 = base + L::kOffStage + (uint32_t)ew * 8192u;   // two staging tiles (STORE == 0)
-        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 3 * kMyCols;
+        float* my_sw = reinterpret_cast<float*>(smem + L::kOffScale) + ew * 4 * kMyCols;
         float* my_bias = my_sw + kMyCols;
         float* my_rcn = my_bias + kMyCols;
+        int* my_zw = reinterpret_cast<int*>(my_rcn);       // asymmetric: the third and fourth arrays hold integers
+        int* my_cs = my_zw + kMyCols;
         const uint32_t tempty0 = mapa_u32(bar_tempty(0), 0);
         constexpr int kElem = (OUT == STWQ_OUT_BF16) ? 2 : (OUT == kOutCodes ? 1 : 4);
         uint32_t t = 0, nstore = 0;
@@ -250,6 +258,27 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             const int n0 = (tile % p.tiles_n) * BN;
             const int64_t row = (int64_t)m0 + q * 32 + lane;
             float st = 0.0f, rtn = 0.0f;
+            int zx = 0, Rm = 0;
+            if (ASYM) {
+                __syncwarp();
+                for (int i = lane * 4; i < kMyCols; i += 128) {
+                    const int k = i / kChunkCols;
+                    const int col = n0 + (sub + k * kSubs) * kChunkCols + (i % kChunkCols);
+                    int4 zw = make_int4(0, 0, 0, 0), cs = make_int4(0, 0, 0, 0);
+                    if (col < p.N) {
+                        zw = __ldg(reinterpret_cast<const int4*>(p.z_w + col));
+                        cs = __ldg(reinterpret_cast<const int4*>(p.colsum + col));
+                    }
+                    *reinterpret_cast<int4*>(my_zw + i) = zw;
+                    *reinterpret_cast<int4*>(my_cs + i) = cs;
+                }
+                if (row < p.M) {
+                    const int pos = p.pos_ids[row];
+                    Rm = p.rowcorr[row];
+                    if (pos >= 0 && pos < p.P) zx = p.z_tok[pos];
+                }
+                __syncwarp();
+            }
             if (OUT != STWQ_OUT_INT32) {
                 // column scales and biases of this warp's chunks -> its private shared copy, and
                 // the row scale, all fetched before the accumulator is waited for
@@ -341,6 +370,22 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             const uint4 a = ld_cg_v4(src + ((size_t)(l * 8 + g) * 32 + lane) * 4);
                             racc[l][g * 4 + 0] += a.x; racc[l][g * 4 + 1] += a.y; racc[l][g * 4 + 2] += a.z; racc[l][g * 4 + 3] += a.w;
                         }
+                }
+            }
+            if (ASYM) {
+                // zero-point correction, exact in int32: acc - z_w[n] rowcorr[m] - z_tok[pos] colsum[n]
+#pragma unroll
+                for (int l = 0; l < kLoads; ++l) {
+                    const int k = l / kLoadsPerChunk, h = l % kLoadsPerChunk;
+#pragma unroll
+                    for (int j = 0; j < 32; j += 4) {
+                        const int4 zw = *reinterpret_cast<const int4*>(my_zw + k * kChunkCols + h * 32 + j);
+                        const int4 cs = *reinterpret_cast<const int4*>(my_cs + k * kChunkCols + h * 32 + j);
+                        racc[l][j + 0] = (uint32_t)((int)racc[l][j + 0] - zw.x * Rm - zx * cs.x);
+                        racc[l][j + 1] = (uint32_t)((int)racc[l][j + 1] - zw.y * Rm - zx * cs.y);
+                        racc[l][j + 2] = (uint32_t)((int)racc[l][j + 2] - zw.z * Rm - zx * cs.z);
+                        racc[l][j + 3] = (uint32_t)((int)racc[l][j + 3] - zw.w * Rm - zx * cs.w);
+                    }
                 }
             }
 #pragma unroll
@@ -513,14 +558,14 @@ int stwq_encode_2d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int 
 
 namespace {
 
-template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE>
+template <int BN, int STAGES, int EPI, int OUT, int ACT, int STORE, bool ASYM = false>
 int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, const CUtensorMap& tmY,
                    const Gemm2Params& p, bool dependent, cudaStream_t st)
 {
     using L = Smem2<BN, STAGES, EPI, STORE>;
-    auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT, STORE>;
+    auto kern = qgemm2_kernel<BN, STAGES, EPI, OUT, ACT, STORE, ASYM>;
     const uint64_t bit = 1ull << ((BN == 256 ? 0 : 16) + OUT * 4 + ACT);
-    uint64_t& mask = ctx->configured_pair[STORE];
+    uint64_t& mask = ctx->configured_pair[STORE + (ASYM ? 2 : 0)];
     if (!(mask & bit)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic);
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
@@ -564,6 +609,22 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
 {
 #define STWQ_CASE(O, A) \
     if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
+    if (p.z_w != nullptr) {                               // asymmetric: staged-store variant of 256-wide tiles only
+        if constexpr (BN == 256 && STORE == 0) {
+#define STWQ_ACASE(O, A) \
+    if (out_dtype == O && act == A) return launch_variant<BN, STAGES, EPI, O, A, STORE, true>(ctx, tmA, tmB, tmY, p, dependent, st);
+            if (out_dtype == STWQ_OUT_INT32)
+                return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE, true>(ctx, tmA, tmB, tmY, p, dependent, st);
+            STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_NONE)
+            STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
+            STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+            STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
+            STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
+            STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+#undef STWQ_ACASE
+        }
+        return STWQ_ERR_DIM;
+    }
     if (out_dtype == STWQ_OUT_INT32)
         return launch_variant<BN, STAGES, EPI, STWQ_OUT_INT32, STWQ_ACT_NONE, STORE>(ctx, tmA, tmB, tmY, p, dependent, st);
     if (out_dtype == kOutCodes) {                         // 128-column chunks: 256-wide tiles only
@@ -601,15 +662,20 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
-                       int act, int out_dtype, void* Y, bool after_quantize, const stwq_chain* chain, cudaStream_t st)
+                       int act, int out_dtype, void* Y, bool after_quantize, const stwq_chain* chain, cudaStream_t st,
+                       const stwq_asym* asym)
 {
     // 256-wide tiles whenever N has more than 128 columns: a 128-wide tile needs 1.5x the
     // L2 -> shared-memory bytes per multiply-accumulate and is bound by that feed.
     const int tiles_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
-    int bn = (N > 128 || out_dtype == kOutCodes) ? 256 : 128;
+    int bn = (N > 128 || out_dtype == kOutCodes || asym != nullptr) ? 256 : 128;
     if (ctx->force_bn == 128 || ctx->force_bn == 256) bn = ctx->force_bn;
 
     Gemm2Params p;
+    p.z_tok = asym ? asym->z_tok : nullptr;
+    p.z_w = asym ? asym->z_w : nullptr;
+    p.colsum = asym ? asym->colsum : nullptr;
+    p.rowcorr = asym ? asym->rowcorr : nullptr;
     p.Y = Y;
     p.s_ch_next = chain ? chain->s_ch_next : nullptr;
     p.s_tok_next = chain ? chain->s_tok_next : nullptr;
@@ -687,9 +753,9 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     // Long main loops hide the epilogue anyway and gain from the deeper ring that the
     // register-direct epilogue leaves room for; short ones (and GELU) are bound by the epilogue,
     // which costs the fewest shared-memory cycles when it goes through staged TMA stores.
-    bool direct = K >= 1536 && act == STWQ_ACT_NONE;
+    bool direct = K >= 1536 && act == STWQ_ACT_NONE && asym == nullptr;
     if (ctx->debug == 1) direct = false;                  // tuning: force one or the other
-    if (ctx->debug == 2) direct = true;
+    if (ctx->debug == 2 && asym == nullptr) direct = true;
     if (direct) return launch_bn<256, 6, 8, 1>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
     return launch_bn<256, 4, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
 }

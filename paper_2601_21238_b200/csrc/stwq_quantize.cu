@@ -219,6 +219,58 @@ quantize_bf16_kernel(const uint16_t* __restrict__ X, const int32_t* __restrict__
     }
 }
 
+// ---------------------------------------------------------------------------- asymmetric codes
+// Eq. 1 as printed with a static zero point per position: cs = clamp(round(u) + zs[pos], -h, h-1).
+// Besides the codes the kernel accumulates rowcorr[m] = sum_k cs[m,k] - K zs[pos[m]] (zeroed by the
+// launcher; one atomic per warp and row), which the GEMM epilogue multiplies by the weights'
+// zero points. A warp owns a 512-column span of a row, as in quantize_kernel.
+__global__ void __launch_bounds__(kThreads)
+quantize_asym_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
+                     const float* __restrict__ s_ch, const float* __restrict__ s_tok, const int32_t* __restrict__ z_tok,
+                     int P, int qmin, int qmax, int8_t* __restrict__ Xq, int32_t* __restrict__ rowcorr, int spans,
+                     int64_t row_stride, uint32_t* __restrict__ status)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    const int span = (int)(warp % spans);
+    const int col0 = span * kSpan + lane * 4;
+    float rc[16];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const int c = col0 + j * 128;
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
+    }
+    for (int64_t m = warp / spans; m < M; m += row_stride) {
+        const int p = pos_ids[m];
+        const bool ok = (p >= 0) && (p < P);
+        const float rt = ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
+        const int zs = ok ? z_tok[p] : 0;
+        if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+        int sum = 0;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int c = col0 + j * 128;
+            if (c < K) {
+                const float4 v = ld_stream(X + m * K + c);
+                const int q0 = stwq_code_asym(__fmul_rn(__fmul_rn(v.x, rc[j * 4 + 0]), rt), zs, qmin, qmax);
+                const int q1 = stwq_code_asym(__fmul_rn(__fmul_rn(v.y, rc[j * 4 + 1]), rt), zs, qmin, qmax);
+                const int q2 = stwq_code_asym(__fmul_rn(__fmul_rn(v.z, rc[j * 4 + 2]), rt), zs, qmin, qmax);
+                const int q3 = stwq_code_asym(__fmul_rn(__fmul_rn(v.w, rc[j * 4 + 3]), rt), zs, qmin, qmax);
+                sum += q0 + q1 + q2 + q3;
+                uint32_t hi, packed;
+                asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+                asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(packed) : "r"(q1), "r"(q0), "r"(hi));
+                *reinterpret_cast<uint32_t*>(Xq + m * K + c) = packed;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (lane == 0) atomicAdd(rowcorr + m, sum - (span == 0 ? K * zs : 0));
+    }
+}
+
 // ---------------------------------------------------------------------------- TMA ring variant
 // X is dense, so a tile is simply 4096 consecutive floats of the flat array (16 KB of contiguous
 // DRAM, which streams a quarter faster than sixteen 1 KB pieces of sixteen rows: 6.0-6.4 against
@@ -419,6 +471,27 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
 }
 
 }  // namespace
+
+int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
+                              const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr,
+                              cudaStream_t st)
+{
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    const int spans = (K + kSpan - 1) / kSpan;
+    const int warps_per_block = kThreads / 32;
+    int64_t rows_in_flight = (int64_t)ctx->sm_count * 6 * warps_per_block / spans;
+    if (rows_in_flight < 1) rows_in_flight = 1;
+    if (rows_in_flight > M) rows_in_flight = M;
+    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    const unsigned blocks = (unsigned)(rows_in_flight * spans / warps_per_block);
+    cudaError_t e = cudaMemsetAsync(rowcorr, 0, (size_t)M * sizeof(int32_t), st);
+    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    quantize_asym_kernel<<<blocks, kThreads, 0, st>>>(X, pos_ids, M, K, s_ch, s_tok, z_tok, P, qmin, qmax, Xq, rowcorr,
+                                                      spans, rows_in_flight, ctx->d_status);
+    ctx->launches += 1;
+    e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
 
 int stwq_launch_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K,
                               const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, cudaStream_t st)

@@ -537,3 +537,70 @@ def test_quantize_bf16_input_bit_exact(gpu, bits, shape):
         gpu.ctx.stwq_quantize_bf16(Xb, gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
         assert gpu.ctx.stwq_device_status() == 0
         np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
+
+
+# ----------------------------------------------------------------------------- asymmetric quantizer (Eq. 1 as printed)
+@pytest.mark.parametrize("bits", [8, 6])
+def test_asym_offline_calls_bit_exact(gpu, bits):
+    torch = gpu.torch
+    N, K = 70, 208
+    W = (0.02 * rng.standard_normal((N, K)) + 0.01 * rng.standard_normal((N, 1))).astype(np.float32)
+    W[5] = np.abs(W[5]) + 0.01
+    W[6] = 0.0
+    s_ch = rng.uniform(0.3, 4, K).astype(np.float32)
+    for sc in (s_ch, None):
+        ref = oracle.gps_fold_asym(W, sc, bits)
+        Wq = torch.full((N, K), 99, dtype=torch.int8, device=gpu.dev)
+        sw = torch.zeros(N, device=gpu.dev)
+        zw = torch.zeros(N, dtype=torch.int32, device=gpu.dev)
+        cs = torch.zeros(N, dtype=torch.int32, device=gpu.dev)
+        gpu.ctx.gps_fold_asym(gpu.T(W), gpu.T(sc), bits, Wq, sw, zw, cs)
+        for got, want in zip((Wq, sw, zw, cs), ref):
+            np.testing.assert_array_equal(got.cpu().numpy(), want)
+    S, P = 6, 9
+    pos = np.tile(np.arange(P, dtype=np.int32), S)
+    X = (rng.standard_normal((S * P, K)) * (1 + pos[:, None]) + 0.3 * pos[:, None]).astype(np.float32)
+    X[pos == 2] = np.abs(X[pos == 2])
+    perm = rng.permutation(S * P)
+    X, pos = X[perm], pos[perm]
+    for pct in (1000000, 990000, 500000):
+        for sc in (s_ch, None):
+            rs, rz = oracle.stwq_calibrate_asym(X, pos, P + 2, sc, bits, pct)
+            st = torch.zeros(P + 2, device=gpu.dev)
+            zt = torch.zeros(P + 2, dtype=torch.int32, device=gpu.dev)
+            gpu.ctx.stwq_calibrate_asym(gpu.T(X), gpu.T(pos), P + 2, gpu.T(sc), bits, pct, st, zt)
+            assert gpu.ctx.stwq_device_status() == 0
+            np.testing.assert_array_equal(st.cpu().numpy(), rs)
+            np.testing.assert_array_equal(zt.cpu().numpy(), rz)
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("act", [0, 1])
+@pytest.mark.parametrize("shape", [(333, 400, 328), (1500, 1024, 768)])
+def test_qlinear_asym_matches_the_oracle(gpu, shape, act, bits):
+    """Asymmetric codes and row corrections bit-exact; the corrected int32 accumulators (which equal
+    sum_k (cs - zx)(ws - zw)) bit-exact; outputs within the usual tolerance."""
+    torch = gpu.torch
+    M, K, N = shape
+    L = wl.scaled(wl.config_layers(2)[2], batch=3, P=680, K=K, N=N, act=act, bits=bits)
+    W, b = wl.weights(L) + np.float32(0.004), wl.bias(L)
+    X = (wl.activations(L)[:M] + np.float32(0.8)).astype(np.float32)           # off-centre on purpose
+    pos = wl.positions(L)[:M]
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    s_tok, z_tok = oracle.stwq_calibrate_asym(X, pos, L.P, s_ch, bits, 999000)
+    Wq, s_w, z_w, cs = oracle.gps_fold_asym(W, s_ch, bits)
+    ref = oracle.qlinear_asym(X, pos, Wq, s_w, z_w, cs, s_tok, z_tok, s_ch, b, bits, act)
+    Xq = torch.full((M, K), 99, dtype=torch.int8, device=gpu.dev)
+    rc = torch.full((M,), 7, dtype=torch.int32, device=gpu.dev)
+    gpu.ctx.stwq_quantize_asym(gpu.T(X), gpu.T(pos), gpu.T(s_ch), gpu.T(s_tok), gpu.T(z_tok), bits, Xq, rc)
+    np.testing.assert_array_equal(Xq.cpu().numpy(), ref["Xq"])
+    np.testing.assert_array_equal(rc.cpu().numpy(), ref["rowcorr"])
+    args = [gpu.T(a) for a in (X, pos, Wq, s_w, z_w, cs, s_tok, z_tok, s_ch, b)]
+    Yi = _out_tensor(gpu, M, N, "int32")
+    gpu.ctx.qlinear_asym(*args, bits, act, gpu.B.OUT_INT32, Yi)
+    np.testing.assert_array_equal(Yi.cpu().numpy(), ref["acc"])
+    for out in ("fp32", "bf16"):
+        Y = _out_tensor(gpu, M, N, out)
+        gpu.ctx.qlinear_asym(*args, bits, act, _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+        assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"qlinear_asym {out}")
