@@ -34,8 +34,8 @@ PCT = 999900
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 INT8_OVER_BF16 = 2.0          # nominal dense tensor ratio (4.5 vs 2.25 PFLOP/s)
 # DRAM bytes (read + write) per launch of the dominant kernel, mean over the four layer shapes, from
-# the ncu capture summarised in profiles/qgemm2_kernel_config2.md (22.5, 12.3, 48.6, 51.6 MB).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 33.8e6
+# the ncu capture summarised in profiles/qgemm2_kernel_config2.md (24.7, 12.3, 46.4, 51.5 MB).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 33.7e6
 
 
 def measured_peaks():

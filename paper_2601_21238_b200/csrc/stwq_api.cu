@@ -55,6 +55,28 @@ int ensure_cal(stwq_ctx* ctx, int P)
     return STWQ_OK;
 }
 
+// Per-row workspace of qlinear_dtwq (row scales + row ids) and qlinear_asym (row corrections).
+int ensure_dyn(stwq_ctx* ctx, size_t bytes)
+{
+    if (ctx->ws_dyn_bytes >= bytes) return STWQ_OK;
+    if (ctx->ws_dyn) {
+        cudaError_t e = cudaFree(ctx->ws_dyn);          // synchronises
+        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+        ctx->ws_dyn = nullptr;
+        ctx->ws_dyn_bytes = 0;
+    }
+    void* p = nullptr;
+    cudaError_t e = cudaMalloc(&p, bytes);
+    if (e != cudaSuccess) {
+        ctx->last_cuda_error = (int)e;
+        (void)cudaGetLastError();
+        return STWQ_ERR_NOMEM;
+    }
+    ctx->ws_dyn = p;
+    ctx->ws_dyn_bytes = bytes;
+    return STWQ_OK;
+}
+
 // Make the context's device current for the duration of a call.
 struct DeviceGuard {
     int prev = -1;
@@ -366,22 +388,8 @@ int qlinear_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t 
     DeviceGuard g(ctx->device);
     rc = ensure_xq(ctx, (size_t)M * (size_t)K);
     if (rc != STWQ_OK) return rc;
-    const size_t need = (size_t)M * 8;
-    if (ctx->ws_dyn_bytes < need) {
-        if (ctx->ws_dyn) {
-            cudaError_t e = cudaFree(ctx->ws_dyn);
-            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-            ctx->ws_dyn = nullptr;
-            ctx->ws_dyn_bytes = 0;
-        }
-        void* ptr = nullptr;
-        if (cudaMalloc(&ptr, need) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return STWQ_ERR_NOMEM;
-        }
-        ctx->ws_dyn = ptr;
-        ctx->ws_dyn_bytes = need;
-    }
+    rc = ensure_dyn(ctx, (size_t)M * 8);
+    if (rc != STWQ_OK) return rc;
     int32_t* rowcorr = static_cast<int32_t*>(ctx->ws_dyn);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rc = stwq_launch_quantize_asym(ctx, X, pos_ids, M, K, s_ch, s_tok, z_tok, P, bits, ctx->ws_xq, rowcorr, st);
@@ -415,22 +423,8 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
     DeviceGuard g(ctx->device);
     rc = ensure_xq(ctx, (size_t)M * (size_t)K);
     if (rc != STWQ_OK) return rc;
-    const size_t need = (size_t)M * 8;
-    if (ctx->ws_dyn_bytes < need) {
-        if (ctx->ws_dyn) {
-            cudaError_t e = cudaFree(ctx->ws_dyn);
-            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-            ctx->ws_dyn = nullptr;
-            ctx->ws_dyn_bytes = 0;
-        }
-        void* ptr = nullptr;
-        if (cudaMalloc(&ptr, need) != cudaSuccess) {
-            (void)cudaGetLastError();
-            return STWQ_ERR_NOMEM;
-        }
-        ctx->ws_dyn = ptr;
-        ctx->ws_dyn_bytes = need;
-    }
+    rc = ensure_dyn(ctx, (size_t)M * 8);
+    if (rc != STWQ_OK) return rc;
     float* s_row = static_cast<float*>(ctx->ws_dyn);
     int32_t* row_ids = reinterpret_cast<int32_t*>(s_row + M);
     cudaStream_t st = static_cast<cudaStream_t>(stream);

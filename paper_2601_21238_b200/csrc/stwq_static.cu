@@ -75,6 +75,7 @@ int setup_device(int device, DeviceSlot** out)
         s.ctx.sm_count = sms;
         s.ctx.l2_bytes = l2;
         s.ctx.wait_limit_ms = 2000;
+        s.ctx.force_ksplit = -1;        // the split-K tail keeps partial sums in allocated scratch: never here
         s.ctx.d_status = reinterpret_cast<uint32_t*>(base);
         s.ctx.ws_xq = reinterpret_cast<int8_t*>(base + kHeaderBytes);
         s.ctx.ws_xq_bytes = kCodeBytes;

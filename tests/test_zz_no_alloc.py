@@ -57,6 +57,27 @@ def test_qlinear_static_matches_qlinear_twice_in_a_row():
                         # and both sit inside the tolerance of the other parity tests
                         assert torch.equal(got, want)
                         assert_close(got.float().cpu().numpy(), ref, rtol, f"qlinear_static {L.name}")
+        # a shape for which qlinear cuts its two tiles along K and exchanges partial sums through
+        # scratch that its context allocates: qlinear_static must give the same bits without it,
+        # and the device's free memory must not move across its calls (after one warm-up call,
+        # which loads the kernel's code)
+        L2 = wl.scaled(wl.config_layers(1)[0], K=4096, N=512, P=64, batch=4, bits=8, act=0)
+        assert L2.M * L2.K <= pk.binding.STATIC_MAX_CODES
+        par = prepare(L2, samples=2, gps_n=32)
+        X, pos = wl.activations(L2), wl.positions(L2)
+        ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], L2.bits, L2.act)
+        d2 = {k: T(par[k]) for k in ("Wq", "s_w", "s_tok", "s_ch", "bias")}
+        Xd, pd = T(X), T(pos)
+        got = torch.full((L2.M, L2.N), -5, dtype=torch.int32, device=dev)
+        args = (Xd, pd, d2["Wq"], d2["s_w"], d2["s_tok"], d2["s_ch"], d2["bias"], L2.bits, L2.act, pk.OUT_INT32, got)
+        pk.qlinear_static(*args)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info(0)[0]
+        for _ in range(3):
+            pk.qlinear_static(*args)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info(0)[0] == free_before
+        np.testing.assert_array_equal(got.cpu().numpy(), ref["acc"])
         # a problem larger than the fixed scratch is refused on the host, nothing is enqueued
         big_M = pk.binding.STATIC_MAX_CODES // 1024 + 1
         Xb = torch.zeros((big_M, 1024), device=dev)
