@@ -293,6 +293,16 @@ def gpu_arm(args):
                              "frac": round(sum(5.0 * s["L"].M * s["L"].K for s in S)
                                            / (sum(tq.values()) * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}}
 
+    if all(s["L"].decode for s in S):
+        # few-row layers: the GEMM is the weight-streaming kernel, bound by bytes, not by the pipe
+        byts = sum(float(s["L"].N) * s["L"].K + float(s["L"].M) * s["L"].K + 2.0 * s["L"].M * s["L"].N for s in S)
+        gbs = byts / (gemm_ms * 1e-3) / 1e9
+        roofline.update({"kernel": "decode_kernel (few-row CTA-pair GEMM, weights streamed once), mean over the layer shapes",
+                         "bound": "hbm", "achieved": round(gbs, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": round(gbs / peaks["hbm_gbs"], 4),
+                         "peak_source": f"hbm_gbs of {peaks['_source']} peaks; weights stay in L2 between replays",
+                         "traffic": None})
+
     # ---- end to end: pinned host X -> device -> qlinear -> device -> pinned host Y ------------
     hX = [torch.empty((s["L"].M, s["L"].K), dtype=torch.float32).pin_memory() for s in S]
     hY = [torch.empty_like(s["Y"], device="cpu").pin_memory() for s in S]

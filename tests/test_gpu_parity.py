@@ -181,7 +181,10 @@ def test_calibrate_flags_nonfinite_and_bad_positions(gpu):
 
 # ----------------------------------------------------------------------------- GEMM accumulators
 GEMM_SHAPES = [(1, 16, 16), (128, 256, 128), (128, 128, 2048), (129, 257, 16), (300, 520, 144), (77, 8, 48),
-               (256, 512, 384), (640, 1000, 1008), (1000, 136, 8192), (257, 3072, 1024), (2000, 1920, 1920)]
+               (256, 512, 384), (640, 1000, 1008), (1000, 136, 8192), (257, 3072, 1024), (2000, 1920, 1920),
+               # more tiles than CTA pairs with a last tile column half inside the matrix; one tile
+               # more than there are pairs
+               (2816, 1920, 256), (600, 640, 128), (19000, 256, 144)]
 
 
 @pytest.mark.parametrize("path", [1, 3, 0])      # CTA-pair GEMM, single-CTA GEMM, automatic choice
