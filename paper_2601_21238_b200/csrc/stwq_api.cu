@@ -1,11 +1,8 @@
 // C ABI of libstwq: context management, argument validation, and the composition of the
 // kernels into the calls declared in stwq.h. No arithmetic of the method lives here.
 #include <cuda.h>
-#include <dlfcn.h>
 
-#include <mutex>
 #include <new>
-#include <string>
 
 #include "stwq_internal.cuh"
 
@@ -110,26 +107,6 @@ int check_gemm_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int
     return STWQ_OK;
 }
 
-// Optional companion library with the shared-operand GEMM (single-GPU builds): looked up once,
-// next to this library; absent is normal and means every problem runs on the kernels in here.
-typedef int (*McLaunchFn)(stwq_ctx*, const int8_t*, const int32_t*, int64_t, int, int, const int8_t*, const float*,
-                          const float*, int, const float*, int, int, void*, int, void*);
-McLaunchFn mc_launch_fn()
-{
-    static std::once_flag once;
-    static McLaunchFn fn = nullptr;
-    std::call_once(once, [] {
-        Dl_info info;
-        if (!dladdr(reinterpret_cast<const void*>(&stwq_strerror), &info) || !info.dli_fname) return;
-        std::string path(info.dli_fname);
-        const size_t slash = path.rfind('/');
-        path = (slash == std::string::npos ? std::string() : path.substr(0, slash + 1)) + "libstwq_mc.so";
-        void* h = dlopen(path.c_str(), RTLD_NOW | RTLD_LOCAL);
-        if (h) fn = reinterpret_cast<McLaunchFn>(dlsym(h, "stwq_mc_launch"));
-    });
-    return fn;
-}
-
 int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
              const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias, int act,
              int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
@@ -141,13 +118,7 @@ int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M,
     if (decode)
         return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
                                   after_quantize, st);
-    const bool pair_ok = stwq_qgemm2_supported(N, out_dtype, s_w, bias);
-    if (ctx->gemm_path == 4 && pair_ok) {
-        McLaunchFn mc = mc_launch_fn();
-        return mc ? mc(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, after_quantize ? 1 : 0, st)
-                  : STWQ_ERR_DIM;
-    }
-    if (ctx->gemm_path != 3 && pair_ok)
+    if (ctx->gemm_path != 3 && stwq_qgemm2_supported(N, out_dtype, s_w, bias))
         return stwq_launch_qgemm2(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
                                   after_quantize, nullptr, st);
     return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
@@ -223,7 +194,7 @@ int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P)
 int stwq_set_option(stwq_ctx* ctx, int option, int value)
 {
     if (!ctx) return STWQ_ERR_NULL;
-    if (option == STWQ_OPT_GEMM_PATH && value >= 0 && value <= 4) {
+    if (option == STWQ_OPT_GEMM_PATH && value >= 0 && value <= 3) {
         ctx->gemm_path = value;
         return STWQ_OK;
     }
