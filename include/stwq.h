@@ -4,6 +4,7 @@
  * The inference hot path of PTQ4ARVG's quantized decoder, as a C library:
  *
  *   offline   stwq_calibrate   per-token-position activation scales      (Section 4.2)
+ *   offline   gps_scales       the per-channel scaling vector s of Eq. 2        (Section 4.1, Algorithm 1)
  *   offline   gps_fold         fold the per-channel scale into W, quantize W (Eq. 2, Appendix B)
  *   online    stwq_quantize    X -> int8 codes with the static scales     (Eq. 1, Eq. 2, Section 4.2)
  *   online    qlinear          quantize -> int8 GEMM -> dequantize (+bias, +GELU)
@@ -91,6 +92,26 @@ int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P);
 int stwq_calibrate(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K,
                    int P, const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok,
                    void* stream);
+
+/*
+ * Gain-Projected Scaling (Section 4.1, Eq. 13-16; Algorithm 1 of Appendix F): the per-input-channel
+ * scaling vector s of Eq. 2 from calibration activations and the layer's weights.
+ *   1. Q(X) per tensor, its range the nearest-rank percentile pct_ppm of |Xcal| (as stwq_calibrate
+ *      with one position), Q(W) per output channel with min-max range, both with the symmetric
+ *      quantizer of `bits` bits; dX = X - Q(X), dW = W - Q(W).
+ *   2. k* = the channel with the largest activation range max_t X[t,k] - min_t X[t,k] (lowest index
+ *      on ties); s[k*] = sqrt(R_x[k*] / R_w[k*]), R_w[k*] the range of column k* of W.
+ *   3. every other channel i:
+ *        variant 0 (Eq. 16):   s[i] = s[k*] sqrt(sum_t sum_n |dW[n,i] X[t,i]|) / sqrt(sum_t sum_n |W[n,i] dX[t,i]|)
+ *        variant 1 (the stationary point of the gain of Eq. 15):
+ *                              s[i] = s[k*] (sum dW^2 X^2 / sum W^2 dX^2)^(1/4)
+ *      A zero numerator, denominator or weight range gives 1; s is clamped to [1e-4, 1e4].
+ * Xcal [rows,K] fp32, W [N,K] fp32, s_ch [K] fp32 out, k_star (device int32, may be NULL) receives k*.
+ * Sums are accumulated in fp64 in a fixed order: repeatable, and within rounding of any other
+ * order of summation. Uses context workspace (allocated on first use or growth).
+ */
+int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const float* W, int N, int bits,
+               uint32_t pct_ppm, int variant, float* s_ch, int32_t* k_star, void* stream);
 
 /*
  * Equivalent scaling, weight side (Eq. 2: Y = (X / s)(s * W)), then per-output-channel

@@ -21,7 +21,7 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
-            "stwq_quantize_asym", "qlinear_asym"]
+            "stwq_quantize_asym", "qlinear_asym", "gps_scales"]
 
 _lib = None
 
@@ -58,6 +58,7 @@ def load_library():
     L.stwq_reserve.argtypes = [vp, i64, i32, i32]
     L.stwq_calibrate.argtypes = [vp, vp, vp, i64, i32, i32, vp, i32, u32, vp, vp]
     L.gps_fold.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, vp]
+    L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
@@ -149,6 +150,12 @@ class Context:
         rows, K = Xcal.shape
         self._check(self._L.stwq_calibrate(self._h, _p(Xcal), _p(pos_ids), rows, K, P, _p(s_ch), bits,
                                            pct_ppm, _p(s_tok), self._stream(stream)), "stwq_calibrate")
+
+    def gps_scales(self, Xcal, W, bits, pct_ppm, variant, s_ch, k_star=None, stream=None):
+        rows, K = Xcal.shape
+        N = W.shape[0]
+        self._check(self._L.gps_scales(self._h, _p(Xcal), rows, K, _p(W), N, bits, pct_ppm, variant, _p(s_ch),
+                                       _p(k_star), self._stream(stream)), "gps_scales")
 
     def gps_fold(self, W, s_ch, bits, Wq, s_w, stream=None):
         N, K = W.shape

@@ -221,6 +221,21 @@ int stwq_calibrate(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int
                                  static_cast<cudaStream_t>(stream));
 }
 
+int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const float* W, int N, int bits,
+               uint32_t pct_ppm, int variant, float* s_ch, int32_t* k_star, void* stream)
+{
+    if (!ctx || !Xcal || !W || !s_ch) return STWQ_ERR_NULL;
+    if (rows <= 0 || K <= 0 || N <= 0) return STWQ_ERR_DIM;
+    if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
+    if (variant != 0 && variant != 1) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    int rc = ensure_cal(ctx, 1);
+    if (rc == STWQ_OK) rc = ensure_dyn(ctx, stwq_gps_ws_bytes(K, N));
+    if (rc != STWQ_OK) return rc;
+    return stwq_launch_gps(ctx, ctx->ws_cal, ctx->ws_dyn, Xcal, rows, K, W, N, bits, pct_ppm, variant, s_ch, k_star,
+                           static_cast<cudaStream_t>(stream));
+}
+
 int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
              float* s_w, void* stream)
 {

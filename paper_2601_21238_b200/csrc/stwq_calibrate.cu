@@ -54,7 +54,7 @@ cal_hist_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
     CalWs w = cal_ws(base, P);
     const int shift = 24 - 8 * pass;
     for (int64_t r = blockIdx.x; r < rows; r += gridDim.x) {
-        const int p = pos_ids[r];
+        const int p = pos_ids ? pos_ids[r] : 0;               // no ids: one population (per-tensor range)
         if (p < 0 || p >= P) {
             if (threadIdx.x == 0 && pass == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
             continue;

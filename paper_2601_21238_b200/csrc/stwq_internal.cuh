@@ -73,6 +73,9 @@ int stwq_launch_calibrate_asym(stwq_ctx* ctx, void* ws, const float* Xcal, const
 int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);
+size_t stwq_gps_ws_bytes(int K, int N);
+int stwq_launch_gps(stwq_ctx* ctx, void* ws_cal, void* ws, const float* X, int64_t T, int K, const float* W, int N,
+                    int bits, uint32_t pct_ppm, int variant, float* s, int32_t* k_star_out, cudaStream_t st);
 int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids,
                           int64_t rows, int K, int P, const float* s_ch, int bits, uint32_t pct_ppm,
                           float* s_tok, cudaStream_t st);

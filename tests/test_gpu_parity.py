@@ -129,6 +129,37 @@ def test_gps_fold_bit_exact(gpu, bits, shape):
         np.testing.assert_array_equal(Wq.cpu().numpy(), Wq_r)
 
 
+# ----------------------------------------------------------------------------- gps_scales
+@pytest.mark.parametrize("variant", [0, 1])
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(1, 16, 1), (37, 48, 5), (300, 1040, 70), (256, 1024, 3072), (4100, 520, 33)])
+def test_gps_scales_match_the_oracle(gpu, shape, bits, variant):
+    """Algorithm 1 on the GPU against the oracle: k* and the clamp decisions are exact; the scales
+    agree to fp32 rounding (both sides sum in fp64, in different orders: relative difference of the
+    sums below 1e-12, so the fp32 results differ by at most one unit in the last place)."""
+    T, K, N = shape
+    X = rng.standard_normal((T, K)).astype(np.float32) * rng.uniform(0.2, 3.0, K).astype(np.float32)
+    X[:, K // 3] *= 25.0                                    # an outlier channel: the one with the widest range
+    W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    if K > 4:
+        W[:, 1] = 0.0                                       # dead input channel: denominator 0 -> s = 1
+        X[:, 2] = 0.0                                       # silent channel: numerator 0 -> s = 1
+    s_ref, k_ref = oracle.gps(X, W, bits, PCT, variant)
+    s = gpu.torch.zeros(K, device=gpu.dev)
+    kstar = gpu.torch.full((1,), -1, dtype=gpu.torch.int32, device=gpu.dev)
+    for _ in range(2):
+        gpu.ctx.gps_scales(gpu.T(X), gpu.T(W), bits, PCT, variant, s, kstar)
+        assert gpu.ctx.stwq_device_status() == 0
+        assert int(kstar.item()) == int(k_ref)
+        got = s.cpu().numpy()
+        np.testing.assert_allclose(got, s_ref, rtol=2.5e-7, atol=0)
+        if K > 4 and T > 1:
+            assert got[1] == 1.0 and got[2] == 1.0
+    first = s.clone()
+    gpu.ctx.gps_scales(gpu.T(X), gpu.T(W), bits, PCT, variant, s, None)
+    assert gpu.torch.equal(first, s)                        # fixed summation order: repeatable bit for bit
+
+
 # ----------------------------------------------------------------------------- stwq_calibrate
 @pytest.mark.parametrize("pct", [1000000, PCT, 990000, 500000, 1])
 def test_calibrate_bit_exact(gpu, pct):

@@ -38,6 +38,7 @@ def test_host_side_argument_errors(lib):
     assert lib.qlinear(None, None, None, 1, 16, 16, None, None, None, 1, None, None, 8, 0, 0, None, None) == -1
     assert lib.stwq_quantize(None, None, None, 1, 16, None, None, 1, 8, None, None) == -1
     assert lib.gps_fold(None, None, 1, 1, None, 8, None, None, None) == -1
+    assert lib.gps_scales(None, None, 1, 1, None, 1, 8, 999900, 0, None, None, None) == -1
     assert lib.stwq_calibrate(None, None, None, 1, 1, 1, None, 8, 1000000, None, None) == -1
     assert lib.stwq_strerror(0) == b"ok"
     assert b"NULL" in lib.stwq_strerror(-1)
