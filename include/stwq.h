@@ -119,7 +119,9 @@ int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const floa
  *     W'[n,k] = W[n,k] * s_ch[k]                  (s_ch == NULL: W' = W)
  *     a_n = max_k |W'[n,k]|,   s_w[n] = 2 a_n / D  (1 if a_n == 0)
  *     Wq[n,k] = clamp(round(W'[n,k] / s_w[n]), qmin, qmax)      (IEEE division, ties to even)
- * W [N,K] fp32 in, Wq [N,K] int8 out, s_w [N] fp32 out.
+ * W [N,K] fp32 in, Wq [N,K] int8 out, s_w [N] fp32 out. bits in {8, 6, 4}: 4-bit weights (the W4A8
+ * setting of Table 11) are codes in [-8, 7] in the same int8 containers, so every GEMM call takes them
+ * unchanged together with 8-bit activations.
  */
 int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
              float* s_w, void* stream);

@@ -11,6 +11,8 @@ namespace {
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int check_bits(int bits) { return (bits == 8 || bits == 6) ? STWQ_OK : STWQ_ERR_BITS; }
+// weights may also be 4-bit (W4A8, Table 11): the codes still travel in int8 containers
+int check_wbits(int bits) { return (bits == 8 || bits == 6 || bits == 4) ? STWQ_OK : STWQ_ERR_BITS; }
 
 int ensure_xq(stwq_ctx* ctx, size_t bytes)
 {
@@ -241,7 +243,7 @@ int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int
 {
     if (!ctx || !W || !Wq || !s_w) return STWQ_ERR_NULL;
     if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
-    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if (check_wbits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
     return stwq_launch_fold(ctx, W, N, K, s_ch, bits, Wq, s_w, static_cast<cudaStream_t>(stream));
 }
@@ -370,7 +372,7 @@ int gps_fold_asym(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch
 {
     if (!ctx || !W || !Wq || !s_w || !z_w || !colsum) return STWQ_ERR_NULL;
     if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
-    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if (check_wbits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
     return stwq_launch_fold_asym(ctx, W, N, K, s_ch, bits, Wq, s_w, z_w, colsum, static_cast<cudaStream_t>(stream));
 }

@@ -113,7 +113,7 @@ def test_host_argument_validation(gpu):
 
 
 # ----------------------------------------------------------------------------- gps_fold
-@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("bits", [8, 6, 4])
 @pytest.mark.parametrize("shape", [(1, 16), (70, 208), (256, 1024), (33, 7680)])
 def test_gps_fold_bit_exact(gpu, bits, shape):
     N, K = shape
@@ -278,6 +278,27 @@ def test_qlinear_small_ragged(gpu, bits, act, out):
     par2 = dict(par, bias=None)
     ref2 = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], None, bits, act)
     assert_close(_run_qlinear(gpu, L, par2, X, pos, out), ref2, RTOL[out], "no bias")
+
+
+@pytest.mark.parametrize("act", [0, 1])
+def test_qlinear_w4a8(gpu, act):
+    """4-bit weights with 8-bit activations (Table 11's W4A8): the weight codes come from gps_fold
+    with bits = 4 on the GPU, everything else is the 8-bit path."""
+    L = wl.scaled(wl.config_layers(1)[0], K=528, N=584, P=37, batch=9, bits=8, act=act)
+    par = prepare(L, samples=8, gps_n=64)
+    Wq4_ref, sw4_ref = oracle.gps_fold(par["W"], par["s_ch"], 4)
+    assert Wq4_ref.min() >= -8 and Wq4_ref.max() <= 7
+    Wq4 = gpu.torch.empty((L.N, L.K), dtype=gpu.torch.int8, device=gpu.dev)
+    sw4 = gpu.torch.empty(L.N, device=gpu.dev)
+    gpu.ctx.gps_fold(gpu.T(par["W"]), gpu.T(par["s_ch"]), 4, Wq4, sw4)
+    np.testing.assert_array_equal(Wq4.cpu().numpy(), Wq4_ref)
+    np.testing.assert_array_equal(sw4.cpu().numpy(), sw4_ref)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, Wq4_ref, sw4_ref, par["s_tok"], par["s_ch"], par["bias"], 8, act)
+    par4 = dict(par, Wq=Wq4_ref, s_w=sw4_ref)
+    np.testing.assert_array_equal(_run_qlinear(gpu, L, par4, X, pos, "int32"), ref["acc"])
+    for out in ("fp32", "bf16"):
+        assert_close(_run_qlinear(gpu, L, par4, X, pos, out), ref, RTOL[out], f"W4A8 act{act} {out}")
 
 
 @pytest.mark.parametrize("out", ["fp32", "bf16"])

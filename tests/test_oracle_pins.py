@@ -83,7 +83,7 @@ def test_ties_round_to_even():
 
 
 # ----------------------------------------------------------------------------- Eq. 2 + weights
-@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("bits", [8, 6, 4])
 def test_gps_fold_properties(bits):
     N, K = 37, 48
     W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
