@@ -316,20 +316,47 @@ def gpu_arm(args):
     h2d = sum(h.numel() * h.element_size() for h in hX)
     d2h = sum(h.numel() * h.element_size() for h in hY)
 
+    # Three streams, as a user streaming batches through the layer would do it: copies in, the
+    # calls, copies out. A layer's X buffer is refilled only after the call that read it, and its
+    # Y buffer rewritten only after the copy that read it (events), so steps overlap but every
+    # byte of every step is still copied in and out inside the timed region.
+    main = torch.cuda.current_stream()
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in S]       # X_i is on the device
+    ev_used = [torch.cuda.Event() for _ in S]     # the call has consumed X_i and written Y_i
+    ev_out = [torch.cuda.Event() for _ in S]      # Y_i is on the host
+    for e in ev_used + ev_out:
+        e.record(main)
+
     def e2e_step():
-        for s, hx, hy in zip(S, hX, hY):
+        for i, (s, hx, hy) in enumerate(zip(S, hX, hY)):
             L = s["L"]
-            s["X"].copy_(hx, non_blocking=True)
+            s_in.wait_event(ev_used[i])
+            with torch.cuda.stream(s_in):
+                s["X"].copy_(hx, non_blocking=True)
+                ev_in[i].record(s_in)
+            main.wait_event(ev_in[i])
+            main.wait_event(ev_out[i])
             ctx.qlinear(s["X"], s["pos"], s["Wq"], s["s_w"], s["s_tok"], s["s_ch"], s["bias"], L.bits, L.act,
                         s["out_code"], s["Y"])
-            hy.copy_(s["Y"], non_blocking=True)
+            ev_used[i].record(main)
+            s_out.wait_event(ev_used[i])
+            with torch.cuda.stream(s_out):
+                hy.copy_(s["Y"], non_blocking=True)
+                ev_out[i].record(s_out)
+
+    def e2e_drain():
+        main.wait_stream(s_in)
+        main.wait_stream(s_out)
 
     for _ in range(min(args.warmup, 3)):
         e2e_step()
+    e2e_drain()
     barrier()
     e0.record()
     for _ in range(args.steps):
         e2e_step()
+    e2e_drain()
     e1.record()
     barrier()
     e2e_ms = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
