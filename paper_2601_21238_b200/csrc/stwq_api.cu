@@ -412,8 +412,9 @@ int qlinear_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t 
     rc = stwq_launch_quantize_asym(ctx, X, pos_ids, M, K, s_ch, s_tok, z_tok, P, bits, ctx->ws_xq, rowcorr, st);
     if (rc != STWQ_OK) return rc;
     const stwq_asym asym = {z_tok, z_w, colsum, rowcorr};
-    return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, false, nullptr,
-                              st, &asym);
+    // the GEMM is a programmatic dependent of the quantize kernel, as in qlinear
+    return stwq_launch_qgemm2(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
+                              ctx->debug != 5, nullptr, st, &asym);
 }
 
 int dtwq_quantize(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,

@@ -232,6 +232,8 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         }
     } else {
         // ------------------------------------------------------------------ epilogue
+        // the asymmetric epilogue reads the row corrections that the quantize kernel accumulates
+        if (ASYM) asm volatile("griddepcontrol.wait;" ::: "memory");
         const int ew = warp - 2;                          // 0..EPI-1
         const int q = warp & 3;                           // TMEM lane quarter
         const int sub = ew >> 2;                          // which of the EPI/4 warps of this quarter
@@ -372,22 +374,6 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         }
                 }
             }
-            if (ASYM) {
-                // zero-point correction, exact in int32: acc - z_w[n] rowcorr[m] - z_tok[pos] colsum[n]
-#pragma unroll
-                for (int l = 0; l < kLoads; ++l) {
-                    const int k = l / kLoadsPerChunk, h = l % kLoadsPerChunk;
-#pragma unroll
-                    for (int j = 0; j < 32; j += 4) {
-                        const int4 zw = *reinterpret_cast<const int4*>(my_zw + k * kChunkCols + h * 32 + j);
-                        const int4 cs = *reinterpret_cast<const int4*>(my_cs + k * kChunkCols + h * 32 + j);
-                        racc[l][j + 0] = (uint32_t)((int)racc[l][j + 0] - zw.x * Rm - zx * cs.x);
-                        racc[l][j + 1] = (uint32_t)((int)racc[l][j + 1] - zw.y * Rm - zx * cs.y);
-                        racc[l][j + 2] = (uint32_t)((int)racc[l][j + 2] - zw.z * Rm - zx * cs.z);
-                        racc[l][j + 3] = (uint32_t)((int)racc[l][j + 3] - zw.w * Rm - zx * cs.w);
-                    }
-                }
-            }
 #pragma unroll
             for (int k = 0; k < kMyChunks; ++k, ++nstore) {
                 const int c = sub + k * kSubs;
@@ -398,6 +384,23 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint32_t* r1 = racc[k * kLoadsPerChunk + kLoadsPerChunk - 1];
                 uint32_t w[32];                           // this row's 128 bytes of output
                 const uint64_t st2 = pack_f2(st, st);
+                if (ASYM) {
+                    // zero-point correction of this chunk, exact in int32:
+                    // acc - z_w[n] rowcorr[m] - z_tok[pos] colsum[n]
+#pragma unroll
+                    for (int h = 0; h < kLoadsPerChunk; ++h) {
+                        uint32_t* r = racc[k * kLoadsPerChunk + h];
+#pragma unroll
+                        for (int j = 0; j < 32; j += 4) {
+                            const int4 zw = *reinterpret_cast<const int4*>(my_zw + k * kChunkCols + h * 32 + j);
+                            const int4 cs = *reinterpret_cast<const int4*>(my_cs + k * kChunkCols + h * 32 + j);
+                            r[j + 0] = (uint32_t)((int)r[j + 0] - zw.x * Rm - zx * cs.x);
+                            r[j + 1] = (uint32_t)((int)r[j + 1] - zw.y * Rm - zx * cs.y);
+                            r[j + 2] = (uint32_t)((int)r[j + 2] - zw.z * Rm - zx * cs.z);
+                            r[j + 3] = (uint32_t)((int)r[j + 3] - zw.w * Rm - zx * cs.w);
+                        }
+                    }
+                }
                 if (OUT == kOutCodes) {
                     // y = act(z) stays in fp32 registers and goes straight through the next layer's
                     // static quantizer: (y * rc_next[n]) * rt_next[pos], round to nearest even, clamp, pack

@@ -223,17 +223,29 @@ quantize_bf16_kernel(const uint16_t* __restrict__ X, const int32_t* __restrict__
 // Eq. 1 as printed with a static zero point per position: cs = clamp(round(u) + zs[pos], -h, h-1).
 // Besides the codes the kernel accumulates rowcorr[m] = sum_k cs[m,k] - K zs[pos[m]] (zeroed by the
 // launcher; one atomic per warp and row), which the GEMM epilogue multiplies by the weights'
-// zero points. A warp owns a 512-column span of a row, as in quantize_kernel.
+// zero points. A warp owns a 512-column span of a row and the loop is pipelined as in
+// quantize_kernel: the next row's loads, scale and zero point are in flight while this row is
+// converted.
 __global__ void __launch_bounds__(kThreads)
 quantize_asym_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
                      const float* __restrict__ s_ch, const float* __restrict__ s_tok, const int32_t* __restrict__ z_tok,
                      int P, int qmin, int qmax, int8_t* __restrict__ Xq, int32_t* __restrict__ rowcorr, int spans,
                      int64_t row_stride, uint32_t* __restrict__ status)
 {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the GEMM's prologue may start (see quantize_kernel)
     const int lane = threadIdx.x & 31;
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
     const int span = (int)(warp % spans);
+    int64_t m = warp / spans;
     const int col0 = span * kSpan + lane * 4;
+    if (m >= M) return;
+
+    float4 v[4], vn[4];
+    load_row(X + m * K, col0, K, v);
+    bool ok;
+    float rt = row_scale(pos_ids, s_tok, P, m, ok);
+    int zs = ok ? z_tok[pos_ids[m]] : 0;
+
     float rc[16];
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -242,22 +254,28 @@ quantize_asym_kernel(const float* __restrict__ X, const int32_t* __restrict__ po
         for (int e = 0; e < 4; ++e)
             rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
     }
-    for (int64_t m = warp / spans; m < M; m += row_stride) {
-        const int p = pos_ids[m];
-        const bool ok = (p >= 0) && (p < P);
-        const float rt = ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
-        const int zs = ok ? z_tok[p] : 0;
+
+    while (true) {
+        const int64_t mn = m + row_stride;
+        const bool more = mn < M;
+        bool okn = false;
+        float rtn = 0.0f;
+        int zsn = 0;
+        if (more) {
+            load_row(X + mn * K, col0, K, vn);
+            rtn = row_scale(pos_ids, s_tok, P, mn, okn);
+            zsn = okn ? z_tok[pos_ids[mn]] : 0;
+        }
         if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
         int sum = 0;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             const int c = col0 + j * 128;
             if (c < K) {
-                const float4 v = ld_stream(X + m * K + c);
-                const int q0 = stwq_code_asym(__fmul_rn(__fmul_rn(v.x, rc[j * 4 + 0]), rt), zs, qmin, qmax);
-                const int q1 = stwq_code_asym(__fmul_rn(__fmul_rn(v.y, rc[j * 4 + 1]), rt), zs, qmin, qmax);
-                const int q2 = stwq_code_asym(__fmul_rn(__fmul_rn(v.z, rc[j * 4 + 2]), rt), zs, qmin, qmax);
-                const int q3 = stwq_code_asym(__fmul_rn(__fmul_rn(v.w, rc[j * 4 + 3]), rt), zs, qmin, qmax);
+                const int q0 = stwq_code_asym(__fmul_rn(__fmul_rn(v[j].x, rc[j * 4 + 0]), rt), zs, qmin, qmax);
+                const int q1 = stwq_code_asym(__fmul_rn(__fmul_rn(v[j].y, rc[j * 4 + 1]), rt), zs, qmin, qmax);
+                const int q2 = stwq_code_asym(__fmul_rn(__fmul_rn(v[j].z, rc[j * 4 + 2]), rt), zs, qmin, qmax);
+                const int q3 = stwq_code_asym(__fmul_rn(__fmul_rn(v[j].w, rc[j * 4 + 3]), rt), zs, qmin, qmax);
                 sum += q0 + q1 + q2 + q3;
                 uint32_t hi, packed;
                 asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
@@ -268,6 +286,13 @@ quantize_asym_kernel(const float* __restrict__ X, const int32_t* __restrict__ po
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
         if (lane == 0) atomicAdd(rowcorr + m, sum - (span == 0 ? K * zs : 0));
+        if (!more) break;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = vn[j];
+        m = mn;
+        rt = rtn;
+        zs = zsn;
+        ok = okn;
     }
 }
 
@@ -482,6 +507,8 @@ int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_
     int64_t rows_in_flight = (int64_t)ctx->sm_count * 6 * warps_per_block / spans;
     if (rows_in_flight < 1) rows_in_flight = 1;
     if (rows_in_flight > M) rows_in_flight = M;
+    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
+    rows_in_flight = (M + passes - 1) / passes;             // every warp sees the same number of rows
     while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
     const unsigned blocks = (unsigned)(rows_in_flight * spans / warps_per_block);
     cudaError_t e = cudaMemsetAsync(rowcorr, 0, (size_t)M * sizeof(int32_t), st);
