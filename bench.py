@@ -591,6 +591,43 @@ def other_configs(ctx, pk, torch, dev, peaks):
                      "asym_qlinear_us": round(res["asym"] * 1e3, 2), "asym_tops": round(L.ops / res["asym"] / 1e9, 1)})
         del X, Wq, Y
     out["asymmetric_config2"] = rows
+    # activations handed over in bf16 (2 bytes read per element instead of 4): qlinear_bf16 beside qlinear
+    rows = []
+    for L in wl.config_layers(2):
+        ncopy = max(2, int(2 * 126e6 // (5.0 * L.M * L.K)) + 1)
+        Xs = [torch.randn(L.M, L.K, device=dev) for _ in range(ncopy)]
+        Xb = [x.to(torch.bfloat16) for x in Xs]
+        Wq = torch.randint(-128, 128, (L.N, L.K), dtype=torch.int8, device=dev)
+        pos = torch.from_numpy(wl.positions(L)).to(dev)
+        s_w = torch.rand(L.N, device=dev) * 1e-3 + 1e-4
+        s_tok = torch.rand(L.P, device=dev) * 0.05 + 0.01
+        s_ch = (torch.rand(L.K, device=dev) + 0.5) if L.use_gps else None
+        b = torch.randn(L.N, device=dev) * 0.02
+        Y = torch.empty((L.M, L.N), dtype=torch.bfloat16, device=dev)
+        res = {}
+        for name, xs, fn in (("fp32", Xs, ctx.qlinear), ("bf16", Xb, ctx.qlinear_bf16)):
+            call = lambda x: fn(x, pos, Wq, s_w, s_tok, s_ch, b, 8, L.act, pk.OUT_BF16, Y)
+            for x in xs:
+                call(x)
+            torch.cuda.synchronize()
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=side):
+                    for x in xs:
+                        call(x)
+                g.replay()
+                a, e = ev(), ev()
+                a.record()
+                for _ in range(5):
+                    g.replay()
+                e.record()
+                torch.cuda.synchronize()
+            res[name] = a.elapsed_time(e) / (5 * len(xs))
+        rows.append({"layer": L.name, "K": L.K, "N": L.N, "fp32_in_qlinear_us": round(res["fp32"] * 1e3, 2),
+                     "bf16_in_qlinear_us": round(res["bf16"] * 1e3, 2), "bf16_in_tops": round(L.ops / res["bf16"] / 1e9, 1)})
+        del Xs, Xb, Wq, Y
+    out["bf16_input_config2"] = rows
     ctx.check_device_status()
     return out
 

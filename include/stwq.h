@@ -144,6 +144,16 @@ int stwq_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int
                        const float* s_ch, const float* s_tok, int P, int bits, int8_t* Xq, void* stream);
 
 /*
+ * qlinear for activations held in bf16 (what a bf16 model hands from layer to layer): the same
+ * quantizer on the widened values (Eq. 1, Section 4.2; see stwq_quantize_bf16), then the GEMM and
+ * epilogue of qlinear. X [M,K] bf16, 16-byte aligned; everything else as qlinear. Reads 2 bytes per
+ * activation instead of 4.
+ */
+int qlinear_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K, int N,
+                 const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+                 const float* bias, int bits, int act, int out_dtype, void* Y, void* stream);
+
+/*
  * The quantized linear layer: stwq_quantize into context workspace, then
  *     acc[m,n] = sum_k Xq[m,k] * Wq[n,k]                          (int32, exact)
  *     z = float(acc) * (s_tok[pos_ids[m]] * s_w[n]) + bias[n]     (fp32: one multiply for the

@@ -21,7 +21,7 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
-            "stwq_quantize_asym", "qlinear_asym", "gps_scales"]
+            "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16"]
 
 _lib = None
 
@@ -61,6 +61,7 @@ def load_library():
     L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.qlinear_bf16.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.qlinear_q.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, i32, i32, vp, vp]
     L.qlinear_static.argtypes = [vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.stwq_calibrate_asym.argtypes = [vp, vp, vp, i64, i32, i32, vp, i32, u32, vp, vp, vp]
@@ -180,6 +181,13 @@ class Context:
         self._check(self._L.qlinear(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
                                     s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
                                     self._stream(stream)), "qlinear")
+
+    def qlinear_bf16(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
+        M, K = X.shape
+        N = Wq.shape[0]
+        self._check(self._L.qlinear_bf16(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
+                                    s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
+                                    self._stream(stream)), "qlinear_bf16")
 
     def qlinear_q(self, Xq, pos_ids, Wq, s_w, s_tok, bias, act, out_dtype, Y, stream=None):
         M, K = Xq.shape

@@ -306,6 +306,25 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, pdl, st);
 }
 
+int qlinear_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M, int K, int N,
+                 const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* s_ch,
+                 const float* bias, int bits, int act, int out_dtype, void* Y, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (!pos_ids || !s_tok || !s_w) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(X, pos_ids, M, K, N, Wq, s_w, s_tok, P, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    if (rc != STWQ_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = stwq_launch_quantize_bf16(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
+    if (rc != STWQ_OK) return rc;
+    // the GEMM is a programmatic dependent of the quantize kernel, as in qlinear
+    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, ctx->debug != 5, st);
+}
+
 static int chain_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int N, const int8_t* Wq,
                       const float* s_w, const float* s_tok, int P, const float* bias, int act,
                       const float* s_ch_next, const float* s_tok_next, int bits_next, const int8_t* Xq_next)

@@ -594,6 +594,31 @@ def test_quantize_bf16_input_bit_exact(gpu, bits, shape):
         np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
 
 
+@pytest.mark.parametrize("act", [0, 1])
+@pytest.mark.parametrize("shape", [(333, 400, 328), (1500, 1024, 1024), (200, 2048, 512)])
+def test_qlinear_bf16_matches_the_oracle(gpu, shape, act):
+    """The whole layer on bf16 activations equals the oracle's layer on the widened values: exact
+    accumulators, outputs within the usual tolerance (the last shape takes the few-row kernel)."""
+    torch = gpu.torch
+    M, K, N = shape
+    L = wl.scaled(wl.config_layers(1)[0], K=K, N=N, P=37, batch=1, bits=8, act=act)
+    par = prepare(L, samples=4, gps_n=64)
+    Xb = torch.from_numpy((rng.standard_normal((M, K)) * 2).astype(np.float32)).to(gpu.dev).to(torch.bfloat16)
+    X = Xb.float().cpu().numpy()
+    pos = rng.integers(0, L.P, M).astype(np.int32)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, act)
+    d = {k: gpu.T(par[k]) for k in ("Wq", "s_w", "s_tok", "s_ch", "bias")}
+    for out in ("int32", "fp32", "bf16"):
+        Y = _out_tensor(gpu, M, N, out)
+        gpu.ctx.qlinear_bf16(Xb, gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["s_ch"], d["bias"], 8,
+                             0 if out == "int32" else act, _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+        if out == "int32":
+            np.testing.assert_array_equal(Y.cpu().numpy(), ref["acc"])
+        else:
+            assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"qlinear_bf16 {out}")
+
+
 # ----------------------------------------------------------------------------- asymmetric quantizer (Eq. 1 as printed)
 @pytest.mark.parametrize("bits", [8, 6])
 def test_asym_offline_calls_bit_exact(gpu, bits):
