@@ -286,8 +286,17 @@ int stwq_device_status(stwq_ctx* ctx, void* stream);
  * 3 = always the single-CTA tiled GEMM (the fallback used when N or the s_w / bias pointers
  * do not meet the 16-byte rules of the CTA-pair kernel).
  * STWQ_OPT_WAIT_LIMIT_MS: limit of every device-side wait in milliseconds (default 2000).
+ * The remaining options choose between kernel variants that compute the same results (the parity
+ * tests use them to reach every variant; 0 = the library's own choice):
+ * STWQ_OPT_TILE_N: 128 or 256 = tile width of the CTA-pair GEMM.
+ * STWQ_OPT_VARIANT: 1 / 2 = CTA-pair GEMM epilogue through staged TMA stores / straight from
+ *   registers; 5 = ordinary launches instead of programmatic dependent ones; 7 / 8 = the
+ *   register-streaming / the TMA-ring quantize kernel.
+ * STWQ_OPT_KSPLIT: -1 = never cut tiles along K, n > 0 = cut the tiles of the last wave of the
+ *   CTA-pair GEMM (every work item of the few-row kernel) into n ranges of K.
  */
-enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2 };
+enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2, STWQ_OPT_TILE_N = 100, STWQ_OPT_VARIANT = 101,
+       STWQ_OPT_KSPLIT = 102 };
 int stwq_set_option(stwq_ctx* ctx, int option, int value);
 
 /* Number of kernels this context has launched since creation (for launch accounting). */

@@ -16,6 +16,7 @@ _LIB_PATH = os.path.join(_HERE, "libstwq.so")
 ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH = 0, 1, 2
 OUT_F32, OUT_BF16, OUT_INT32 = 0, 1, 2
 OPT_GEMM_PATH, OPT_WAIT_LIMIT_MS = 1, 2
+OPT_TILE_N, OPT_VARIANT, OPT_KSPLIT = 100, 101, 102
 STATIC_MAX_CODES = 4 * 1024 * 1024
 
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",

@@ -204,9 +204,9 @@ int stwq_set_option(stwq_ctx* ctx, int option, int value)
         ctx->wait_limit_ms = value;
         return STWQ_OK;
     }
-    if (option == 100) { ctx->force_bn = value; return STWQ_OK; }   // undocumented tuning knobs
-    if (option == 101) { ctx->debug = value; return STWQ_OK; }
-    if (option == 102) { ctx->force_ksplit = value; return STWQ_OK; }
+    if (option == STWQ_OPT_TILE_N) { ctx->force_bn = value; return STWQ_OK; }
+    if (option == STWQ_OPT_VARIANT) { ctx->debug = value; return STWQ_OK; }
+    if (option == STWQ_OPT_KSPLIT) { ctx->force_ksplit = value; return STWQ_OK; }
     return STWQ_ERR_DIM;
 }
 

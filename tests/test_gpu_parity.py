@@ -64,12 +64,12 @@ def test_quantize_codes_bit_exact(gpu, bits, shape):
         ref = oracle.quantize(X, pos, sc, s_tok, bits)
         for variant in (7, 8):              # the register-streaming kernel, the TMA-ring kernel
             Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
-            gpu.ctx.stwq_set_option(101, variant)
+            gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
             try:
                 gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), gpu.T(sc), gpu.T(s_tok), bits, Xq)
                 assert gpu.ctx.stwq_device_status() == 0
             finally:
-                gpu.ctx.stwq_set_option(101, 0)
+                gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, 0)
             np.testing.assert_array_equal(Xq.cpu().numpy(), ref)
 
 
@@ -81,11 +81,11 @@ def test_quantize_reports_bad_position_and_zeroes_the_row(gpu):
     s_tok = rng.uniform(0.01, 0.1, P).astype(np.float32)
     for variant in (7, 8):
         Xq = gpu.torch.full((M, K), 99, dtype=gpu.torch.int8, device=gpu.dev)
-        gpu.ctx.stwq_set_option(101, variant)
+        gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
         try:
             gpu.ctx.stwq_quantize(gpu.T(X), gpu.T(pos), None, gpu.T(s_tok), 8, Xq)
         finally:
-            gpu.ctx.stwq_set_option(101, 0)
+            gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, 0)
         assert gpu.ctx.stwq_device_status() == -8               # STWQ_ERR_POS_RANGE
         assert gpu.ctx.stwq_device_status() == 0                # reading clears it
         got = Xq.cpu().numpy()
@@ -410,14 +410,14 @@ def test_decode_split_k_is_exact_and_repeatable(gpu, shape, ksplit):
     X = wl.activations(wl.scaled(L, batch=256))[:M]
     pos = rng.integers(0, L.P, M).astype(np.int32)
     ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 2)
-    gpu.ctx.stwq_set_option(102, ksplit)
+    gpu.ctx.stwq_set_option(gpu.B.OPT_KSPLIT, ksplit)
     try:
         for _ in range(2):
             np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", act=2, path=2), ref["acc"])
             assert_close(_run_qlinear(gpu, L, par, X, pos, "fp32", act=2, path=2), ref, RTOL["fp32"], "decode fp32")
             assert_close(_run_qlinear(gpu, L, par, X, pos, "bf16", act=2, path=2), ref, RTOL["bf16"], "decode bf16")
     finally:
-        gpu.ctx.stwq_set_option(102, 0)
+        gpu.ctx.stwq_set_option(gpu.B.OPT_KSPLIT, 0)
 
 
 @pytest.mark.parametrize("ksplit", [-1, 0, 3, 7])
@@ -438,7 +438,7 @@ def test_tiled_gemm_split_tail_is_exact_and_repeatable(gpu, shape, ksplit):
     ref = {"Y": Yref, "mag": mag}
     d = [gpu.T(a) for a in (Xq, pos, Wq, s_w, s_tok, bias)]
     gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 1)
-    gpu.ctx.stwq_set_option(102, ksplit)
+    gpu.ctx.stwq_set_option(gpu.B.OPT_KSPLIT, ksplit)
     try:
         for _ in range(2):
             Yi = _out_tensor(gpu, M, N, "int32")
@@ -450,7 +450,7 @@ def test_tiled_gemm_split_tail_is_exact_and_repeatable(gpu, shape, ksplit):
                 assert gpu.ctx.stwq_device_status() == 0
                 assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"split tail {out}")
     finally:
-        gpu.ctx.stwq_set_option(102, 0)
+        gpu.ctx.stwq_set_option(gpu.B.OPT_KSPLIT, 0)
         gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
 
 
