@@ -25,7 +25,10 @@
  *    on the host before anything is enqueued. Errors only the device can see (a pos_id
  *    outside [0,P), a non-finite calibration value, a device-side wait that ran out) are
  *    recorded in the context and read with stwq_device_status().
- *  - A context may be used from one host thread at a time.
+ *  - A context may be used from one host thread at a time, and its calls share its workspace
+ *    (the int8 copy of X, per-row scratch, calibration and split-K buffers): calls on one
+ *    context that could overlap on the device (different streams without an ordering between
+ *    them) race. Use one context per stream that runs concurrently.
  *  - Alignment: X, Xq, Wq, Y 16-byte aligned; K a multiple of 16.
  */
 #ifndef STWQ_H
@@ -47,7 +50,7 @@ enum {
     STWQ_ERR_NULL = -1,           /* a required pointer is NULL                              */
     STWQ_ERR_DIM = -2,            /* a size is zero, negative or beyond what is supported    */
     STWQ_ERR_ALIGN = -3,          /* pointer or K alignment rule violated                    */
-    STWQ_ERR_BITS = -4,           /* bits is not 6 or 8, or act / out_dtype / pct invalid    */
+    STWQ_ERR_BITS = -4,           /* bits not 6 or 8 (4 too for weights), or act / out_dtype / pct invalid */
     STWQ_ERR_ARCH = -5,           /* the device is not compute capability 10.x               */
     STWQ_ERR_CUDA = -6,           /* a CUDA call failed; see stwq_last_cuda_error()          */
     STWQ_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired; output is invalid   */
