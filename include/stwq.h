@@ -295,8 +295,9 @@ int stwq_device_status(stwq_ctx* ctx, void* stream);
  * STWQ_OPT_VARIANT: 1 / 2 = CTA-pair GEMM epilogue through staged TMA stores / straight from
  *   registers; 5 = ordinary launches instead of programmatic dependent ones; 7 / 8 = the
  *   register-streaming / the TMA-ring quantize kernel.
- * STWQ_OPT_KSPLIT: -1 = never cut tiles along K, n > 0 = cut the tiles of the last wave of the
- *   CTA-pair GEMM (every work item of the few-row kernel) into n ranges of K.
+ * STWQ_OPT_KSPLIT: n > 0 = cut the tiles of the last wave of the CTA-pair GEMM (every work item of
+ *   the few-row kernel) into n ranges of K; -1 = the few-row kernel never cuts. The CTA-pair GEMM
+ *   cuts only on request.
  */
 enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2, STWQ_OPT_TILE_N = 100, STWQ_OPT_VARIANT = 101,
        STWQ_OPT_KSPLIT = 102 };

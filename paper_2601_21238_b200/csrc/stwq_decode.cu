@@ -447,6 +447,7 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
         if (ksplit < 1) ksplit = 1;
     }
     if (ctx->force_ksplit > 0) ksplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
+    if (ctx->force_ksplit < 0) ksplit = 1;
     p.kb_per_split = (p.num_kb + ksplit - 1) / ksplit;
     p.ksplit = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;      // every range holds at least one k-block
     const int items = tiles_n * p.ksplit;

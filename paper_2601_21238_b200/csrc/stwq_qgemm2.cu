@@ -696,13 +696,12 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
 
     // The last wave of a static tile schedule is partly empty unless the tile count divides by
-    // the number of pairs. When at most half the pairs would have work in it, its tiles can be cut
-    // along K into nsplit units each, so that the wave costs 1 / nsplit of a tile time. The price
-    // is the exchange of partial sums through scratch memory: 256 KB written per unit and as much
-    // read back, all at the end of the kernel when nothing overlaps it (measured: about 4 us of
-    // latency plus 0.12 us per unit at ~5 TB/s of L2 traffic), against about 0.38 us per k-block
-    // saved. For the 170-700 tile problems of the VAR / MAR layers this does not pay; it does for
-    // problems of a few tiles with long K.
+    // the number of pairs. Its tiles can be cut along K into nsplit units each, whose int32
+    // partial sums meet in scratch memory (the last unit to arrive adds them up). Measured, this
+    // never pays here: each unit writes 256 KB and the last arriver reads them back one after the
+    // other at the very end of the kernel, which costs 1 us and more per range (M 4736, N 1024,
+    // K 4096, a two-tile tail: 25.6 us whole tiles, 26.9 / 33.0 / 48.4 us with 2 / 4 / 8 ranges),
+    // more than the k-blocks saved. So the cut is made only on request (STWQ_OPT_KSPLIT > 0).
     p.full_units = p.num_tiles;
     p.num_units = p.num_tiles;
     p.nsplit = 1;
@@ -711,16 +710,8 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.counters = nullptr;
     const int pairs = ctx->max_pairs > 0 ? ctx->max_pairs : ctx->sm_count / 2;
     const int tail = p.num_tiles % pairs;
-    if (bn == 256 && tail > 0 && 2 * tail <= pairs && ctx->force_ksplit >= 0) {
-        int nsplit = pairs / tail;
-        if (nsplit > p.num_kb / 4) nsplit = p.num_kb / 4;
-        if (nsplit > 8) nsplit = 8;
-        if (nsplit >= 2) {
-            const double saved_us = (1.0 - 1.0 / nsplit) * p.num_kb * 0.38;
-            const double cost_us = 4.0 + 0.12 * tail * nsplit;
-            if (saved_us < 1.5 * cost_us) nsplit = 1;
-        }
-        if (ctx->force_ksplit > 0) nsplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
+    if (bn == 256 && tail > 0 && 2 * tail <= pairs && ctx->force_ksplit > 0) {
+        int nsplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
         if (nsplit >= 2) {
             const int kbps = (p.num_kb + nsplit - 1) / nsplit;
             nsplit = (p.num_kb + kbps - 1) / kbps;             // every range holds at least one k-block
