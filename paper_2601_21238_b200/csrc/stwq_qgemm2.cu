@@ -747,7 +747,9 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     // Long main loops hide the epilogue anyway and gain from the deeper ring that the
     // register-direct epilogue leaves room for; short ones (and GELU) are bound by the epilogue,
     // which costs the fewest shared-memory cycles when it goes through staged TMA stores.
-    bool direct = K >= 1536 && act == STWQ_ACT_NONE && asym == nullptr;
+    // (crossover measured at M 10880, N 1024 and 4096: between K 1536 and 1920 for 2-byte outputs,
+    // between 1920 and 2560 for 4-byte ones)
+    bool direct = K >= (elem == 4 ? 2304 : 1792) && act == STWQ_ACT_NONE && asym == nullptr;
     if (ctx->debug == 1) direct = false;                  // tuning: force one or the other
     if (ctx->debug == 2 && asym == nullptr) direct = true;
     if (direct) return launch_bn<256, 6, 8, 1>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
