@@ -497,6 +497,22 @@ int launch_ring(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M
 
 }  // namespace
 
+// Rows handled concurrently by the register-streaming kernels: a warp owns one 512-column span of
+// a row and strides over the rows. Chosen so that (a) the grid fits the resident blocks (one
+// block beyond them would run alone after all the others: a second wave for a single block),
+// (b) every warp sees the same number of rows, (c) the warp count is a multiple of a block's.
+static int64_t rows_in_flight_for(int64_t max_blocks, int warps_per_block, int spans, int64_t M)
+{
+    int64_t rows = max_blocks * warps_per_block / spans;
+    if (rows < 1) rows = 1;
+    if (rows > M) rows = M;
+    for (int64_t passes = (M + rows - 1) / rows;; ++passes) {
+        int64_t r = (M + passes - 1) / passes;
+        while ((r * spans) % warps_per_block != 0) ++r;
+        if (r * spans / warps_per_block <= max_blocks || r <= 1 || passes >= M) return r;
+    }
+}
+
 int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, const float* s_ch,
                               const float* s_tok, const int32_t* z_tok, int P, int bits, int8_t* Xq, int32_t* rowcorr,
                               cudaStream_t st)
@@ -504,12 +520,14 @@ int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
-    int64_t rows_in_flight = (int64_t)ctx->sm_count * 6 * warps_per_block / spans;
-    if (rows_in_flight < 1) rows_in_flight = 1;
-    if (rows_in_flight > M) rows_in_flight = M;
-    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
-    rows_in_flight = (M + passes - 1) / passes;             // every warp sees the same number of rows
-    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    static int per_sm_asym = 0;                             // resident blocks per SM (the same on every B200)
+    if (per_sm_asym <= 0) {
+        int n = 0;
+        cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_asym_kernel, kThreads, 0);
+        if (eo != cudaSuccess) return stwq_cuda_fail(ctx, eo);
+        per_sm_asym = n > 0 ? n : 1;
+    }
+    const int64_t rows_in_flight = rows_in_flight_for((int64_t)ctx->sm_count * per_sm_asym, warps_per_block, spans, M);
     const unsigned blocks = (unsigned)(rows_in_flight * spans / warps_per_block);
     cudaError_t e = cudaMemsetAsync(rowcorr, 0, (size_t)M * sizeof(int32_t), st);
     if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
@@ -526,13 +544,14 @@ int stwq_launch_quantize_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_i
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
-    const int64_t max_warps = (int64_t)ctx->sm_count * 4 * warps_per_block;
-    int64_t rows_in_flight = max_warps / spans;
-    if (rows_in_flight < 1) rows_in_flight = 1;
-    if (rows_in_flight > M) rows_in_flight = M;
-    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
-    rows_in_flight = (M + passes - 1) / passes;
-    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    static int per_sm_bf16 = 0;                             // resident blocks per SM (the same on every B200)
+    if (per_sm_bf16 <= 0) {
+        int n = 0;
+        cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_bf16_kernel<true>, kThreads, 0);
+        if (eo != cudaSuccess) return stwq_cuda_fail(ctx, eo);
+        per_sm_bf16 = n > 0 ? n : 1;
+    }
+    const int64_t rows_in_flight = rows_in_flight_for((int64_t)ctx->sm_count * per_sm_bf16, warps_per_block, spans, M);
     const unsigned blocks = (unsigned)(rows_in_flight * spans / warps_per_block);
     const uint16_t* x = static_cast<const uint16_t*>(X);
     if (bits == 8)
@@ -551,13 +570,12 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
                          bool dependent, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    // the ring kernel's tables bound K and P; it only wins (by 25-30 %) on inputs of hundreds of MB,
-    // where the output no longer stays in L2 and more bytes in flight help
+    // The TMA-ring kernel is kept as a variant (STWQ_OPT_VARIANT = 8; its tables bound K and P): with
+    // the grid sized as below the register-streaming kernel is the faster one at every size
+    // measured (6.3-6.4 TB/s of algorithmic bytes on 0.7-1.3 GB inputs against 5.4-5.6).
     const bool ring_ok = K <= kRingMaxK && P <= kRingMaxP && ctx->encode_tiled != nullptr && M < ((int64_t)1 << 29) &&
                          (M * (int64_t)K) % 256 == 0;
-    bool ring = ring_ok && (int64_t)M * K >= ((int64_t)1 << 27);
-    if (ctx->debug == 7) ring = false;                    // tuning: force one or the other
-    if (ctx->debug == 8) ring = ring_ok;
+    const bool ring = ring_ok && ctx->debug == 8;
     if (ring) return launch_ring(ctx, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, dependent, st);
     const int spans = (K + kSpan - 1) / kSpan;
     const int warps_per_block = kThreads / 32;
@@ -570,13 +588,7 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
         ctx->quant_blocks_per_sm = n > 0 ? n : 1;
     }
     const int64_t max_warps = (int64_t)ctx->sm_count * ctx->quant_blocks_per_sm * warps_per_block;
-    int64_t rows_in_flight = max_warps / spans;
-    if (rows_in_flight < 1) rows_in_flight = 1;
-    if (rows_in_flight > M) rows_in_flight = M;
-    const int64_t passes = (M + rows_in_flight - 1) / rows_in_flight;
-    rows_in_flight = (M + passes - 1) / passes;
-    // total warps must be rows_in_flight * spans and a multiple of warps_per_block
-    while ((rows_in_flight * spans) % warps_per_block != 0) ++rows_in_flight;
+    const int64_t rows_in_flight = rows_in_flight_for(max_warps / warps_per_block, warps_per_block, spans, M);
     const int64_t blocks = rows_in_flight * spans / warps_per_block;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
