@@ -436,14 +436,17 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
     p.num_kb = (K + kBK - 1) / kBK;
     const int tiles_n = (N + kBN - 1) / kBN;
-    // One work item per CTA pair if N allows; otherwise split K so that about sm_count / 2 pairs
-    // have work, keeping at least four k-blocks per item.
+    // One work item per CTA pair if N allows; otherwise K may be split so that more pairs have
+    // work. The exchange of partial sums costs 2-3 us, so this pays only for long K: measured
+    // (M 256, weights from HBM, N 1024-4096) no split is best up to K 2048 (7.7-11.3 us against
+    // 10.3-13.0 us with two ranges), and from K 4096 on two to four ranges of at least eight
+    // k-blocks each (K 8192, N 1024: 27.2 us whole, 17.2 us in four ranges, 18.3 in eight).
     const int pairs = ctx->sm_count / 2;
     int ksplit = 1;
-    if (tiles_n * 4 < pairs * 3) {
+    if (tiles_n * 4 < pairs * 3 && p.num_kb >= 32) {
         ksplit = pairs / tiles_n;
-        if (ksplit > p.num_kb / 4) ksplit = p.num_kb / 4;
-        if (ksplit > 32) ksplit = 32;
+        if (ksplit > p.num_kb / 8) ksplit = p.num_kb / 8;
+        if (ksplit > 4) ksplit = 4;
         if (ksplit < 1) ksplit = 1;
     }
     if (ctx->force_ksplit > 0) ksplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
