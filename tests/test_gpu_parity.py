@@ -280,6 +280,42 @@ def test_qlinear_small_ragged(gpu, bits, act, out):
     assert_close(_run_qlinear(gpu, L, par2, X, pos, out), ref2, RTOL[out], "no bias")
 
 
+@pytest.mark.parametrize("seed", [11, 12, 13])
+def test_random_shapes_match_the_oracle(gpu, seed):
+    """Seeded random problem sizes (ragged in every dimension, N a multiple of 4 or of 16, with and
+    without channel scale and bias) through every GEMM route: exact accumulators, outputs in tolerance."""
+    r = np.random.default_rng(seed)
+    for _ in range(10):
+        M = int(r.choice([1, 7, 128, 129, 255, 257, 300, 511, int(r.integers(1, 700))]))
+        N = int(4 * r.integers(1, 150)) if r.random() < 0.6 else int(16 * r.integers(1, 40))
+        K = int(16 * r.integers(1, 64))
+        P = int(r.integers(1, 20))
+        act = int(r.integers(0, 3))
+        path = int(r.choice([0, 0, 1, 3]))
+        X = (r.standard_normal((M, K)) * 2).astype(np.float32)
+        Wq = r.integers(-128, 128, (N, K)).astype(np.int8)
+        pos = r.integers(0, P, M).astype(np.int32)
+        s_w = r.uniform(1e-4, 1e-3, N).astype(np.float32)
+        s_tok = r.uniform(0.01, 0.06, P).astype(np.float32)
+        s_ch = r.uniform(0.5, 1.5, K).astype(np.float32) if r.random() < 0.5 else None
+        bias = (0.5 * r.standard_normal(N)).astype(np.float32) if r.random() < 0.7 else None
+        ref = oracle.qlinear(X, pos, Wq, s_w, s_tok, s_ch, bias, 8, act)
+        what = f"seed {seed} M={M} N={N} K={K} act={act} path={path}"
+        gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, path)
+        try:
+            for out in ("int32", "fp32", "bf16"):
+                Y = _out_tensor(gpu, M, N, out)
+                gpu.ctx.qlinear(gpu.T(X), gpu.T(pos), gpu.T(Wq), gpu.T(s_w), gpu.T(s_tok), gpu.T(s_ch), gpu.T(bias), 8,
+                                0 if out == "int32" else act, _out_code(gpu, out), Y)
+                assert gpu.ctx.stwq_device_status() == 0, what
+                if out == "int32":
+                    np.testing.assert_array_equal(Y.cpu().numpy(), ref["acc"], err_msg=what)
+                else:
+                    assert_close(Y.float().cpu().numpy(), ref, RTOL[out], what + " " + out)
+        finally:
+            gpu.ctx.stwq_set_option(gpu.B.OPT_GEMM_PATH, 0)
+
+
 @pytest.mark.parametrize("act", [0, 1])
 def test_qlinear_w4a8(gpu, act):
     """4-bit weights with 8-bit activations (Table 11's W4A8): the weight codes come from gps_fold
