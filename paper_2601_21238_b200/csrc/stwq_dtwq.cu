@@ -6,9 +6,9 @@
 // be timed beside the static kernel: it has to finish a reduction over the row (warp shuffles,
 // then one exchange through shared memory) before it can emit the first code of that row.
 //
-// One block per row at a time (grid-stride), 256 threads; a thread keeps its 4 NV values of the
-// row in registers between the two phases, so X is read once; the reciprocal channel scales of
-// its columns stay in registers across rows. K <= 8192.
+// K > 1024: one block per row at a time (grid-stride), 256 threads; a thread keeps its 4 NV values of
+// the row in registers between the two phases, so X is read once; the reciprocal channel scales
+// of its columns stay in registers across rows. K <= 8192. K <= 1024: a warp per row (below).
 #include "stwq_internal.cuh"
 
 namespace {
@@ -92,11 +92,120 @@ dtwq_kernel(const float* __restrict__ X, int64_t M, int K, const float* __restri
     }
 }
 
+// K <= 1024: a warp per row (no block barrier: the row maximum is a warp-shuffle reduction), a lane
+// keeps up to eight float4 of the row, and the next row's loads are in flight while this row is
+// reduced and converted, as in the static kernel.
+template <int NV>
+__global__ void __launch_bounds__(kThreads)
+dtwq_warp_kernel(const float* __restrict__ X, int64_t M, int K, const float* __restrict__ s_ch, int bits,
+                 int8_t* __restrict__ Xq, float* __restrict__ s_row, int32_t* __restrict__ row_ids, int64_t row_stride)
+{
+    // the reciprocal channel scales are the same for every warp: the block computes them once
+    __shared__ __align__(16) float rc_sh[128 * NV];
+    for (int c = threadIdx.x; c < 128 * NV; c += kThreads)
+        rc_sh[c] = (s_ch != nullptr && c < K) ? __fdiv_rn(1.0f, s_ch[c]) : 1.0f;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    int64_t m = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
+    if (m >= M) return;
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    float4 x[NV], xn[NV];
+    auto load = [&](int64_t r, float4 (&d)[NV]) {
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int c = 4 * lane + 128 * j;
+            if (c < K) d[j] = ld_stream(X + r * K + c);
+        }
+    };
+    load(m, x);
+    float rc[NV][4];
+#pragma unroll
+    for (int j = 0; j < NV; ++j) {
+        const float4 r4 = *reinterpret_cast<const float4*>(rc_sh + 4 * lane + 128 * j);
+        rc[j][0] = r4.x; rc[j][1] = r4.y; rc[j][2] = r4.z; rc[j][3] = r4.w;
+    }
+    while (true) {
+        const int64_t mn = m + row_stride;
+        const bool more = mn < M;
+        if (more) load(mn, xn);
+        // the products x * rc are formed twice (for the maximum, then for the codes) rather than
+        // kept: two multiplies per element are cheaper than 32 more registers per thread
+        float a = 0.0f;
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int c = 4 * lane + 128 * j;
+            if (c < K) {
+                const float av0 = fabsf(__fmul_rn(x[j].x, rc[j][0])), av1 = fabsf(__fmul_rn(x[j].y, rc[j][1]));
+                const float av2 = fabsf(__fmul_rn(x[j].z, rc[j][2])), av3 = fabsf(__fmul_rn(x[j].w, rc[j][3]));
+                if (av0 > a) a = av0;                     // false for NaN: it does not take part
+                if (av1 > a) a = av1;
+                if (av2 > a) a = av2;
+                if (av3 > a) a = av3;
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
+        const float s = stwq_delta(a, bits);
+        const float rt = __fdiv_rn(1.0f, s);
+        if (lane == 0) {
+            s_row[m] = s;
+            if (row_ids != nullptr) row_ids[m] = (int32_t)m;
+        }
+        int8_t* qrow = Xq + m * K;
+#pragma unroll
+        for (int j = 0; j < NV; ++j) {
+            const int c = 4 * lane + 128 * j;
+            if (c < K) {
+                const int q0 = stwq_code(__fmul_rn(__fmul_rn(x[j].x, rc[j][0]), rt), qmin, qmax);
+                const int q1 = stwq_code(__fmul_rn(__fmul_rn(x[j].y, rc[j][1]), rt), qmin, qmax);
+                const int q2 = stwq_code(__fmul_rn(__fmul_rn(x[j].z, rc[j][2]), rt), qmin, qmax);
+                const int q3 = stwq_code(__fmul_rn(__fmul_rn(x[j].w, rc[j][3]), rt), qmin, qmax);
+                uint32_t hi, packed;
+                asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(q3), "r"(q2), "r"(0));
+                asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(packed) : "r"(q1), "r"(q0), "r"(hi));
+                *reinterpret_cast<uint32_t*>(qrow + c) = packed;
+            }
+        }
+        if (!more) break;
+#pragma unroll
+        for (int j = 0; j < NV; ++j) x[j] = xn[j];
+        m = mn;
+    }
+}
+
+template <int NV>
+int launch_warp_rows(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
+                     float* s_row, int32_t* row_ids, cudaStream_t st)
+{
+    static int per_sm = 0;                                  // resident blocks per SM (the same on every B200)
+    if (per_sm <= 0) {
+        int n = 0;
+        cudaError_t eo = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dtwq_warp_kernel<NV>, kThreads, 0);
+        if (eo != cudaSuccess) return stwq_cuda_fail(ctx, eo);
+        per_sm = n > 0 ? n : 1;
+    }
+    // as many warps as are resident, every warp the same number of rows, whole blocks
+    const int wpb = kThreads / 32;
+    const int64_t max_warps = (int64_t)ctx->sm_count * per_sm * wpb;
+    int64_t rows = max_warps < M ? max_warps : M;
+    for (int64_t passes = (M + rows - 1) / rows;; ++passes) {
+        rows = (M + passes - 1) / passes;
+        rows = (rows + wpb - 1) / wpb * wpb;
+        if (rows <= max_warps || passes >= M) break;
+    }
+    dtwq_warp_kernel<NV><<<(unsigned)(rows / wpb), kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids, rows);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
 }  // namespace
 
 int stwq_launch_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
                      float* s_row, int32_t* row_ids, cudaStream_t st)
 {
+    if (K <= 512) return launch_warp_rows<4>(ctx, X, M, K, s_ch, bits, Xq, s_row, row_ids, st);
+    if (K <= 1024) return launch_warp_rows<8>(ctx, X, M, K, s_ch, bits, Xq, s_row, row_ids, st);
     const int64_t max_blocks = (int64_t)ctx->sm_count * 8;
     const unsigned grid = (unsigned)(M < max_blocks ? M : max_blocks);
     const int nv = (K + 4 * kThreads - 1) / (4 * kThreads);
