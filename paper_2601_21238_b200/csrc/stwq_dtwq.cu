@@ -37,7 +37,7 @@ dtwq_kernel(const float* __restrict__ X, int64_t M, int K, const float* __restri
     for (int j = 0; j < NV; ++j) {
         const int c = 4 * threadIdx.x + j * 4 * kThreads;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) rc[j][e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
+        for (int e = 0; e < 4; ++e) rc[j][e] = (s_ch != nullptr && c + e < K) ? __frcp_rn(s_ch[c + e]) : 1.0f;
     }
     int it = 0;
     for (int64_t m = blockIdx.x; m < M; m += gridDim.x, ++it) {
@@ -69,7 +69,7 @@ dtwq_kernel(const float* __restrict__ X, int64_t M, int K, const float* __restri
 #pragma unroll
         for (int i = 1; i < kThreads / 32; ++i) t = fmaxf(t, wm[i]);
         const float s = stwq_delta(t, bits);
-        const float rt = __fdiv_rn(1.0f, s);
+        const float rt = __frcp_rn(s);
         if (threadIdx.x == 0) {
             s_row[m] = s;
             if (row_ids != nullptr) row_ids[m] = (int32_t)m;
@@ -103,7 +103,7 @@ dtwq_warp_kernel(const float* __restrict__ X, int64_t M, int K, const float* __r
     // the reciprocal channel scales are the same for every warp: the block computes them once
     __shared__ __align__(16) float rc_sh[128 * NV];
     for (int c = threadIdx.x; c < 128 * NV; c += kThreads)
-        rc_sh[c] = (s_ch != nullptr && c < K) ? __fdiv_rn(1.0f, s_ch[c]) : 1.0f;
+        rc_sh[c] = (s_ch != nullptr && c < K) ? __frcp_rn(s_ch[c]) : 1.0f;
     __syncthreads();
     const int lane = threadIdx.x & 31;
     int64_t m = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
@@ -146,7 +146,7 @@ dtwq_warp_kernel(const float* __restrict__ X, int64_t M, int K, const float* __r
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, o));
         const float s = stwq_delta(a, bits);
-        const float rt = __fdiv_rn(1.0f, s);
+        const float rt = __frcp_rn(s);
         if (lane == 0) {
             s_row[m] = s;
             if (row_ids != nullptr) row_ids[m] = (int32_t)m;

@@ -70,7 +70,7 @@ __device__ __forceinline__ float row_scale(const int32_t* pos_ids, const float* 
 {
     const int p = pos_ids[m];
     ok = (p >= 0) && (p < P);
-    return ok ? __fdiv_rn(1.0f, s_tok[p]) : 0.0f;
+    return ok ? __frcp_rn(s_tok[p]) : 0.0f;
 }
 
 // The loop is software-pipelined: the loads of the next row (and its position scale) are in
@@ -111,7 +111,7 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
         const int c = col0 + j * 128;
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
+            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __frcp_rn(s_ch[c + e]) : 1.0f;
     }
 
     while (true) {
@@ -186,7 +186,7 @@ quantize_bf16_kernel(const uint16_t* __restrict__ X, const int32_t* __restrict__
 #pragma unroll
         for (int e = 0; e < 8; ++e) {
             const int c = col0 + j * 256 + e;
-            rc[j * 8 + e] = (s_ch != nullptr && c < K) ? __fdiv_rn(1.0f, s_ch[c]) : 1.0f;
+            rc[j * 8 + e] = (s_ch != nullptr && c < K) ? __frcp_rn(s_ch[c]) : 1.0f;
         }
     while (true) {
         const int64_t mn = m + row_stride;
@@ -252,7 +252,7 @@ quantize_asym_kernel(const float* __restrict__ X, const int32_t* __restrict__ po
         const int c = col0 + j * 128;
 #pragma unroll
         for (int e = 0; e < 4; ++e)
-            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __fdiv_rn(1.0f, s_ch[c + e]) : 1.0f;
+            rc[j * 4 + e] = (s_ch != nullptr && c + e < K) ? __frcp_rn(s_ch[c + e]) : 1.0f;
     }
 
     while (true) {
@@ -373,8 +373,8 @@ quantize_ring_kernel(const __grid_constant__ CUtensorMap tmX, const int32_t* __r
         // ------------------------------------------------------------------ consumers
         const int cw = warp - 1;
         const int ct = threadIdx.x - 32;
-        for (int i = ct; i < K; i += 32 * kConsumerWarps) rc_s[i] = s_ch != nullptr ? __fdiv_rn(1.0f, s_ch[i]) : 1.0f;
-        for (int i = ct; i < P; i += 32 * kConsumerWarps) rt_s[i] = __fdiv_rn(1.0f, s_tok[i]);
+        for (int i = ct; i < K; i += 32 * kConsumerWarps) rc_s[i] = s_ch != nullptr ? __frcp_rn(s_ch[i]) : 1.0f;
+        for (int i = ct; i < P; i += 32 * kConsumerWarps) rt_s[i] = __frcp_rn(s_tok[i]);
         asm volatile("bar.sync 1, %0;" ::"n"(32 * kConsumerWarps) : "memory");
         // slot j of this thread: floats [256 cw + 128 j + 4 lane, +4) of every tile; K is a
         // multiple of 4, so a slot never straddles two rows
