@@ -22,6 +22,7 @@ struct stwq_ctx {
     int force_bn;              // tuning: 0 = choose, 128 / 256 = force the tile width
     int debug;                 // tuning: variant of the pair GEMM (epilogue store mode, prefetch distance)
     int quant_blocks_per_sm;   // resident blocks per SM of the quantize kernel (0 = not yet queried)
+    int quant_blocks_per_sm2;  // the same for its 256-column-span variant
     int quant_ring_configured; // the ring quantize kernel has its shared-memory attribute set
     int max_pairs;             // CTA pairs of the pair GEMM that can be resident at once (0 = not yet queried)
     uint64_t configured_mask;  // kernels whose shared-memory attribute is already set (single-CTA GEMM)

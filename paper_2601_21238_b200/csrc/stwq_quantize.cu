@@ -77,7 +77,9 @@ __device__ __forceinline__ float row_scale(const int32_t* pos_ids, const float* 
 // flight while the current row is converted, and the first row's loads are issued before the
 // reciprocal channel scales are computed, so that a warp that only sees a few rows (M of a few
 // thousand) does not serialise two memory round trips and sixteen divisions in front of them.
-template <bool B8>
+// VPL = float4 per lane and row: a warp's span is 128 VPL columns (512, or 256 where that leaves fewer
+// lanes without columns, e.g. K = 1280 = 5 x 256).
+template <bool B8, int VPL>
 __global__ void __launch_bounds__(kThreads)
 quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids, int64_t M, int K,
                 const float* __restrict__ s_ch, const float* __restrict__ s_tok, int P, int qmin,
@@ -96,18 +98,25 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
     const int64_t warp = ((int64_t)blockIdx.x * kThreads + threadIdx.x) >> 5;
     const int span = (int)(warp % spans);
     int64_t m = warp / spans;
-    const int col0 = span * kSpan + lane * 4;
+    const int col0 = span * (128 * VPL) + lane * 4;
     if (m >= M) return;
 
-    float4 v[4], vn[4];
-    load_row(X + m * K, col0, K, v);
+    float4 v[VPL], vn[VPL];
+    auto load = [&](int64_t r, float4 (&d)[VPL]) {
+#pragma unroll
+        for (int j = 0; j < VPL; ++j) {
+            const int c = col0 + j * 128;
+            if (c < K) d[j] = ld_stream(X + r * K + c);
+        }
+    };
+    load(m, v);
     bool ok;
     float rt = row_scale(pos_ids, s_tok, P, m, ok);
 
-    // reciprocal channel scales of this lane's 16 columns (1 where there is no scaling)
-    float rc[16];
+    // reciprocal channel scales of this lane's 4 VPL columns (1 where there is no scaling)
+    float rc[4 * VPL];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < VPL; ++j) {
         const int c = col0 + j * 128;
 #pragma unroll
         for (int e = 0; e < 4; ++e)
@@ -120,13 +129,13 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
         bool okn = false;
         float rtn = 0.0f;
         if (more) {
-            load_row(X + mn * K, col0, K, vn);
+            load(mn, vn);
             rtn = row_scale(pos_ids, s_tok, P, mn, okn);
         }
         if (!ok && lane == 0 && span == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
         int8_t* qrow = Xq + m * K;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+        for (int j = 0; j < VPL; ++j) {
             const int c = col0 + j * 128;
             if (c < K)
                 *reinterpret_cast<uint32_t*>(qrow + c) =
@@ -134,7 +143,7 @@ quantize_kernel(const float* __restrict__ X, const int32_t* __restrict__ pos_ids
         }
         if (!more) break;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) v[j] = vn[j];
+        for (int j = 0; j < VPL; ++j) v[j] = vn[j];
         m = mn;
         rt = rtn;
         ok = okn;
@@ -577,18 +586,24 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
                          (M * (int64_t)K) % 256 == 0;
     const bool ring = ring_ok && ctx->debug == 8;
     if (ring) return launch_ring(ctx, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, dependent, st);
-    const int spans = (K + kSpan - 1) / kSpan;
+    // 512-column spans, or 256-column ones where the last 512-column span would be at most half
+    // full (K = 768, 1280, ...): fewer lanes without columns
+    const int rem = K % kSpan;
+    const int vpl = (rem != 0 && rem <= kSpan / 2) ? 2 : 4;
+    const int span_cols = 128 * vpl;
+    const int spans = (K + span_cols - 1) / span_cols;
     const int warps_per_block = kThreads / 32;
     // As many warps as can be resident, then the row stride is shrunk so that every warp sees the
     // same number of rows (no ragged last pass).
-    if (ctx->quant_blocks_per_sm <= 0) {
+    int& per_sm = vpl == 4 ? ctx->quant_blocks_per_sm : ctx->quant_blocks_per_sm2;
+    if (per_sm <= 0) {
         int n = 0;
-        cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel<true>, kThreads, 0);
+        cudaError_t e = vpl == 4 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel<true, 4>, kThreads, 0)
+                                 : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, quantize_kernel<true, 2>, kThreads, 0);
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->quant_blocks_per_sm = n > 0 ? n : 1;
+        per_sm = n > 0 ? n : 1;
     }
-    const int64_t max_warps = (int64_t)ctx->sm_count * ctx->quant_blocks_per_sm * warps_per_block;
-    const int64_t rows_in_flight = rows_in_flight_for(max_warps / warps_per_block, warps_per_block, spans, M);
+    const int64_t rows_in_flight = rows_in_flight_for((int64_t)ctx->sm_count * per_sm, warps_per_block, spans, M);
     const int64_t blocks = rows_in_flight * spans / warps_per_block;
     cudaLaunchConfig_t cfg = {};
     cudaLaunchAttribute attr[1];
@@ -600,8 +615,10 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     cfg.stream = st;
     cfg.attrs = attr;
     cfg.numAttrs = dependent ? 1 : 0;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, bits == 8 ? quantize_kernel<true> : quantize_kernel<false>, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans,
-                                       rows_in_flight, ctx->d_status);
+    auto kern = vpl == 4 ? (bits == 8 ? quantize_kernel<true, 4> : quantize_kernel<false, 4>)
+                         : (bits == 8 ? quantize_kernel<true, 2> : quantize_kernel<false, 2>);
+    cudaError_t e = cudaLaunchKernelEx(&cfg, kern, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, spans, rows_in_flight,
+                                       ctx->d_status);
     ctx->launches += 1;
     if (e == cudaSuccess) e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
