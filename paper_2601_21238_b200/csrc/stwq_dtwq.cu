@@ -206,14 +206,26 @@ int stwq_launch_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, const floa
 {
     if (K <= 512) return launch_warp_rows<4>(ctx, X, M, K, s_ch, bits, Xq, s_row, row_ids, st);
     if (K <= 1024) return launch_warp_rows<8>(ctx, X, M, K, s_ch, bits, Xq, s_row, row_ids, st);
-    const int64_t max_blocks = (int64_t)ctx->sm_count * 8;
-    const unsigned grid = (unsigned)(M < max_blocks ? M : max_blocks);
     const int nv = (K + 4 * kThreads - 1) / (4 * kThreads);
-    if (nv <= 1) dtwq_kernel<1><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
-    else if (nv <= 2) dtwq_kernel<2><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
-    else if (nv <= 4) dtwq_kernel<4><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
-    else if (nv <= 8) dtwq_kernel<8><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
-    else return STWQ_ERR_DIM;
+    if (nv > 8) return STWQ_ERR_DIM;
+    // grid-stride over the rows with exactly the resident blocks (more would start as a second wave)
+    static int per_sm[4] = {0, 0, 0, 0};
+    const int v = nv <= 1 ? 0 : (nv <= 2 ? 1 : (nv <= 4 ? 2 : 3));
+    if (per_sm[v] <= 0) {
+        int n = 0;
+        cudaError_t eo = v == 0   ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dtwq_kernel<1>, kThreads, 0)
+                         : v == 1 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dtwq_kernel<2>, kThreads, 0)
+                         : v == 2 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dtwq_kernel<4>, kThreads, 0)
+                                  : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, dtwq_kernel<8>, kThreads, 0);
+        if (eo != cudaSuccess) return stwq_cuda_fail(ctx, eo);
+        per_sm[v] = n > 0 ? n : 1;
+    }
+    const int64_t max_blocks = (int64_t)ctx->sm_count * per_sm[v];
+    const unsigned grid = (unsigned)(M < max_blocks ? M : max_blocks);
+    if (v == 0) dtwq_kernel<1><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
+    else if (v == 1) dtwq_kernel<2><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
+    else if (v == 2) dtwq_kernel<4><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
+    else dtwq_kernel<8><<<grid, kThreads, 0, st>>>(X, M, K, s_ch, bits, Xq, s_row, row_ids);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
