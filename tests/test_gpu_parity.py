@@ -109,6 +109,23 @@ def test_host_argument_validation(gpu):
     assert L.stwq_quantize(h, None, p(pos), 4, 32, None, p(s_tok), 1, 8, p(Xq), None) == -1
     assert L.stwq_calibrate(h, p(X), p(pos), 4, 32, 1, None, 8, 0, p(s_tok), None) == -4       # pct
     assert L.stwq_set_option(h, 99, 0) == -2
+    # the later entry points: 4-bit codes are for weights only; GPS takes variant 0 or 1
+    W = gpu.torch.zeros((8, 32), device=gpu.dev)
+    Wq = gpu.torch.zeros((8, 32), dtype=gpu.torch.int8, device=gpu.dev)
+    s_w = gpu.torch.zeros(8, device=gpu.dev)
+    s_ch = gpu.torch.zeros(32, device=gpu.dev)
+    assert L.gps_fold(h, p(W), 8, 32, None, 4, p(Wq), p(s_w), None) == 0
+    assert L.gps_fold(h, p(W), 8, 32, None, 5, p(Wq), p(s_w), None) == -4
+    assert L.stwq_quantize(h, p(X), p(pos), 4, 32, None, p(s_tok), 1, 4, p(Xq), None) == -4
+    assert L.gps_scales(h, p(X), 4, 32, p(W), 8, 8, 999900, 2, p(s_ch), None, None) == -4     # variant
+    assert L.gps_scales(h, p(X), 4, 32, p(W), 8, 8, 0, 0, p(s_ch), None, None) == -4          # pct
+    assert L.gps_scales(h, p(X), 4, 32, p(W), 0, 8, 999900, 0, p(s_ch), None, None) == -2     # N
+    assert L.gps_scales(h, p(X), 4, 32, None, 8, 8, 999900, 0, p(s_ch), None, None) == -1
+    Xb = gpu.torch.zeros((4, 32), dtype=gpu.torch.bfloat16, device=gpu.dev)
+    Y = gpu.torch.zeros((4, 8), device=gpu.dev)
+    assert L.qlinear_bf16(h, p(Xb), p(pos), 4, 24, 8, p(Wq), p(s_w), p(s_tok), 1, None, None, 8, 0, 0, p(Y), None) == -3
+    assert L.qlinear_bf16(h, p(Xb), p(pos), 4, 32, 8, p(Wq), p(s_w), p(s_tok), 1, None, None, 8, 3, 0, p(Y), None) == -4
+    gpu.torch.cuda.synchronize()
     assert gpu.ctx.stwq_device_status() == 0
 
 
