@@ -586,7 +586,7 @@ def test_qlinear_dtwq_matches_the_oracle(gpu, M):
 # ----------------------------------------------------------------------------- chained layers
 @pytest.mark.parametrize("act", [0, 1, 2])
 @pytest.mark.parametrize("bits_next", [8, 6])
-@pytest.mark.parametrize("shape", [(333, 400, 336), (1500, 1024, 1024)])
+@pytest.mark.parametrize("shape", [(333, 400, 336), (1500, 1024, 1024), (77, 48, 32), (700, 272, 1040)])
 def test_chained_output_codes(gpu, shape, bits_next, act):
     """qlinear_chain: the epilogue applies the next layer's static quantizer. Without activation
     the codes are bit-exact. With GELU the kernel's short form moves y by at most 6e-4 |z|, so a
@@ -709,7 +709,7 @@ def test_asym_offline_calls_bit_exact(gpu, bits):
 
 @pytest.mark.parametrize("bits", [8, 6])
 @pytest.mark.parametrize("act", [0, 1])
-@pytest.mark.parametrize("shape", [(333, 400, 328), (1500, 1024, 768)])
+@pytest.mark.parametrize("shape", [(333, 400, 328), (1500, 1024, 768), (77, 48, 24), (700, 272, 1048)])
 def test_qlinear_asym_matches_the_oracle(gpu, shape, act, bits):
     """Asymmetric codes and row corrections bit-exact; the corrected int32 accumulators (which equal
     sum_k (cs - zx)(ws - zw)) bit-exact; outputs within the usual tolerance."""
