@@ -587,9 +587,11 @@ int stwq_launch_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, 
     const bool ring = ring_ok && ctx->debug == 8;
     if (ring) return launch_ring(ctx, X, pos_ids, M, K, s_ch, s_tok, P, qmin, qmax, Xq, dependent, st);
     // 512-column spans, or 256-column ones where the last 512-column span would be at most half
-    // full (K = 768, 1280, ...): fewer lanes without columns
+    // full (K = 768, 1280, ...: fewer lanes without columns) and on inputs of up to 2^24 elements,
+    // where more, lighter warps start and finish the short kernel sooner (45 MB: 11.1 -> 10.6 us;
+    // from 170 MB on the wider spans are 5 % faster)
     const int rem = K % kSpan;
-    const int vpl = (rem != 0 && rem <= kSpan / 2) ? 2 : 4;
+    const int vpl = ((rem != 0 && rem <= kSpan / 2) || M * (int64_t)K <= ((int64_t)1 << 24)) ? 2 : 4;
     const int span_cols = 128 * vpl;
     const int spans = (K + span_cols - 1) / span_cols;
     const int warps_per_block = kThreads / 32;
