@@ -114,9 +114,13 @@ int run_gemm(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M,
              int out_dtype, void* Y, bool after_quantize, cudaStream_t st)
 {
     const bool can_decode = M <= 256;
-    bool decode = can_decode;
+    // the few-row kernel gives each CTA pair one 128-column slice; with more slices than pairs it
+    // would run in two rounds and re-read Xq once per slice, and the tiled GEMM with its
+    // 256-column tiles is the faster one (M 256, N 16384, K 4096: 22 against 34 us)
+    bool decode = can_decode && (N + 127) / 128 <= ctx->sm_count / 2;
     if (ctx->gemm_path == 1 || ctx->gemm_path == 3) decode = false;
     if (ctx->gemm_path == 2 && !can_decode) return STWQ_ERR_DIM;
+    if (ctx->gemm_path == 2) decode = true;
     if (decode)
         return stwq_launch_decode(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y,
                                   after_quantize, st);
