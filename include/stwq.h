@@ -56,11 +56,23 @@ enum {
     STWQ_ERR_DEVICE_TIMEOUT = -7, /* a bounded device-side wait expired; output is invalid   */
     STWQ_ERR_POS_RANGE = -8,      /* a pos_id was outside [0,P); that row was written as 0   */
     STWQ_ERR_NONFINITE = -9,      /* calibration saw NaN or Inf                              */
-    STWQ_ERR_NOMEM = -10          /* workspace allocation failed                             */
+    STWQ_ERR_NOMEM = -10,         /* workspace allocation failed                             */
+    STWQ_ERR_CAPTURE = -11        /* the call would have to (re)allocate workspace while its stream is being
+                                     captured into a CUDA graph; reserve the workspace before capturing */
 };
 
-/* activation applied by the epilogue */
-enum { STWQ_ACT_NONE = 0, STWQ_ACT_GELU_ERF = 1, STWQ_ACT_GELU_TANH = 2 };
+/*
+ * Activation applied by the epilogue.
+ *   STWQ_ACT_GELU_ERF   y = z Phi(z), with Phi(-|z|) = erfc(|z| / sqrt2) / 2 as one exp2 of a fitted
+ *                       polynomial (absolute error on Phi below 1.5e-7), for every output type.
+ *   STWQ_ACT_GELU_TANH  y = z/2 (1 + tanh(sqrt(2/pi)(z + 0.044715 z^3))), evaluated as z sigmoid(2u) in fp32.
+ *   STWQ_ACT_GELU_FAST  the tanh form with the hardware's approximate tanh (relative error about 2^-11 on
+ *                       tanh, i.e. up to 6e-4 |z| on y): six instructions per element instead of about
+ *                       twenty. Meant for bf16 output (rounding unit 2^-9), where it stays inside the 1e-2
+ *                       tolerance of either GELU form; chained codes computed with it can differ by one
+ *                       from those of the exact activation.
+ */
+enum { STWQ_ACT_NONE = 0, STWQ_ACT_GELU_ERF = 1, STWQ_ACT_GELU_TANH = 2, STWQ_ACT_GELU_FAST = 3 };
 /* element type of Y. INT32 returns the raw accumulators (no scale, bias or activation). */
 enum { STWQ_OUT_F32 = 0, STWQ_OUT_BF16 = 1, STWQ_OUT_INT32 = 2 };
 
@@ -74,11 +86,23 @@ int stwq_create(stwq_ctx** out, int device);
 void stwq_destroy(stwq_ctx* ctx);
 
 /*
- * Pre-size the workspace so that later calls allocate nothing: room for an [M,K] int8
- * activation copy and for calibration over P positions. Synchronous (may allocate).
- * Without it the first call that needs more workspace allocates (and synchronises) itself.
+ * Workspace. A context keeps four buffers: the int8 copy of X, per-row scratch (row scales of
+ * qlinear_dtwq, row corrections of qlinear_asym, column statistics of gps_scales), calibration
+ * histograms, and int32 partial sums for the calls that split K. Each is allocated on first use and
+ * re-allocated (cudaFree + cudaMalloc, which synchronise the device) when a call needs more.
+ *  - stwq_reserve sizes the first and third for an [M,K] activation and P positions;
+ *    stwq_reserve_layer sizes all four for every call this header declares on an [M,K] x [N,K] layer
+ *    with P positions. After either, calls within those sizes allocate nothing.
+ *  - A call that would have to grow a buffer while its stream is being captured into a CUDA graph
+ *    returns STWQ_ERR_CAPTURE and enqueues nothing (an allocation would invalidate the capture).
+ *  - Growth moves the buffer: a graph captured earlier still holds the old, freed address and must
+ *    not be replayed. stwq_workspace_generation() changes whenever any buffer was (re)allocated, so
+ *    a caller that keeps graphs can compare the value it saw at capture time before each replay.
+ * Both reserve calls are synchronous and may allocate.
  */
 int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P);
+int stwq_reserve_layer(stwq_ctx* ctx, int64_t M, int K, int N, int P);
+uint64_t stwq_workspace_generation(const stwq_ctx* ctx);
 
 /*
  * Static token-wise calibration (Section 4.2: one set of quantization parameters per token
@@ -284,24 +308,45 @@ int qlinear_static(const float* X, const int32_t* pos_ids, int64_t M, int K, int
 int stwq_device_status(stwq_ctx* ctx, void* stream);
 
 /*
+ * Self-test of the bounded device-side wait (the paper has no counterpart; failure handling of the
+ * library). Launches one small CTA that waits, with the wait routine and the limit
+ * (STWQ_OPT_WAIT_LIMIT_MS, at most one second here) of the GEMM kernels, for a barrier that nothing
+ * completes. The wait gives up, the kernel records the timeout in the context's status word and
+ * returns; stwq_device_status() then reports STWQ_ERR_DEVICE_TIMEOUT once. waited_ns (device pointer
+ * to one uint64, may be NULL) receives the time the wait lasted. The context stays usable.
+ */
+int stwq_selftest_wait_expiry(stwq_ctx* ctx, uint64_t* waited_ns, void* stream);
+
+/*
  * Options (for tests and tuning). STWQ_OPT_GEMM_PATH: 0 = choose by shape (default),
  * 1 = always a tiled tensor-core GEMM, 2 = always the few-row (decode) variant (M <= 256 only),
  * 3 = always the single-CTA tiled GEMM (the fallback used when N or the s_w / bias pointers
  * do not meet the 16-byte rules of the CTA-pair kernel).
  * STWQ_OPT_WAIT_LIMIT_MS: limit of every device-side wait in milliseconds (default 2000).
  * The remaining options choose between kernel variants that compute the same results (the parity
- * tests use them to reach every variant; 0 = the library's own choice):
+ * tests use them to reach every variant; 0 = the library's own choice; any other value than those
+ * listed is refused with STWQ_ERR_DIM):
  * STWQ_OPT_TILE_N: 128 or 256 = tile width of the CTA-pair GEMM.
  * STWQ_OPT_VARIANT: 1 / 2 = CTA-pair GEMM epilogue through staged TMA stores / straight from
  *   registers; 5 = ordinary launches instead of programmatic dependent ones; 7 / 8 = the
  *   register-streaming / the TMA-ring quantize kernel.
- * STWQ_OPT_KSPLIT: n > 0 = cut the tiles of the last wave of the CTA-pair GEMM (every work item of
+ * STWQ_OPT_KSPLIT (-1 .. 64): n > 0 = cut the tiles of the last wave of the CTA-pair GEMM (every work item of
  *   the few-row kernel) into n ranges of K; -1 = the few-row kernel never cuts. The CTA-pair GEMM
  *   cuts only on request.
  */
 enum { STWQ_OPT_GEMM_PATH = 1, STWQ_OPT_WAIT_LIMIT_MS = 2, STWQ_OPT_TILE_N = 100, STWQ_OPT_VARIANT = 101,
        STWQ_OPT_KSPLIT = 102 };
 int stwq_set_option(stwq_ctx* ctx, int option, int value);
+
+/*
+ * Peak probe of the int8 tensor path (measurement aid; the paper has no counterpart). Launches one
+ * kernel in which `cta_pairs` CTA pairs (0 = as many as are resident at once, one pair per two SMs)
+ * each issue kblocks x 4 tcgen05.mma.cta_group::2.kind::i8 instructions (M 256, N 256, K 32) on operand
+ * tiles that stay in shared memory: no global traffic, no epilogue. *ops_per_launch (HOST pointer, may
+ * be NULL) receives pairs * kblocks * 4 * 2 * 256 * 256 * 32. The caller times the launch with events;
+ * ops / time is the rate the pipe delivers at the clocks the GPU holds. kblocks in 1 .. 2^22.
+ */
+int stwq_probe_int8_peak(stwq_ctx* ctx, int kblocks, int cta_pairs, int64_t* ops_per_launch, void* stream);
 
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t stwq_launch_count(const stwq_ctx* ctx);

@@ -84,6 +84,9 @@ def lib():
                                       C.c_int, C.c_int, dp, bp, ip, dp]
             L.orc_gps.argtypes = [fp, C.c_int64, C.c_int, fp, C.c_int, C.c_int, C.c_uint32, C.c_int,
                                   fp, ip]
+            L.orc_pack4.restype = C.c_int
+            L.orc_pack4.argtypes = [bp, C.c_int64, C.POINTER(C.c_uint8)]
+            L.orc_unpack4.argtypes = [C.POINTER(C.c_uint8), C.c_int64, bp]
             L.orc_gps_gain.restype = C.c_double
             L.orc_gps_gain.argtypes = [C.c_double] * 4
             _lib = L
@@ -313,7 +316,7 @@ def chain_codes(acc, pos_ids, s_tok, s_w, bias, act, s_ch_next, s_tok_next, bits
 
 
 def qlinear(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act=0):
-    """The whole quantized linear. Returns dict(Y float64, Xq int8, acc int32, mag float64)."""
+    """The whole quantized linear. Returns dict(Y float64, Xq int8, acc int32, mag float64, act)."""
     X = _f32(X)
     pos_ids = np.ascontiguousarray(pos_ids, np.int32)
     Wq = np.ascontiguousarray(Wq, np.int8)
@@ -332,7 +335,7 @@ def qlinear(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act=0):
                            _ptr(mag, C.c_double))
     if st != 0:
         raise ValueError("pos_ids outside [0, P)")
-    return {"Y": Y, "Xq": Xq, "acc": acc, "mag": mag}
+    return {"Y": Y, "Xq": Xq, "acc": acc, "mag": mag, "act": act}
 
 
 def gps(X, W, bits, pct_ppm=999900, variant=0):
@@ -352,3 +355,21 @@ def gps(X, W, bits, pct_ppm=999900, variant=0):
 def gps_gain(A, B, s_k, s_i):
     """Scaling gain of Eq. 13 / Eq. 15 given A = sum W^2 dX^2 and B = sum dW^2 X^2."""
     return float(lib().orc_gps_gain(A, B, s_k, s_i))
+
+
+def pack4(codes):
+    """Signed 4-bit codes [..., K] (K even, values in [-8, 7]) -> bytes [..., K/2], low nibble = even channel."""
+    codes = np.ascontiguousarray(codes, np.int8)
+    assert codes.shape[-1] % 2 == 0
+    out = np.empty(codes.shape[:-1] + (codes.shape[-1] // 2,), np.uint8)
+    if lib().orc_pack4(_ptr(codes, C.c_int8), out.size, _ptr(out, C.c_uint8)) != 0:
+        raise ValueError("a code lies outside [-8, 7]")
+    return out
+
+
+def unpack4(packed):
+    """Bytes [..., K/2] -> signed 4-bit codes [..., K] as int8."""
+    packed = np.ascontiguousarray(packed, np.uint8)
+    out = np.empty(packed.shape[:-1] + (packed.shape[-1] * 2,), np.int8)
+    lib().orc_unpack4(_ptr(packed, C.c_uint8), packed.size, _ptr(out, C.c_int8))
+    return out

@@ -718,3 +718,34 @@ double orc_gps_gain(double A, double B, double s_k, double s_i)
     return 0.5 * (A + B) - (s_i * s_i) / (2.0 * s_k * s_k) * A
            - (s_k * s_k) / (2.0 * s_i * s_i) * B;
 }
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Packed storage of 4-bit weight codes (the W4A8 setting of Appendix J, Table 11:
+ * 4-bit weights with 8-bit activations). The paper fixes the bit width, not a
+ * storage format; the format here is the plain one: two signed 4-bit codes in
+ * [-8, 7] per byte, two's complement nibbles, the code of the EVEN input channel
+ * in the low nibble and the code of the following ODD channel in the high one:
+ *   byte = (c[2j] & 0xF) | ((c[2j+1] & 0xF) << 4).
+ * Unpacking sign-extends each nibble. A row of K codes (K even) takes K/2 bytes.
+ * orc_pack4 returns -1 if a code lies outside [-8, 7] (nothing is clamped here:
+ * clamping is the quantizer's job).
+ */
+int orc_pack4(const int8_t* codes, int64_t n_pairs, uint8_t* bytes)
+{
+    for (int64_t j = 0; j < n_pairs; ++j) {
+        const int lo = codes[2 * j], hi = codes[2 * j + 1];
+        if (lo < -8 || lo > 7 || hi < -8 || hi > 7) return -1;
+        bytes[j] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
+    }
+    return 0;
+}
+
+void orc_unpack4(const uint8_t* bytes, int64_t n_pairs, int8_t* codes)
+{
+    for (int64_t j = 0; j < n_pairs; ++j) {
+        const int lo = bytes[j] & 0xF, hi = (bytes[j] >> 4) & 0xF;
+        codes[2 * j] = (int8_t)(lo >= 8 ? lo - 16 : lo);
+        codes[2 * j + 1] = (int8_t)(hi >= 8 ? hi - 16 : hi);
+    }
+}

@@ -13,7 +13,7 @@ import os
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libstwq.so")
 
-ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH = 0, 1, 2
+ACT_NONE, ACT_GELU_ERF, ACT_GELU_TANH, ACT_GELU_FAST = 0, 1, 2, 3
 OUT_F32, OUT_BF16, OUT_INT32 = 0, 1, 2
 OPT_GEMM_PATH, OPT_WAIT_LIMIT_MS = 1, 2
 OPT_TILE_N, OPT_VARIANT, OPT_KSPLIT = 100, 101, 102
@@ -22,7 +22,8 @@ STATIC_MAX_CODES = 4 * 1024 * 1024
 _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gps_fold", "stwq_quantize",
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
-            "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16"]
+            "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16", "stwq_reserve_layer",
+            "stwq_workspace_generation", "stwq_selftest_wait_expiry", "stwq_probe_int8_peak"]
 
 _lib = None
 
@@ -57,6 +58,11 @@ def load_library():
     L.stwq_destroy.argtypes = [vp]
     L.stwq_destroy.restype = None
     L.stwq_reserve.argtypes = [vp, i64, i32, i32]
+    L.stwq_reserve_layer.argtypes = [vp, i64, i32, i32, i32]
+    L.stwq_workspace_generation.argtypes = [vp]
+    L.stwq_workspace_generation.restype = C.c_uint64
+    L.stwq_selftest_wait_expiry.argtypes = [vp, vp, vp]
+    L.stwq_probe_int8_peak.argtypes = [vp, i32, i32, C.POINTER(i64), vp]
     L.stwq_calibrate.argtypes = [vp, vp, vp, i64, i32, i32, vp, i32, u32, vp, vp]
     L.gps_fold.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, vp]
     L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
@@ -91,17 +97,71 @@ def _p(t):
     return None if t is None else C.c_void_p(t.data_ptr())
 
 
+ERR_NULL, ERR_DIM, ERR_ALIGN, ERR_BITS, ERR_CUDA = -1, -2, -3, -4, -6
+_F32, _BF16, _I8, _I32 = "torch.float32", "torch.bfloat16", "torch.int8", "torch.int32"
+_OUT_DTYPES = {OUT_F32: _F32, OUT_BF16: _BF16, OUT_INT32: _I32}
+
+
+def check_args(where, device, *specs):
+    """Host-side check of the tensors handed to one C call, before any pointer is taken: every
+    tensor must be a dense (contiguous) CUDA tensor on `device` with the element type and the exact
+    shape the call's sizes imply. A spec is (name, tensor, dtype string, shape tuple, optional).
+    The C library sees only raw addresses and sizes; a transposed view, a wrong dtype or a short
+    vector would make a kernel read or write out of bounds. Raises StwqError; computes nothing."""
+    for name, t, dtype, shape, optional in specs:
+        if t is None:
+            if optional:
+                continue
+            raise StwqError(ERR_NULL, where, f"{name} is None")
+        if not getattr(t, "is_cuda", False):
+            raise StwqError(ERR_CUDA, where, f"{name} is not a CUDA tensor")
+        idx = t.device.index
+        if device is not None and idx is not None and idx != device:
+            raise StwqError(ERR_CUDA, where, f"{name} lives on cuda:{idx}, the call runs on cuda:{device}")
+        if str(t.dtype) != dtype:
+            raise StwqError(ERR_BITS, where, f"{name} has dtype {t.dtype}, expected {dtype}")
+        if tuple(t.shape) != tuple(shape):
+            raise StwqError(ERR_DIM, where, f"{name} has shape {tuple(t.shape)}, expected {tuple(shape)}")
+        if not t.is_contiguous():
+            raise StwqError(ERR_ALIGN, where, f"{name} is not contiguous (row-major dense storage is required)")
+
+
+def _mk(X, what="X"):
+    if X is None or len(X.shape) != 2:
+        raise StwqError(ERR_DIM, what, "a 2-D tensor is required")
+    return int(X.shape[0]), int(X.shape[1])
+
+
+def _out_dtype(where, out_dtype):
+    if out_dtype not in _OUT_DTYPES:
+        raise StwqError(ERR_BITS, where, f"out_dtype {out_dtype} is not OUT_F32 / OUT_BF16 / OUT_INT32")
+    return _OUT_DTYPES[out_dtype]
+
+
+def _layer_specs(where, X, x_dtype, pos_ids, Wq, s_w, s_tok, s_ch, bias, out_dtype, Y, need_scales=True):
+    """The tensors of a qlinear-shaped call: X [M,K], pos_ids [M], Wq [N,K], s_w [N], s_tok [P],
+    s_ch [K] or None, bias [N] or None, Y [M,N] of the type out_dtype names."""
+    M, K = _mk(X)
+    N, _ = _mk(Wq, "Wq")
+    P = int(s_tok.numel()) if s_tok is not None else 1
+    ydt = _out_dtype(where, out_dtype)
+    return M, K, N, P, [("X", X, x_dtype, (M, K), False), ("pos_ids", pos_ids, _I32, (M,), not need_scales),
+                        ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), not need_scales),
+                        ("s_tok", s_tok, _F32, (P,), not need_scales), ("s_ch", s_ch, _F32, (K,), True),
+                        ("bias", bias, _F32, (N,), True), ("Y", Y, ydt, (M, N), False)]
+
+
 def qlinear_static(X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
     """The context-free, allocation-free entry point: same arguments as Context.qlinear, runs on
     the tensors' device (made current for the call), scratch limited to STATIC_MAX_CODES codes."""
     import torch
     L = load_library()
-    M, K = X.shape
-    N = Wq.shape[0]
+    M, K, N, P, specs = _layer_specs("qlinear_static", X, _F32, pos_ids, Wq, s_w, s_tok, s_ch, bias, out_dtype, Y)
+    check_args("qlinear_static", X.device.index if getattr(X, "is_cuda", False) else None, *specs)
     with torch.cuda.device(X.device):
         if stream is None:
             stream = torch.cuda.current_stream(X.device)
-        rc = L.qlinear_static(_p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok), s_tok.numel(),
+        rc = L.qlinear_static(_p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok), P,
                               _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y), C.c_void_p(stream.cuda_stream))
     if rc != 0:
         raise StwqError(rc, "qlinear_static", L.stwq_strerror(rc).decode())
@@ -141,112 +201,161 @@ class Context:
             stream = self._torch.cuda.current_stream(self.device)
         return C.c_void_p(stream.cuda_stream)
 
+    def _args(self, where, *specs):
+        check_args(where, self.device, *specs)
+
     # ---- one method per C entry point, same name, same argument order -------------------
     def stwq_reserve(self, M, K, P):
         self._check(self._L.stwq_reserve(self._h, M, K, P), "stwq_reserve")
+
+    def stwq_reserve_layer(self, M, K, N, P):
+        self._check(self._L.stwq_reserve_layer(self._h, M, K, N, P), "stwq_reserve_layer")
+
+    def stwq_workspace_generation(self) -> int:
+        return int(self._L.stwq_workspace_generation(self._h))
 
     def stwq_set_option(self, option, value):
         self._check(self._L.stwq_set_option(self._h, option, value), "stwq_set_option")
 
     def stwq_calibrate(self, Xcal, pos_ids, P, s_ch, bits, pct_ppm, s_tok, stream=None):
-        rows, K = Xcal.shape
+        rows, K = _mk(Xcal, "Xcal")
+        self._args("stwq_calibrate", ("Xcal", Xcal, _F32, (rows, K), False), ("pos_ids", pos_ids, _I32, (rows,), False),
+                   ("s_ch", s_ch, _F32, (K,), True), ("s_tok", s_tok, _F32, (P,), False))
         self._check(self._L.stwq_calibrate(self._h, _p(Xcal), _p(pos_ids), rows, K, P, _p(s_ch), bits,
                                            pct_ppm, _p(s_tok), self._stream(stream)), "stwq_calibrate")
 
     def gps_scales(self, Xcal, W, bits, pct_ppm, variant, s_ch, k_star=None, stream=None):
-        rows, K = Xcal.shape
-        N = W.shape[0]
+        rows, K = _mk(Xcal, "Xcal")
+        N, _ = _mk(W, "W")
+        self._args("gps_scales", ("Xcal", Xcal, _F32, (rows, K), False), ("W", W, _F32, (N, K), False),
+                   ("s_ch", s_ch, _F32, (K,), False), ("k_star", k_star, _I32, (1,), True))
         self._check(self._L.gps_scales(self._h, _p(Xcal), rows, K, _p(W), N, bits, pct_ppm, variant, _p(s_ch),
                                        _p(k_star), self._stream(stream)), "gps_scales")
 
     def gps_fold(self, W, s_ch, bits, Wq, s_w, stream=None):
-        N, K = W.shape
+        N, K = _mk(W, "W")
+        self._args("gps_fold", ("W", W, _F32, (N, K), False), ("s_ch", s_ch, _F32, (K,), True),
+                   ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), False))
         self._check(self._L.gps_fold(self._h, _p(W), N, K, _p(s_ch), bits, _p(Wq), _p(s_w),
                                      self._stream(stream)), "gps_fold")
 
+    def _quantize_specs(self, X, x_dtype, pos_ids, s_ch, s_tok, Xq):
+        M, K = _mk(X)
+        P = int(s_tok.numel()) if s_tok is not None else 1
+        return M, K, P, [("X", X, x_dtype, (M, K), False), ("pos_ids", pos_ids, _I32, (M,), False),
+                         ("s_ch", s_ch, _F32, (K,), True), ("s_tok", s_tok, _F32, (P,), False),
+                         ("Xq", Xq, _I8, (M, K), False)]
+
     def stwq_quantize(self, X, pos_ids, s_ch, s_tok, bits, Xq, stream=None):
-        M, K = X.shape
+        M, K, P, specs = self._quantize_specs(X, _F32, pos_ids, s_ch, s_tok, Xq)
+        self._args("stwq_quantize", *specs)
         self._check(self._L.stwq_quantize(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok),
-                                          s_tok.numel(), bits, _p(Xq), self._stream(stream)),
-                    "stwq_quantize")
+                                          P, bits, _p(Xq), self._stream(stream)), "stwq_quantize")
 
     def stwq_quantize_bf16(self, X, pos_ids, s_ch, s_tok, bits, Xq, stream=None):
-        M, K = X.shape
+        M, K, P, specs = self._quantize_specs(X, _BF16, pos_ids, s_ch, s_tok, Xq)
+        self._args("stwq_quantize_bf16", *specs)
         self._check(self._L.stwq_quantize_bf16(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok),
-                                               s_tok.numel(), bits, _p(Xq), self._stream(stream)),
-                    "stwq_quantize_bf16")
+                                               P, bits, _p(Xq), self._stream(stream)), "stwq_quantize_bf16")
 
     def qlinear(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
-        M, K = X.shape
-        N = Wq.shape[0]
+        M, K, N, P, specs = _layer_specs("qlinear", X, _F32, pos_ids, Wq, s_w, s_tok, s_ch, bias, out_dtype, Y)
+        self._args("qlinear", *specs)
         self._check(self._L.qlinear(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
-                                    s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
+                                    P, _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
                                     self._stream(stream)), "qlinear")
 
     def qlinear_bf16(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
-        M, K = X.shape
-        N = Wq.shape[0]
+        M, K, N, P, specs = _layer_specs("qlinear_bf16", X, _BF16, pos_ids, Wq, s_w, s_tok, s_ch, bias, out_dtype, Y)
+        self._args("qlinear_bf16", *specs)
         self._check(self._L.qlinear_bf16(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
-                                    s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
-                                    self._stream(stream)), "qlinear_bf16")
+                                         P, _p(s_ch), _p(bias), bits, act, out_dtype, _p(Y),
+                                         self._stream(stream)), "qlinear_bf16")
 
     def qlinear_q(self, Xq, pos_ids, Wq, s_w, s_tok, bias, act, out_dtype, Y, stream=None):
-        M, K = Xq.shape
-        N = Wq.shape[0]
-        P = s_tok.numel() if s_tok is not None else 1
+        # raw accumulators (OUT_INT32) need no scales or positions
+        M, K, N, P, specs = _layer_specs("qlinear_q", Xq, _I8, pos_ids, Wq, s_w, s_tok, None, bias, out_dtype, Y,
+                                         need_scales=out_dtype != OUT_INT32)
+        self._args("qlinear_q", *specs)
         self._check(self._L.qlinear_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
                                       P, _p(bias), act, out_dtype, _p(Y), self._stream(stream)),
                     "qlinear_q")
 
+    def _chain_specs(self, where, X, x_dtype, pos_ids, Wq, s_w, s_tok, s_ch, bias, s_ch_next, s_tok_next, Xq_next):
+        M, K = _mk(X)
+        N, _ = _mk(Wq, "Wq")
+        P = int(s_tok.numel()) if s_tok is not None else 1
+        return M, K, N, P, [("X", X, x_dtype, (M, K), False), ("pos_ids", pos_ids, _I32, (M,), False),
+                            ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), False),
+                            ("s_tok", s_tok, _F32, (P,), False), ("s_ch", s_ch, _F32, (K,), True),
+                            ("bias", bias, _F32, (N,), True), ("s_ch_next", s_ch_next, _F32, (N,), True),
+                            ("s_tok_next", s_tok_next, _F32, (P,), False), ("Xq_next", Xq_next, _I8, (M, N), False)]
+
     def qlinear_chain(self, X, pos_ids, Wq, s_w, s_tok, s_ch, bias, bits, act, s_ch_next, s_tok_next, bits_next,
                       Xq_next, stream=None):
-        M, K = X.shape
-        N = Wq.shape[0]
+        M, K, N, P, specs = self._chain_specs("qlinear_chain", X, _F32, pos_ids, Wq, s_w, s_tok, s_ch, bias, s_ch_next,
+                                              s_tok_next, Xq_next)
+        self._args("qlinear_chain", *specs)
         self._check(self._L.qlinear_chain(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
-                                          s_tok.numel(), _p(s_ch), _p(bias), bits, act, _p(s_ch_next),
+                                          P, _p(s_ch), _p(bias), bits, act, _p(s_ch_next),
                                           _p(s_tok_next), bits_next, _p(Xq_next), self._stream(stream)),
                     "qlinear_chain")
 
     def qlinear_chain_q(self, Xq, pos_ids, Wq, s_w, s_tok, bias, act, s_ch_next, s_tok_next, bits_next, Xq_next,
                         stream=None):
-        M, K = Xq.shape
-        N = Wq.shape[0]
+        M, K, N, P, specs = self._chain_specs("qlinear_chain_q", Xq, _I8, pos_ids, Wq, s_w, s_tok, None, bias,
+                                              s_ch_next, s_tok_next, Xq_next)
+        self._args("qlinear_chain_q", *specs)
         self._check(self._L.qlinear_chain_q(self._h, _p(Xq), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(s_tok),
-                                            s_tok.numel(), _p(bias), act, _p(s_ch_next), _p(s_tok_next),
+                                            P, _p(bias), act, _p(s_ch_next), _p(s_tok_next),
                                             bits_next, _p(Xq_next), self._stream(stream)), "qlinear_chain_q")
 
     def stwq_calibrate_asym(self, Xcal, pos_ids, P, s_ch, bits, pct_ppm, s_tok, z_tok, stream=None):
-        rows, K = Xcal.shape
+        rows, K = _mk(Xcal, "Xcal")
+        self._args("stwq_calibrate_asym", ("Xcal", Xcal, _F32, (rows, K), False),
+                   ("pos_ids", pos_ids, _I32, (rows,), False), ("s_ch", s_ch, _F32, (K,), True),
+                   ("s_tok", s_tok, _F32, (P,), False), ("z_tok", z_tok, _I32, (P,), False))
         self._check(self._L.stwq_calibrate_asym(self._h, _p(Xcal), _p(pos_ids), rows, K, P, _p(s_ch), bits, pct_ppm,
                                                 _p(s_tok), _p(z_tok), self._stream(stream)), "stwq_calibrate_asym")
 
     def gps_fold_asym(self, W, s_ch, bits, Wq, s_w, z_w, colsum, stream=None):
-        N, K = W.shape
+        N, K = _mk(W, "W")
+        self._args("gps_fold_asym", ("W", W, _F32, (N, K), False), ("s_ch", s_ch, _F32, (K,), True),
+                   ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), False), ("z_w", z_w, _I32, (N,), False),
+                   ("colsum", colsum, _I32, (N,), False))
         self._check(self._L.gps_fold_asym(self._h, _p(W), N, K, _p(s_ch), bits, _p(Wq), _p(s_w), _p(z_w), _p(colsum),
                                           self._stream(stream)), "gps_fold_asym")
 
     def stwq_quantize_asym(self, X, pos_ids, s_ch, s_tok, z_tok, bits, Xq, rowcorr, stream=None):
-        M, K = X.shape
+        M, K, P, specs = self._quantize_specs(X, _F32, pos_ids, s_ch, s_tok, Xq)
+        self._args("stwq_quantize_asym", *specs, ("z_tok", z_tok, _I32, (P,), False),
+                   ("rowcorr", rowcorr, _I32, (M,), False))
         self._check(self._L.stwq_quantize_asym(self._h, _p(X), _p(pos_ids), M, K, _p(s_ch), _p(s_tok), _p(z_tok),
-                                               s_tok.numel(), bits, _p(Xq), _p(rowcorr), self._stream(stream)),
+                                               P, bits, _p(Xq), _p(rowcorr), self._stream(stream)),
                     "stwq_quantize_asym")
 
     def qlinear_asym(self, X, pos_ids, Wq, s_w, z_w, colsum, s_tok, z_tok, s_ch, bias, bits, act, out_dtype, Y,
                      stream=None):
-        M, K = X.shape
-        N = Wq.shape[0]
+        M, K, N, P, specs = _layer_specs("qlinear_asym", X, _F32, pos_ids, Wq, s_w, s_tok, s_ch, bias, out_dtype, Y)
+        self._args("qlinear_asym", *specs, ("z_w", z_w, _I32, (N,), False), ("colsum", colsum, _I32, (N,), False),
+                   ("z_tok", z_tok, _I32, (P,), False))
         self._check(self._L.qlinear_asym(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wq), _p(s_w), _p(z_w), _p(colsum),
-                                         _p(s_tok), _p(z_tok), s_tok.numel(), _p(s_ch), _p(bias), bits, act, out_dtype,
+                                         _p(s_tok), _p(z_tok), P, _p(s_ch), _p(bias), bits, act, out_dtype,
                                          _p(Y), self._stream(stream)), "qlinear_asym")
 
     def dtwq_quantize(self, X, s_ch, bits, Xq, s_row, stream=None):
-        M, K = X.shape
+        M, K = _mk(X)
+        self._args("dtwq_quantize", ("X", X, _F32, (M, K), False), ("s_ch", s_ch, _F32, (K,), True),
+                   ("Xq", Xq, _I8, (M, K), False), ("s_row", s_row, _F32, (M,), False))
         self._check(self._L.dtwq_quantize(self._h, _p(X), M, K, _p(s_ch), bits, _p(Xq), _p(s_row),
                                           self._stream(stream)), "dtwq_quantize")
 
     def qlinear_dtwq(self, X, Wq, s_w, s_ch, bias, bits, act, out_dtype, Y, stream=None):
-        M, K = X.shape
-        N = Wq.shape[0]
+        M, K = _mk(X)
+        N, _ = _mk(Wq, "Wq")
+        self._args("qlinear_dtwq", ("X", X, _F32, (M, K), False), ("Wq", Wq, _I8, (N, K), False),
+                   ("s_w", s_w, _F32, (N,), False), ("s_ch", s_ch, _F32, (K,), True), ("bias", bias, _F32, (N,), True),
+                   ("Y", Y, _out_dtype("qlinear_dtwq", out_dtype), (M, N), False))
         self._check(self._L.qlinear_dtwq(self._h, _p(X), M, K, N, _p(Wq), _p(s_w), _p(s_ch), _p(bias), bits, act,
                                          out_dtype, _p(Y), self._stream(stream)), "qlinear_dtwq")
 
@@ -255,6 +364,18 @@ class Context:
 
     def check_device_status(self, stream=None):
         self._check(self.stwq_device_status(stream), "device status")
+
+    def stwq_selftest_wait_expiry(self, waited_ns=None, stream=None):
+        self._args("stwq_selftest_wait_expiry", ("waited_ns", waited_ns, "torch.int64", (1,), True))
+        self._check(self._L.stwq_selftest_wait_expiry(self._h, _p(waited_ns), self._stream(stream)),
+                    "stwq_selftest_wait_expiry")
+
+    def stwq_probe_int8_peak(self, kblocks, cta_pairs=0, stream=None) -> int:
+        """Launch the peak probe; returns the int8 operations the launch performs."""
+        ops = C.c_int64(0)
+        self._check(self._L.stwq_probe_int8_peak(self._h, kblocks, cta_pairs, C.byref(ops), self._stream(stream)),
+                    "stwq_probe_int8_peak")
+        return int(ops.value)
 
     def stwq_launch_count(self) -> int:
         return int(self._L.stwq_launch_count(self._h))

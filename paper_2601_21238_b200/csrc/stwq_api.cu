@@ -14,69 +14,56 @@ int check_bits(int bits) { return (bits == 8 || bits == 6) ? STWQ_OK : STWQ_ERR_
 // weights may also be 4-bit (W4A8, Table 11): the codes still travel in int8 containers
 int check_wbits(int bits) { return (bits == 8 || bits == 6 || bits == 4) ? STWQ_OK : STWQ_ERR_BITS; }
 
-int ensure_xq(stwq_ctx* ctx, size_t bytes)
+}  // namespace
+
+// One workspace buffer of the context, grown on demand: free + allocate (both synchronise the
+// device). Growth is refused while the stream is being captured into a CUDA graph (an allocation
+// there would break the capture) and it bumps the context's workspace generation, because graphs
+// captured earlier hold the old address.
+int stwq_ensure_ws(stwq_ctx* ctx, void** buf, size_t* have, size_t bytes, cudaStream_t st, size_t zero_prefix)
 {
-    if (ctx->ws_xq_bytes >= bytes) return STWQ_OK;
-    if (ctx->ws_xq) {
-        cudaError_t e = cudaFree(ctx->ws_xq);           // synchronises
+    if (*have >= bytes) return STWQ_OK;
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess) {
+        (void)cudaGetLastError();
+        return STWQ_ERR_CAPTURE;        // the query itself fails while another stream of the thread captures
+    }
+    if (cap != cudaStreamCaptureStatusNone) return STWQ_ERR_CAPTURE;
+    if (*buf) {
+        cudaError_t e = cudaFree(*buf);                 // synchronises
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->ws_xq = nullptr;
-        ctx->ws_xq_bytes = 0;
+        *buf = nullptr;
+        *have = 0;
     }
     void* p = nullptr;
     cudaError_t e = cudaMalloc(&p, bytes);
+    if (e == cudaSuccess && zero_prefix > 0) e = cudaMemset(p, 0, zero_prefix);
     if (e != cudaSuccess) {
         ctx->last_cuda_error = (int)e;
         (void)cudaGetLastError();
+        if (p) cudaFree(p);
         return STWQ_ERR_NOMEM;
     }
-    ctx->ws_xq = static_cast<int8_t*>(p);
-    ctx->ws_xq_bytes = bytes;
+    *buf = p;
+    *have = bytes;
+    ctx->ws_generation += 1;
     return STWQ_OK;
 }
 
-int ensure_cal(stwq_ctx* ctx, int P)
+namespace {
+
+int ensure_xq(stwq_ctx* ctx, size_t bytes, cudaStream_t st)
 {
-    const size_t bytes = stwq_calibrate_ws_bytes(P);
-    if (ctx->ws_cal_bytes >= bytes) return STWQ_OK;
-    if (ctx->ws_cal) {
-        cudaError_t e = cudaFree(ctx->ws_cal);
-        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->ws_cal = nullptr;
-        ctx->ws_cal_bytes = 0;
-    }
-    void* p = nullptr;
-    cudaError_t e = cudaMalloc(&p, bytes);
-    if (e != cudaSuccess) {
-        ctx->last_cuda_error = (int)e;
-        (void)cudaGetLastError();
-        return STWQ_ERR_NOMEM;
-    }
-    ctx->ws_cal = p;
-    ctx->ws_cal_bytes = bytes;
-    return STWQ_OK;
+    return stwq_ensure_ws(ctx, reinterpret_cast<void**>(&ctx->ws_xq), &ctx->ws_xq_bytes, bytes, st, 0);
 }
-
+int ensure_cal(stwq_ctx* ctx, int P, cudaStream_t st)
+{
+    return stwq_ensure_ws(ctx, &ctx->ws_cal, &ctx->ws_cal_bytes, stwq_calibrate_ws_bytes(P), st, 0);
+}
 // Per-row workspace of qlinear_dtwq (row scales + row ids) and qlinear_asym (row corrections).
-int ensure_dyn(stwq_ctx* ctx, size_t bytes)
+int ensure_dyn(stwq_ctx* ctx, size_t bytes, cudaStream_t st)
 {
-    if (ctx->ws_dyn_bytes >= bytes) return STWQ_OK;
-    if (ctx->ws_dyn) {
-        cudaError_t e = cudaFree(ctx->ws_dyn);          // synchronises
-        if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-        ctx->ws_dyn = nullptr;
-        ctx->ws_dyn_bytes = 0;
-    }
-    void* p = nullptr;
-    cudaError_t e = cudaMalloc(&p, bytes);
-    if (e != cudaSuccess) {
-        ctx->last_cuda_error = (int)e;
-        (void)cudaGetLastError();
-        return STWQ_ERR_NOMEM;
-    }
-    ctx->ws_dyn = p;
-    ctx->ws_dyn_bytes = bytes;
-    return STWQ_OK;
+    return stwq_ensure_ws(ctx, &ctx->ws_dyn, &ctx->ws_dyn_bytes, bytes, st, 0);
 }
 
 // Make the context's device current for the duration of a call.
@@ -104,7 +91,7 @@ int check_gemm_args(const void* A, const int32_t* pos_ids, int64_t M, int K, int
     if (M <= 0 || K <= 0 || N <= 0 || P <= 0) return STWQ_ERR_DIM;
     if (M > (int64_t)0x7fffff00 || K >= 131072) return STWQ_ERR_DIM;   // int32 accumulation bound
     if ((K & 15) != 0 || !aligned16(A) || !aligned16(Wq) || !aligned16(Y)) return STWQ_ERR_ALIGN;
-    if (act < STWQ_ACT_NONE || act > STWQ_ACT_GELU_TANH) return STWQ_ERR_BITS;
+    if (act < STWQ_ACT_NONE || act > STWQ_ACT_GELU_FAST) return STWQ_ERR_BITS;
     if (out_dtype < STWQ_OUT_F32 || out_dtype > STWQ_OUT_INT32) return STWQ_ERR_BITS;
     return STWQ_OK;
 }
@@ -192,8 +179,32 @@ int stwq_reserve(stwq_ctx* ctx, int64_t M, int K, int P)
     if (M < 0 || K < 0 || P < 0) return STWQ_ERR_DIM;
     DeviceGuard g(ctx->device);
     int rc = STWQ_OK;
-    if (M > 0 && K > 0) rc = ensure_xq(ctx, (size_t)M * (size_t)K);
-    if (rc == STWQ_OK && P > 0) rc = ensure_cal(ctx, P);
+    if (M > 0 && K > 0) rc = ensure_xq(ctx, (size_t)M * (size_t)K, nullptr);
+    if (rc == STWQ_OK && P > 0) rc = ensure_cal(ctx, P, nullptr);
+    return rc;
+}
+
+int stwq_reserve_layer(stwq_ctx* ctx, int64_t M, int K, int N, int P)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (M <= 0 || K <= 0 || N <= 0 || P <= 0) return STWQ_ERR_DIM;
+    DeviceGuard g(ctx->device);
+    int rc = ensure_xq(ctx, (size_t)M * (size_t)K, nullptr);
+    if (rc == STWQ_OK) rc = ensure_cal(ctx, P, nullptr);
+    // per-row scratch of qlinear_dtwq / qlinear_asym, column statistics of gps_scales
+    size_t dyn = (size_t)M * 8;
+    if (stwq_gps_ws_bytes(K, N) > dyn) dyn = stwq_gps_ws_bytes(K, N);
+    if (rc == STWQ_OK) rc = ensure_dyn(ctx, dyn, nullptr);
+    // int32 partial sums of the few-row path when it splits K
+    if (rc == STWQ_OK && M <= 256) {
+        const size_t split = stwq_decode_split_bytes(ctx, K, N);
+        uint32_t* c = nullptr;
+        int32_t* part = nullptr;
+        if (split > 0) {
+            rc = stwq_split_ws(ctx, split, 1, &c, &part, nullptr);
+            if (rc == STWQ_ERR_DIM) rc = STWQ_OK;
+        }
+    }
     return rc;
 }
 
@@ -208,9 +219,18 @@ int stwq_set_option(stwq_ctx* ctx, int option, int value)
         ctx->wait_limit_ms = value;
         return STWQ_OK;
     }
-    if (option == STWQ_OPT_TILE_N) { ctx->force_bn = value; return STWQ_OK; }
-    if (option == STWQ_OPT_VARIANT) { ctx->debug = value; return STWQ_OK; }
-    if (option == STWQ_OPT_KSPLIT) { ctx->force_ksplit = value; return STWQ_OK; }
+    if (option == STWQ_OPT_TILE_N && (value == 0 || value == 128 || value == 256)) {
+        ctx->force_bn = value;
+        return STWQ_OK;
+    }
+    if (option == STWQ_OPT_VARIANT && (value == 0 || value == 1 || value == 2 || value == 5 || value == 7 || value == 8)) {
+        ctx->debug = value;
+        return STWQ_OK;
+    }
+    if (option == STWQ_OPT_KSPLIT && value >= -1 && value <= 64) {
+        ctx->force_ksplit = value;
+        return STWQ_OK;
+    }
     return STWQ_ERR_DIM;
 }
 
@@ -221,7 +241,7 @@ int stwq_calibrate(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids, int
     if (rows <= 0 || K <= 0 || P <= 0 || P > (1 << 20)) return STWQ_ERR_DIM;
     if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    int rc = ensure_cal(ctx, P);
+    int rc = ensure_cal(ctx, P, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     return stwq_launch_calibrate(ctx, ctx->ws_cal, Xcal, pos_ids, rows, K, P, s_ch, bits, pct_ppm, s_tok,
                                  static_cast<cudaStream_t>(stream));
@@ -235,8 +255,8 @@ int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const floa
     if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
     if (variant != 0 && variant != 1) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    int rc = ensure_cal(ctx, 1);
-    if (rc == STWQ_OK) rc = ensure_dyn(ctx, stwq_gps_ws_bytes(K, N));
+    int rc = ensure_cal(ctx, 1, static_cast<cudaStream_t>(stream));
+    if (rc == STWQ_OK) rc = ensure_dyn(ctx, stwq_gps_ws_bytes(K, N), static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     return stwq_launch_gps(ctx, ctx->ws_cal, ctx->ws_dyn, Xcal, rows, K, W, N, bits, pct_ppm, variant, s_ch, k_star,
                            static_cast<cudaStream_t>(stream));
@@ -297,7 +317,7 @@ int qlinear(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, in
     if (rc != STWQ_OK) return rc;
     if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     // Both kernels are launched as programmatic dependents of their predecessor in the stream:
@@ -320,7 +340,7 @@ int qlinear_bf16(stwq_ctx* ctx, const void* X, const int32_t* pos_ids, int64_t M
     if (rc != STWQ_OK) return rc;
     if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     rc = stwq_launch_quantize_bf16(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, st);
@@ -366,7 +386,7 @@ int qlinear_chain(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t
     if (rc != STWQ_OK) return rc;
     if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool pdl = ctx->debug != 5;
@@ -384,7 +404,7 @@ int stwq_calibrate_asym(stwq_ctx* ctx, const float* Xcal, const int32_t* pos_ids
     if (rows <= 0 || K <= 0 || P <= 0 || P > (1 << 20)) return STWQ_ERR_DIM;
     if (check_bits(bits) != STWQ_OK || pct_ppm < 1u || pct_ppm > 1000000u) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
-    int rc = ensure_cal(ctx, P);
+    int rc = ensure_cal(ctx, P, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     return stwq_launch_calibrate_asym(ctx, ctx->ws_cal, Xcal, pos_ids, rows, K, P, s_ch, bits, pct_ppm, s_tok, z_tok,
                                       static_cast<cudaStream_t>(stream));
@@ -426,9 +446,9 @@ int qlinear_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t 
     if (!stwq_qgemm2_supported(N, out_dtype, s_w, bias) || (N & 3) != 0 || !aligned16(z_w) || !aligned16(colsum))
         return STWQ_ERR_ALIGN;
     DeviceGuard g(ctx->device);
-    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
-    rc = ensure_dyn(ctx, (size_t)M * 8);
+    rc = ensure_dyn(ctx, (size_t)M * 8, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     int32_t* rowcorr = static_cast<int32_t*>(ctx->ws_dyn);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -462,9 +482,9 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
     if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     if (K > 8192 || M > (int64_t)0x7fffffff) return STWQ_ERR_DIM;
     DeviceGuard g(ctx->device);
-    rc = ensure_xq(ctx, (size_t)M * (size_t)K);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
-    rc = ensure_dyn(ctx, (size_t)M * 8);
+    rc = ensure_dyn(ctx, (size_t)M * 8, static_cast<cudaStream_t>(stream));
     if (rc != STWQ_OK) return rc;
     float* s_row = static_cast<float*>(ctx->ws_dyn);
     int32_t* row_ids = reinterpret_cast<int32_t*>(s_row + M);
@@ -493,6 +513,8 @@ int stwq_device_status(stwq_ctx* ctx, void* stream)
 
 int64_t stwq_launch_count(const stwq_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+uint64_t stwq_workspace_generation(const stwq_ctx* ctx) { return ctx ? ctx->ws_generation : 0; }
+
 int stwq_last_cuda_error(const stwq_ctx* ctx) { return ctx ? ctx->last_cuda_error : 0; }
 
 const char* stwq_strerror(int status)
@@ -509,6 +531,7 @@ const char* stwq_strerror(int status)
         case STWQ_ERR_POS_RANGE: return "a position id was outside [0, P)";
         case STWQ_ERR_NONFINITE: return "calibration input contains NaN or Inf";
         case STWQ_ERR_NOMEM: return "workspace allocation failed";
+        case STWQ_ERR_CAPTURE: return "workspace would have to grow during stream capture (reserve it first)";
         default: return "unknown status";
     }
 }

@@ -292,7 +292,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             const uint64_t sw = pack_f2(my_sw[h * 32 + j], my_sw[h * 32 + j + 1]);
                             const uint64_t bi = pack_f2(my_bias[h * 32 + j], my_bias[h * 32 + j + 1]);
                             uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
-                            if (ACT != STWQ_ACT_NONE) z = gelu_fast_f2(z);
+                            z = apply_act_f2<ACT>(z);
                             float v0, v1;
                             unpack_f2(z, v0, v1);
                             w[j / 2] = pack_bf16(v0, v1);
@@ -315,8 +315,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                 const uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
                                 float v0, v1;
                                 unpack_f2(z, v0, v1);
-                                w[j] = __float_as_uint(apply_act<ACT, false>(v0));
-                                w[j + 1] = __float_as_uint(apply_act<ACT, false>(v1));
+                                w[j] = __float_as_uint(apply_act<ACT>(v0));
+                                w[j + 1] = __float_as_uint(apply_act<ACT>(v1));
                             }
                         }
 #pragma unroll
@@ -387,36 +387,56 @@ int launch_variant(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
 }
 
+// How a few-row problem is cut into work items.
+struct DecPlan {
+    int num_kb, tiles_n, ksplit, kb_per_split, items;
+};
+DecPlan plan_decode(const stwq_ctx* ctx, int K, int N)
+{
+    DecPlan d;
+    d.num_kb = (K + kBK - 1) / kBK;
+    d.tiles_n = (N + kBN - 1) / kBN;
+    // One work item per CTA pair if N allows; otherwise K may be split so that more pairs have
+    // work. The exchange of partial sums costs 2-3 us, so this pays only for long K: measured
+    // (M 256, weights from HBM, N 1024-4096) no split is best up to K 2048 (7.7-11.3 us against
+    // 10.3-13.0 us with two ranges), and from K 4096 on two to four ranges of at least eight
+    // k-blocks each (K 8192, N 1024: 27.2 us whole, 17.2 us in four ranges, 18.3 in eight).
+    const int pairs = ctx->sm_count / 2;
+    int ksplit = 1;
+    if (d.tiles_n * 4 < pairs * 3 && d.num_kb >= 32) {
+        ksplit = pairs / d.tiles_n;
+        if (ksplit > d.num_kb / 8) ksplit = d.num_kb / 8;
+        if (ksplit > 4) ksplit = 4;
+        if (ksplit < 1) ksplit = 1;
+    }
+    if (ctx->force_ksplit > 0) ksplit = ctx->force_ksplit < d.num_kb ? ctx->force_ksplit : d.num_kb;
+    if (ctx->force_ksplit < 0) ksplit = 1;
+    d.kb_per_split = (d.num_kb + ksplit - 1) / ksplit;
+    d.ksplit = (d.num_kb + d.kb_per_split - 1) / d.kb_per_split;      // every range holds at least one k-block
+    d.items = d.tiles_n * d.ksplit;
+    return d;
+}
+
 }  // namespace
+
+// Bytes of split-K scratch the few-row path wants for a [<= 256, K] x [N, K] problem (0: no split).
+size_t stwq_decode_split_bytes(const stwq_ctx* ctx, int K, int N)
+{
+    const DecPlan d = plan_decode(ctx, K, N);
+    return d.ksplit > 1 ? (size_t)d.items * 2 * kEpi * kPieceInts * sizeof(int32_t) : 0;
+}
 
 // Scratch for split-K (shared by the few-row kernel and the tail of the tiled GEMM): a fixed
 // region of kSplitCounters arrival counters, zero between calls because the last arriver resets
 // its counter, followed by room for the int32 partial sums.
-int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial)
+int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial,
+                  cudaStream_t st)
 {
     constexpr size_t kSplitCounters = 16384;
     constexpr size_t counter_bytes = kSplitCounters * sizeof(uint32_t);
     if (n_counters > kSplitCounters) return STWQ_ERR_DIM;
-    const size_t need = partial_bytes + counter_bytes;
-    if (ctx->ws_dec_bytes < need) {
-        if (ctx->ws_dec) {
-            cudaError_t e = cudaFree(ctx->ws_dec);        // synchronises
-            if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-            ctx->ws_dec = nullptr;
-            ctx->ws_dec_bytes = 0;
-        }
-        void* ptr = nullptr;
-        cudaError_t e = cudaMalloc(&ptr, need);
-        if (e == cudaSuccess) e = cudaMemset(ptr, 0, counter_bytes);
-        if (e != cudaSuccess) {
-            ctx->last_cuda_error = (int)e;
-            (void)cudaGetLastError();
-            if (ptr) cudaFree(ptr);
-            return STWQ_ERR_NOMEM;
-        }
-        ctx->ws_dec = ptr;
-        ctx->ws_dec_bytes = need;
-    }
+    int rc = stwq_ensure_ws(ctx, &ctx->ws_dec, &ctx->ws_dec_bytes, partial_bytes + counter_bytes, st, counter_bytes);
+    if (rc != STWQ_OK) return rc;
     *counters = reinterpret_cast<uint32_t*>(ctx->ws_dec);
     *partial = reinterpret_cast<int32_t*>(reinterpret_cast<uint8_t*>(ctx->ws_dec) + counter_bytes);
     return STWQ_OK;
@@ -434,31 +454,17 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     DecParams p;
     p.M = M; p.N = N; p.K = K; p.P = P;
     p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
-    p.num_kb = (K + kBK - 1) / kBK;
-    const int tiles_n = (N + kBN - 1) / kBN;
-    // One work item per CTA pair if N allows; otherwise K may be split so that more pairs have
-    // work. The exchange of partial sums costs 2-3 us, so this pays only for long K: measured
-    // (M 256, weights from HBM, N 1024-4096) no split is best up to K 2048 (7.7-11.3 us against
-    // 10.3-13.0 us with two ranges), and from K 4096 on two to four ranges of at least eight
-    // k-blocks each (K 8192, N 1024: 27.2 us whole, 17.2 us in four ranges, 18.3 in eight).
-    const int pairs = ctx->sm_count / 2;
-    int ksplit = 1;
-    if (tiles_n * 4 < pairs * 3 && p.num_kb >= 32) {
-        ksplit = pairs / tiles_n;
-        if (ksplit > p.num_kb / 8) ksplit = p.num_kb / 8;
-        if (ksplit > 4) ksplit = 4;
-        if (ksplit < 1) ksplit = 1;
-    }
-    if (ctx->force_ksplit > 0) ksplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
-    if (ctx->force_ksplit < 0) ksplit = 1;
-    p.kb_per_split = (p.num_kb + ksplit - 1) / ksplit;
-    p.ksplit = (p.num_kb + p.kb_per_split - 1) / p.kb_per_split;      // every range holds at least one k-block
-    const int items = tiles_n * p.ksplit;
+    const DecPlan plan = plan_decode(ctx, K, N);
+    p.num_kb = plan.num_kb;
+    p.kb_per_split = plan.kb_per_split;
+    p.ksplit = plan.ksplit;
+    const int tiles_n = plan.tiles_n;
+    const int items = plan.items;
     p.partial = nullptr;
     p.counters = nullptr;
     if (p.ksplit > 1) {
         int rc = stwq_split_ws(ctx, (size_t)items * 2 * kEpi * kPieceInts * sizeof(int32_t), (size_t)tiles_n * 2 * kEpi,
-                               &p.counters, &p.partial);
+                               &p.counters, &p.partial, st);
         if (rc == STWQ_ERR_DIM)                            // more N slices than counters: no split-K path
             return stwq_launch_qgemm(ctx, Xq, pos_ids, M, K, N, Wq, s_w, s_tok, P, bias, act, out_dtype, Y, st);
         if (rc != STWQ_OK) return rc;
@@ -486,9 +492,11 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_FAST)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_FAST)
 #undef STWQ_CASE
     return STWQ_ERR_BITS;
 }

@@ -38,6 +38,8 @@ struct stwq_ctx {
     size_t ws_dec_bytes;
     uint64_t configured_decode;
     int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
+    uint64_t ws_generation;    // bumped whenever a workspace buffer is (re)allocated
+    int probe_configured;      // the peak-probe kernel has its shared-memory attribute set
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
 };
 
@@ -94,7 +96,12 @@ int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
 
 int stwq_launch_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, const float* s_ch, int bits, int8_t* Xq,
                      float* s_row, int32_t* row_ids, cudaStream_t st);
-int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial);
+size_t stwq_decode_split_bytes(const stwq_ctx* ctx, int K, int N);
+int stwq_split_ws(stwq_ctx* ctx, size_t partial_bytes, size_t n_counters, uint32_t** counters, int32_t** partial,
+                  cudaStream_t st);
+// Grow one workspace buffer of the context to `bytes` (no-op if it is large enough). Refused with
+// STWQ_ERR_CAPTURE while `st` is being captured; the first zero_prefix bytes of a new buffer are cleared.
+int stwq_ensure_ws(stwq_ctx* ctx, void** buf, size_t* have, size_t bytes, cudaStream_t st, size_t zero_prefix);
 
 static inline int stwq_cuda_fail(stwq_ctx* ctx, cudaError_t e)
 {

@@ -201,24 +201,34 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
 }
 
 
-// GELU in the epilogue, two accuracy classes.
+// GELU in the epilogue.
 //
-// FAST = false (fp32 output, tolerance 1e-5). The erf form uses the rational approximation of
-// the complementary error function by Abramowitz and Stegun (formula 7.1.26; absolute error
-// below 1.5e-7):  erfc(x) ~ (a1 t + ... + a5 t^5) exp(-x^2),  t = 1 / (1 + p x),  x >= 0,
-// so that Phi(z) = erfc(|z|/sqrt2)/2 for z < 0 and 1 - erfc(|z|/sqrt2)/2 otherwise. The tanh form
-// is z * sigmoid(2u), u = sqrt(2/pi) (z + 0.044715 z^3).
-//
-// FAST = true (bf16 output, tolerance 1e-2, rounding unit 2^-9). Both forms are evaluated as
-// z/2 (1 + tanh(u)) with the hardware tanh (tanh.approx.f32, relative error about 2^-11): six
-// instructions per element. For the erf form this relies on the classical fit
-// erf(x / sqrt2) ~ tanh(sqrt(2/pi) (x + 0.044715 x^3)), whose error on Phi stays below 5e-4, a
-// quarter of the bf16 rounding unit. The epilogue of a K = 1024 tile has only a few thousand
-// issue slots, and a 25-instruction erf more than doubles the kernel time.
+// STWQ_ACT_GELU_ERF is z Phi(z) with Phi(-|z|) = erfc(|z| / sqrt2) / 2 evaluated as one exp2 of a
+// polynomial (see gelu_erf_f2; absolute error on Phi below 1.5e-7) and Phi(|z|) = 1 - Phi(-|z|).
+// STWQ_ACT_GELU_TANH is z * sigmoid(2u), u = sqrt(2/pi) (z + 0.044715 z^3), with the hardware's
+// exp2 and reciprocal (relative error about 2^-22 each).
+// STWQ_ACT_GELU_FAST is z/2 (1 + tanh(u)) with the hardware tanh (tanh.approx.f32, relative error
+// about 2^-11): six instructions per element. Its error on y stays below 6e-4 |z|, a quarter of
+// the bf16 rounding unit. The epilogue of a K = 1024 tile has only a few thousand issue slots,
+// which is why the short form exists; the caller asks for it by name.
+// Each form comes as a scalar function (fp32 output) and as a packed one on two values (bf16
+// output and chained codes), the packed one sharing its multiplies between the two halves.
 __device__ __forceinline__ float tanh_approx(float x)
 {
     float y;
     asm("tanh.approx.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float ex2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_approx(float x)
+{
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 // Packed fp32 arithmetic (two IEEE round-to-nearest operations per instruction on sm_100): the
@@ -246,38 +256,94 @@ __device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c)
     asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
     return r;
 }
-// The short GELU (see below) on a pair: z/2 (1 + tanh(z (c1 + c3 z^2))).
+__device__ __forceinline__ uint64_t dup_f2(float v) { return pack_f2(v, v); }
+// The short GELU on a pair: z/2 (1 + tanh(z (c1 + c3 z^2))).
 __device__ __forceinline__ uint64_t gelu_fast_f2(uint64_t z)
 {
-    const uint64_t c3 = pack_f2(0.035677408136300125f, 0.035677408136300125f);
-    const uint64_t c1 = pack_f2(0.79788456080286536f, 0.79788456080286536f);
-    const uint64_t half = pack_f2(0.5f, 0.5f);
-    const uint64_t u = mul_f2(z, fma_f2(c3, mul_f2(z, z), c1));
+    const uint64_t u = mul_f2(z, fma_f2(dup_f2(0.035677408136300125f), mul_f2(z, z), dup_f2(0.79788456080286536f)));
     float u0, u1;
     unpack_f2(u, u0, u1);
     const uint64_t t = pack_f2(tanh_approx(u0), tanh_approx(u1));
-    const uint64_t h = mul_f2(half, z);
+    const uint64_t h = mul_f2(dup_f2(0.5f), z);
     return fma_f2(h, t, h);
 }
-template <int ACT, bool FAST = false>
+// The tanh form to fp32 accuracy on a pair: z / (1 + exp(-2u)).
+__device__ __forceinline__ uint64_t gelu_tanh_f2(uint64_t z)
+{
+    // -2 log2(e) sqrt(2/pi) (1 + 0.044715 z^2) z
+    const uint64_t a = mul_f2(z, fma_f2(dup_f2(-0.1029432395800235f), mul_f2(z, z), dup_f2(-2.302208198144325f)));
+    float a0, a1;
+    unpack_f2(a, a0, a1);
+    const uint64_t den = fma_f2(dup_f2(1.0f), pack_f2(ex2_approx(a0), ex2_approx(a1)), dup_f2(1.0f));
+    float d0, d1;
+    unpack_f2(den, d0, d1);
+    return mul_f2(z, pack_f2(rcp_approx(d0), rcp_approx(d1)));
+}
+// The erf form on a pair. For m = |z|: Phi(-m) = erfc(m / sqrt2) / 2 = 2^(-m^2 log2(e) / 2 + q(m)),
+// q(m) = log2(erfcx(m / sqrt2)) - 1, a smooth, slowly varying function that a degree-7 polynomial
+// (STWQ_ERF_Q0..7, a weighted least-maximum fit on [0, 5.94]) follows closely enough for an absolute error
+// on Phi below 4e-8; evaluated in fp32 with the hardware exp2 the error stays below 1.5e-7. Beyond
+// m = 5.94 the argument is clamped (Phi < 1.5e-9 there). One special-function instruction per
+// element, where the textbook rational forms of erfc need a reciprocal and an exponential.
+#define STWQ_ERF_Q0 -0.9999998807907104f
+#define STWQ_ERF_Q1 -1.1511108875274658f
+#define STWQ_ERF_Q2 0.26219436526298523f
+#define STWQ_ERF_Q3 -0.05269109085202217f
+#define STWQ_ERF_Q4 0.007389252074062824f
+#define STWQ_ERF_Q5 -0.0004212251224089414f
+#define STWQ_ERF_Q6 -5.390652222558856e-05f
+#define STWQ_ERF_Q7 8.4704415712622e-06f
+#define STWQ_ERF_MMAX 5.94f
+#define STWQ_ERF_HALF_LOG2E -0.72134752044448170368f
+__device__ __forceinline__ uint64_t gelu_erf_f2(uint64_t z)
+{
+    float z0, z1;
+    unpack_f2(z, z0, z1);
+    const uint64_t m = pack_f2(fminf(fabsf(z0), STWQ_ERF_MMAX), fminf(fabsf(z1), STWQ_ERF_MMAX));
+    uint64_t q = fma_f2(dup_f2(STWQ_ERF_Q7), m, dup_f2(STWQ_ERF_Q6));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q5));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q4));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q3));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q2));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q1));
+    q = fma_f2(q, m, dup_f2(STWQ_ERF_Q0));
+    const uint64_t a = fma_f2(mul_f2(m, m), dup_f2(STWQ_ERF_HALF_LOG2E), q);
+    float a0, a1;
+    unpack_f2(a, a0, a1);
+    float h0, h1;
+    unpack_f2(mul_f2(z, pack_f2(ex2_approx(a0), ex2_approx(a1))), h0, h1);    // z Phi(-|z|)
+    return pack_f2(z0 < 0.0f ? h0 : z0 - h0, z1 < 0.0f ? h1 : z1 - h1);
+}
+__device__ __forceinline__ float gelu_erf(float z)
+{
+    const float m = fminf(fabsf(z), STWQ_ERF_MMAX);
+    float q = fmaf(STWQ_ERF_Q7, m, STWQ_ERF_Q6);
+    q = fmaf(q, m, STWQ_ERF_Q5);
+    q = fmaf(q, m, STWQ_ERF_Q4);
+    q = fmaf(q, m, STWQ_ERF_Q3);
+    q = fmaf(q, m, STWQ_ERF_Q2);
+    q = fmaf(q, m, STWQ_ERF_Q1);
+    q = fmaf(q, m, STWQ_ERF_Q0);
+    const float h = z * ex2_approx(fmaf(m * m, STWQ_ERF_HALF_LOG2E, q));
+    return z < 0.0f ? h : z - h;
+}
+template <int ACT>
+__device__ __forceinline__ uint64_t apply_act_f2(uint64_t z)
+{
+    if (ACT == STWQ_ACT_GELU_ERF) return gelu_erf_f2(z);
+    if (ACT == STWQ_ACT_GELU_TANH) return gelu_tanh_f2(z);
+    if (ACT == STWQ_ACT_GELU_FAST) return gelu_fast_f2(z);
+    return z;
+}
+template <int ACT>
 __device__ __forceinline__ float apply_act(float z)
 {
-    if (ACT != STWQ_ACT_NONE && FAST) {
+    if (ACT == STWQ_ACT_GELU_FAST) {
         const float u = z * fmaf(0.035677408136300125f, z * z, 0.79788456080286536f);
         const float h = 0.5f * z;
         return fmaf(h, tanh_approx(u), h);
     }
-    if (ACT == STWQ_ACT_GELU_ERF) {
-        const float x = fabsf(z) * 0.70710678118654752f;
-        const float t = __fdividef(1.0f, fmaf(0.3275911f, x, 1.0f));
-        float poly = fmaf(1.061405429f, t, -1.453152027f);
-        poly = fmaf(poly, t, 1.421413741f);
-        poly = fmaf(poly, t, -0.284496736f);
-        poly = fmaf(poly, t, 0.254829592f);
-        const float half_erfc = 0.5f * poly * t * __expf(-x * x);
-        const float phi = z < 0.0f ? half_erfc : 1.0f - half_erfc;
-        return z * phi;
-    }
+    if (ACT == STWQ_ACT_GELU_ERF) return gelu_erf(z);
     if (ACT == STWQ_ACT_GELU_TANH) {
         const float u = 0.79788456080286536f * fmaf(0.044715f * z * z, z, z);
         return __fdividef(z, 1.0f + __expf(-2.0f * u));

@@ -325,9 +325,11 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_FAST)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_FAST)
 #undef STWQ_CASE
     return STWQ_ERR_BITS;
 }

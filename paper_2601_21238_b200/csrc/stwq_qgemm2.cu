@@ -417,10 +417,8 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                                   mul_f2(st2, pack_f2(sw.x, sw.y)), pack_f2(bi.x, bi.y));
                             uint64_t z23 = fma_f2(pack_f2((float)(int32_t)r[j + 2], (float)(int32_t)r[j + 3]),
                                                   mul_f2(st2, pack_f2(sw.z, sw.w)), pack_f2(bi.z, bi.w));
-                            if (ACT != STWQ_ACT_NONE) {
-                                z01 = gelu_fast_f2(z01);
-                                z23 = gelu_fast_f2(z23);
-                            }
+                            z01 = apply_act_f2<ACT>(z01);
+                            z23 = apply_act_f2<ACT>(z23);
                             float v0, v1, v2, v3;
                             unpack_f2(z01, v0, v1);
                             unpack_f2(z23, v2, v3);
@@ -452,10 +450,8 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                                                   mul_f2(st2, pack_f2(sw.x, sw.y)), pack_f2(bi.x, bi.y));
                             uint64_t z23 = fma_f2(pack_f2((float)(int32_t)r[j + 2], (float)(int32_t)r[j + 3]),
                                                   mul_f2(st2, pack_f2(sw.z, sw.w)), pack_f2(bi.z, bi.w));
-                            if (ACT != STWQ_ACT_NONE) {
-                                z01 = gelu_fast_f2(z01);
-                                z23 = gelu_fast_f2(z23);
-                            }
+                            z01 = apply_act_f2<ACT>(z01);
+                            z23 = apply_act_f2<ACT>(z23);
                             float v0, v1, v2, v3;
                             unpack_f2(z01, v0, v1);
                             unpack_f2(z23, v2, v3);
@@ -475,10 +471,10 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         float v0, v1, v2, v3;
                         unpack_f2(z01, v0, v1);
                         unpack_f2(z23, v2, v3);
-                        w[j + 0] = __float_as_uint(apply_act<ACT, false>(v0));
-                        w[j + 1] = __float_as_uint(apply_act<ACT, false>(v1));
-                        w[j + 2] = __float_as_uint(apply_act<ACT, false>(v2));
-                        w[j + 3] = __float_as_uint(apply_act<ACT, false>(v3));
+                        w[j + 0] = __float_as_uint(apply_act<ACT>(v0));
+                        w[j + 1] = __float_as_uint(apply_act<ACT>(v1));
+                        w[j + 2] = __float_as_uint(apply_act<ACT>(v2));
+                        w[j + 3] = __float_as_uint(apply_act<ACT>(v3));
                     }
                 } else {
 #pragma unroll
@@ -621,9 +617,11 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
             STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_NONE)
             STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
             STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+            STWQ_ACASE(STWQ_OUT_F32, STWQ_ACT_GELU_FAST)
             STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
             STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
             STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+            STWQ_ACASE(STWQ_OUT_BF16, STWQ_ACT_GELU_FAST)
 #undef STWQ_ACASE
         }
         return STWQ_ERR_DIM;
@@ -635,15 +633,18 @@ int launch_bn(stwq_ctx* ctx, const CUtensorMap& tmA, const CUtensorMap& tmB, con
             STWQ_CASE(kOutCodes, STWQ_ACT_NONE)
             STWQ_CASE(kOutCodes, STWQ_ACT_GELU_ERF)
             STWQ_CASE(kOutCodes, STWQ_ACT_GELU_TANH)
+            STWQ_CASE(kOutCodes, STWQ_ACT_GELU_FAST)
         }
         return STWQ_ERR_DIM;
     }
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_F32, STWQ_ACT_GELU_FAST)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_NONE)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_ERF)
     STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_TANH)
+    STWQ_CASE(STWQ_OUT_BF16, STWQ_ACT_GELU_FAST)
 #undef STWQ_CASE
     return STWQ_ERR_BITS;
 }
@@ -717,7 +718,7 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
             nsplit = (p.num_kb + kbps - 1) / kbps;             // every range holds at least one k-block
             const size_t piece_bytes = (size_t)4 * 32 * 32 * sizeof(int32_t);      // 32 rows x 128 columns
             int rc = stwq_split_ws(ctx, (size_t)tail * nsplit * 2 * 8 * piece_bytes, (size_t)tail * 2 * 8, &p.counters,
-                                   &p.partial);
+                                   &p.partial, st);
             if (rc == STWQ_OK && nsplit >= 2) {
                 p.full_units = p.num_tiles - tail;
                 p.nsplit = nsplit;

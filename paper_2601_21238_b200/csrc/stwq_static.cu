@@ -98,7 +98,7 @@ extern "C" int qlinear_static(const float* X, const int32_t* pos_ids, int64_t M,
     if ((uint64_t)M * (uint64_t)K > (uint64_t)kCodeBytes) return STWQ_ERR_DIM;   // beyond the fixed scratch
     if ((K & 15) != 0 || !aligned16(X) || !aligned16(Wq) || !aligned16(Y)) return STWQ_ERR_ALIGN;
     if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
-    if (act < STWQ_ACT_NONE || act > STWQ_ACT_GELU_TANH) return STWQ_ERR_BITS;
+    if (act < STWQ_ACT_NONE || act > STWQ_ACT_GELU_FAST) return STWQ_ERR_BITS;
     if (out_dtype < STWQ_OUT_F32 || out_dtype > STWQ_OUT_INT32) return STWQ_ERR_BITS;
 
     int device = -1;

@@ -28,9 +28,21 @@ def sample_rows(M: int, n: int = 768, tile: int = 128) -> np.ndarray:
 
 
 def assert_close(Y, ref, rtol, what=""):
-    """|y - y_ref| <= rtol * (|y_ref| + |acc * s_tok * s_w| + |bias|), element by element."""
+    """Element-by-element bound on |y - y_ref|, with mag = |acc * s_tok * s_w| + |bias|:
+
+    * no activation (ref["act"] == 0): rtol * |y_ref| + 4 * 2^-24 * mag. The first term is the
+      relative error the target names; the second is the fp32 rounding of the terms y is built from
+      (int -> float of the accumulator, the scale product, the fused multiply-add), which is all that
+      is left of y where the bias cancels the product and a pure relative error has no meaning.
+    * with GELU (or when the reference does not say): rtol * (|y_ref| + mag). The bound is absolute in
+      |z| on purpose: in GELU's negative tail y = z Phi(z) is many orders below |z|, and the kernel's
+      Phi carries an absolute error (1.5e-7 for the erf form), so the error is a fraction of |z|, not
+      of |y|."""
     Y = np.asarray(Y, np.float64)
-    tol = rtol * (np.abs(ref["Y"]) + ref["mag"])
+    if ref.get("act", None) == 0:
+        tol = rtol * np.abs(ref["Y"]) + 4.0 * 2.0 ** -24 * ref["mag"]
+    else:
+        tol = rtol * (np.abs(ref["Y"]) + ref["mag"])
     err = np.abs(Y - ref["Y"])
     bad = err > tol
     assert not bad.any(), (f"{what}: {bad.sum()} of {bad.size} outside rtol={rtol}; worst ratio "

@@ -124,7 +124,7 @@ def test_host_argument_validation(gpu):
     Xb = gpu.torch.zeros((4, 32), dtype=gpu.torch.bfloat16, device=gpu.dev)
     Y = gpu.torch.zeros((4, 8), device=gpu.dev)
     assert L.qlinear_bf16(h, p(Xb), p(pos), 4, 24, 8, p(Wq), p(s_w), p(s_tok), 1, None, None, 8, 0, 0, p(Y), None) == -3
-    assert L.qlinear_bf16(h, p(Xb), p(pos), 4, 32, 8, p(Wq), p(s_w), p(s_tok), 1, None, None, 8, 3, 0, p(Y), None) == -4
+    assert L.qlinear_bf16(h, p(Xb), p(pos), 4, 32, 8, p(Wq), p(s_w), p(s_tok), 1, None, None, 8, 4, 0, p(Y), None) == -4
     gpu.torch.cuda.synchronize()
     assert gpu.ctx.stwq_device_status() == 0
 
@@ -541,6 +541,116 @@ def test_graph_replay_matches_the_oracle(gpu, cfg, idx):
     assert_close(Y.float().cpu().numpy(), ref, RTOL["bf16"], f"graph replay cfg{cfg} {L.name}")
 
 
+@pytest.mark.parametrize("option,value", [("TILE_N", 128), ("TILE_N", 256), ("VARIANT", 1), ("VARIANT", 2), ("VARIANT", 5)])
+def test_forced_kernel_variants_match_the_oracle(gpu, option, value):
+    """Every variant the options name computes the same layer: tile width 128 / 256 of the
+    CTA-pair GEMM, staged TMA stores / stores from registers, ordinary instead of programmatic
+    dependent launches. Exact accumulators, outputs in tolerance, on a ragged multi-tile shape."""
+    opt = {"TILE_N": gpu.B.OPT_TILE_N, "VARIANT": gpu.B.OPT_VARIANT}[option]
+    L = wl.scaled(wl.config_layers(1)[0], K=656, N=1032, P=37, batch=21, bits=8, act=1)
+    par = prepare(L, samples=4, gps_n=64)
+    X, pos = wl.activations(L), wl.positions(L)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 1)
+    ref0 = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 0)
+    gpu.ctx.stwq_set_option(opt, value)
+    try:
+        np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", path=1), ref["acc"])
+        for out in ("fp32", "bf16"):
+            assert_close(_run_qlinear(gpu, L, par, X, pos, out, path=1), ref, RTOL[out], f"{option}={value} {out}")
+            assert_close(_run_qlinear(gpu, L, par, X, pos, out, act=0, path=1), ref0, RTOL[out], f"{option}={value} {out}")
+    finally:
+        gpu.ctx.stwq_set_option(opt, 0)
+
+
+def test_options_reject_values_they_do_not_name(gpu):
+    L, h = gpu.ctx.lib, gpu.ctx.handle
+    for opt, bad in ((gpu.B.OPT_TILE_N, 64), (gpu.B.OPT_TILE_N, 192), (gpu.B.OPT_VARIANT, 3), (gpu.B.OPT_VARIANT, 9),
+                     (gpu.B.OPT_KSPLIT, -2), (gpu.B.OPT_KSPLIT, 65), (gpu.B.OPT_GEMM_PATH, 4),
+                     (gpu.B.OPT_WAIT_LIMIT_MS, 0)):
+        assert L.stwq_set_option(h, opt, bad) == -2
+    for opt in (gpu.B.OPT_TILE_N, gpu.B.OPT_VARIANT, gpu.B.OPT_KSPLIT, gpu.B.OPT_GEMM_PATH):
+        assert L.stwq_set_option(h, opt, 0) == 0
+
+
+# ----------------------------------------------------------------------------- failure handling
+def test_bounded_wait_expires_and_the_context_stays_usable(gpu):
+    """The wait every GEMM kernel uses gives up after the limit, the kernel reports the timeout and
+    returns; the status is read once and clears; the next call computes correctly. The wait that
+    runs out belongs to a one-CTA self-test kernel (a barrier nothing arrives at), never to a
+    kernel that moves data."""
+    torch = gpu.torch
+    waited = torch.zeros(1, dtype=torch.int64, device=gpu.dev)
+    gpu.ctx.stwq_set_option(gpu.B.OPT_WAIT_LIMIT_MS, 2)
+    try:
+        gpu.ctx.stwq_selftest_wait_expiry(waited)
+        assert gpu.ctx.stwq_device_status() == -7             # STWQ_ERR_DEVICE_TIMEOUT
+        assert gpu.ctx.stwq_device_status() == 0              # reading clears it
+        ns = int(waited.item())
+        assert 2_000_000 <= ns < 200_000_000, ns               # it waited for the limit, not forever
+    finally:
+        gpu.ctx.stwq_set_option(gpu.B.OPT_WAIT_LIMIT_MS, 2000)
+    M, N, K = 300, 520, 144
+    Xq = rng.integers(-128, 128, (M, K)).astype(np.int8)
+    Wq = rng.integers(-128, 128, (N, K)).astype(np.int8)
+    Y = _out_tensor(gpu, M, N, "int32")
+    gpu.ctx.qlinear_q(gpu.T(Xq), None, gpu.T(Wq), None, None, None, 0, gpu.B.OUT_INT32, Y)
+    assert gpu.ctx.stwq_device_status() == 0
+    np.testing.assert_array_equal(Y.cpu().numpy(), oracle.igemm(Xq, Wq))
+
+
+def test_workspace_growth_is_refused_during_capture(gpu):
+    """A call that would have to allocate workspace while its stream is being captured returns
+    STWQ_ERR_CAPTURE and enqueues nothing; after stwq_reserve_layer the same capture succeeds, and
+    the workspace generation tells a holder of older graphs that buffers moved."""
+    torch = gpu.torch
+    import paper_2601_21238_b200 as pk
+    ctx = pk.Context(0)
+    try:
+        M, K, N, P = 384, 256, 512, 8
+        X = torch.randn(M, K, device=gpu.dev)
+        pos = torch.zeros(M, dtype=torch.int32, device=gpu.dev)
+        Wq = torch.randint(-128, 128, (N, K), dtype=torch.int8, device=gpu.dev)
+        s_w = torch.full((N,), 1e-3, device=gpu.dev)
+        s_tok = torch.full((P,), 0.05, device=gpu.dev)
+        Y = torch.zeros((M, N), device=gpu.dev)
+        call = lambda: ctx.qlinear(X, pos, Wq, s_w, s_tok, None, None, 8, 0, gpu.B.OUT_F32, Y)
+        gen0 = ctx.stwq_workspace_generation()
+        side = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                with pytest.raises(pk.StwqError) as ei:
+                    call()                                   # fresh context: no workspace yet
+            assert ei.value.code == -11                       # STWQ_ERR_CAPTURE
+        torch.cuda.synchronize()
+        assert ctx.stwq_workspace_generation() == gen0        # nothing was allocated
+        ctx.stwq_reserve_layer(M, K, N, P)
+        gen1 = ctx.stwq_workspace_generation()
+        assert gen1 > gen0
+        with torch.cuda.stream(side):
+            g2 = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g2, stream=side):
+                call()
+            g2.replay()
+        torch.cuda.synchronize()
+        assert ctx.stwq_device_status() == 0
+        assert ctx.stwq_workspace_generation() == gen1        # the capture and the replay allocated nothing
+        want = torch.zeros((M, N), device=gpu.dev)
+        ctx.qlinear(X, pos, Wq, s_w, s_tok, None, None, 8, 0, gpu.B.OUT_F32, want)
+        torch.cuda.synchronize()
+        assert torch.equal(Y, want)
+        # a larger problem moves the buffer: the generation changes, which is the cue to re-capture
+        X2 = torch.randn(4 * M, K, device=gpu.dev)
+        pos2 = torch.zeros(4 * M, dtype=torch.int32, device=gpu.dev)
+        Y2 = torch.zeros((4 * M, N), device=gpu.dev)
+        ctx.qlinear(X2, pos2, Wq, s_w, s_tok, None, None, 8, 0, gpu.B.OUT_F32, Y2)
+        torch.cuda.synchronize()
+        assert ctx.stwq_workspace_generation() > gen1
+    finally:
+        ctx.close()
+
+
 # ----------------------------------------------------------------------------- dynamic token-wise baseline
 @pytest.mark.parametrize("bits", [8, 6])
 @pytest.mark.parametrize("shape", [(1, 16), (37, 1040), (300, 2048), (64, 5120), (9, 8192)])
@@ -584,18 +694,21 @@ def test_qlinear_dtwq_matches_the_oracle(gpu, M):
 
 
 # ----------------------------------------------------------------------------- chained layers
-@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("act", [0, 1, 2, 3])
 @pytest.mark.parametrize("bits_next", [8, 6])
 @pytest.mark.parametrize("shape", [(333, 400, 336), (1500, 1024, 1024), (77, 48, 32), (700, 272, 1040)])
 def test_chained_output_codes(gpu, shape, bits_next, act):
     """qlinear_chain: the epilogue applies the next layer's static quantizer. Without activation
-    the codes are bit-exact. With GELU the kernel's short form moves y by at most 6e-4 |z|, so a
-    code may differ by one, and only where the oracle's pre-round value lies that close to a tie."""
+    the codes are bit-exact. With GELU (erf or tanh form) the activation is evaluated to fp32
+    accuracy, and a code may differ from the oracle's (which rounds the exact activation to fp32)
+    only where the oracle's pre-round value sits within fp32 noise of a rounding tie. The short
+    GELU (act 3, asked for by name) moves y by up to 6e-4 |z| and is held to that."""
     M0, K, N = shape
-    L = wl.scaled(wl.config_layers(2)[2], batch=3, P=680, K=K, N=N, act=act)
+    ref_act = 2 if act == 3 else act                      # the short form approximates the tanh form
+    L = wl.scaled(wl.config_layers(2)[2], batch=3, P=680, K=K, N=N, act=ref_act)
     par = prepare(L, samples=4, gps_n=64)
     X, pos = wl.activations(L)[:M0], wl.positions(L)[:M0]
-    first = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, act)
+    first = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, ref_act)
     s_chn = rng.uniform(0.5, 2, N).astype(np.float32)
     # next-layer scales sized so that the codes use the range: y / (s_ch s_tok) of order 30
     typical = np.maximum(np.abs(first["Y"]).mean(axis=1), 1e-3)
@@ -603,7 +716,7 @@ def test_chained_output_codes(gpu, shape, bits_next, act):
     for p_ in range(L.P):
         sel = pos == p_
         s_tokn[p_] = np.float32(typical[sel].mean() / 20) if sel.any() else np.float32(1)
-    ref = oracle.chain_codes(first["acc"], pos, par["s_tok"], par["s_w"], par["bias"], act, s_chn, s_tokn, bits_next)
+    ref = oracle.chain_codes(first["acc"], pos, par["s_tok"], par["s_w"], par["bias"], ref_act, s_chn, s_tokn, bits_next)
     d = {k: gpu.T(par[k]) for k in ("Wq", "s_w", "s_tok", "s_ch", "bias")}
     out = gpu.torch.full((M0, N), 99, dtype=gpu.torch.int8, device=gpu.dev)
     gpu.ctx.qlinear_chain(gpu.T(X), gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["s_ch"], d["bias"], 8, act,
@@ -617,15 +730,45 @@ def test_chained_output_codes(gpu, shape, bits_next, act):
         diff = got != want
         assert np.abs(got - want).max() <= 1
         u = ref["u"].astype(np.float64)
-        slack = 1e-3 * ref["zmag"].astype(np.float64) + 1e-3
+        if act == 3:
+            slack = 1e-3 * ref["zmag"].astype(np.float64) + 1e-3
+            limit = 0.05
+        else:
+            # fp32 noise on u, plus the activation's own error carried to u: at most 3e-7 |z| on y
+            # (the erf form's fitted polynomial 4e-8, its fp32 evaluation 5e-8, the hardware exp2
+            # 2^-22 of Phi <= 1/2; the tanh form's exp2 / reciprocal are closer)
+            slack = 8e-6 * np.maximum(1.0, np.abs(u)) + 1e-6 + 3e-7 * ref["zmag"].astype(np.float64)
+            limit = 2e-3
         assert (np.abs(u - np.floor(u) - 0.5)[diff] <= slack[diff]).all()
-        assert diff.mean() < 0.05
+        assert diff.mean() < limit
+        print(f"chained codes act={act} bits_next={bits_next} {shape}: {diff.sum()} of {diff.size} differ by one")
     assert np.abs(got).max() > 2 ** (bits_next - 1) // 2       # the range is really used
     # the same from codes already held
     out2 = gpu.torch.full((M0, N), 99, dtype=gpu.torch.int8, device=gpu.dev)
     gpu.ctx.qlinear_chain_q(gpu.T(first["Xq"]), gpu.T(pos), d["Wq"], d["s_w"], d["s_tok"], d["bias"], act,
                             gpu.T(s_chn), gpu.T(s_tokn), bits_next, out2)
     assert gpu.torch.equal(out, out2)
+
+
+@pytest.mark.parametrize("out", ["fp32", "bf16"])
+@pytest.mark.parametrize("shape", [(333, 400, 328), (200, 2048, 512)])
+def test_short_gelu_is_the_tanh_form_within_its_stated_error(gpu, shape, out):
+    """STWQ_ACT_GELU_FAST: within 6e-4 |z| (+ output rounding) of the tanh form, on the tiled and
+    the few-row route; inside the bf16 tolerance of either GELU form."""
+    M, K, N = shape
+    L = wl.scaled(wl.config_layers(1)[0], K=K, N=N, P=37, batch=1, bits=8, act=2)
+    par = prepare(L, samples=4, gps_n=64)
+    X = (rng.standard_normal((M, K)) * 2).astype(np.float32)
+    pos = rng.integers(0, L.P, M).astype(np.int32)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 2)
+    ref_erf = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 1)
+    Y = _run_qlinear(gpu, L, par, X, pos, out, act=gpu.B.ACT_GELU_FAST)
+    zmag = ref["mag"]
+    rounding = 2.0 ** -8 if out == "bf16" else 2.0 ** -22
+    assert (np.abs(Y - ref["Y"]) <= 6e-4 * zmag + rounding * np.abs(ref["Y"]) + 1e-30).all()
+    if out == "bf16":
+        assert_close(Y, ref, RTOL["bf16"], "short GELU against the tanh form")
+        assert_close(Y, ref_erf, RTOL["bf16"], "short GELU against the erf form")
 
 
 @pytest.mark.parametrize("bits", [8, 6])

@@ -576,3 +576,47 @@ def test_asym_activation_codes_and_its_advantage_on_one_sided_data():
     big[1, 1] = -1e9
     q2, _ = oracle.quantize_asym(big, pos, None, s_tok, z_tok, 8)
     assert q2[0, 0] == 127 and q2[1, 1] == -128
+
+
+# ----------------------------------------------------------------------------- packed 4-bit weight codes
+def test_pack4_is_a_bijection_on_all_256_code_pairs_and_matches_hand_worked_bytes():
+    """Two signed 4-bit codes per byte, even channel in the low nibble. Exhaustive over the 16 x 16
+    code pairs: every pair maps to a distinct byte, unpacking returns the pair, and all 256 bytes
+    occur. Hand-worked cases: (0,0) -> 0x00, (1,0) -> 0x01, (0,1) -> 0x10, (-1,-1) -> 0xFF,
+    (-8,7) -> 0x78, (7,-8) -> 0x87, (3,-2) -> 0xE3."""
+    pairs = np.array([(a, b) for a in range(-8, 8) for b in range(-8, 8)], np.int8)
+    packed = oracle.pack4(pairs)
+    assert packed.shape == (256, 1) and len(set(packed[:, 0].tolist())) == 256
+    np.testing.assert_array_equal(oracle.unpack4(packed), pairs)
+    every_byte = np.arange(256, dtype=np.uint8)[:, None]
+    np.testing.assert_array_equal(oracle.pack4(oracle.unpack4(every_byte)), every_byte)
+    for (a, b), byte in {(0, 0): 0x00, (1, 0): 0x01, (0, 1): 0x10, (-1, -1): 0xFF, (-8, 7): 0x78, (7, -8): 0x87,
+                         (3, -2): 0xE3}.items():
+        assert oracle.pack4(np.array([[a, b]], np.int8))[0, 0] == byte
+        np.testing.assert_array_equal(oracle.unpack4(np.array([[byte]], np.uint8))[0], [a, b])
+    # the arithmetic meaning, independent of bit tricks: low nibble + 16 * high nibble, each nibble = code mod 16
+    np.testing.assert_array_equal(packed[:, 0].astype(int), (pairs[:, 0].astype(int) % 16) + 16 * (pairs[:, 1].astype(int) % 16))
+    with pytest.raises(ValueError):
+        oracle.pack4(np.array([[8, 0]], np.int8))
+    with pytest.raises(ValueError):
+        oracle.pack4(np.array([[0, -9]], np.int8))
+
+
+def test_packed_rows_keep_the_channel_order_and_the_4bit_fold_fits():
+    """A row of K codes packs to K/2 bytes in channel order; the 4-bit weight codes of gps_fold are in
+    range, so a folded matrix survives the round trip, and the integer GEMM on the unpacked codes is
+    the GEMM on the original ones."""
+    rng = np.random.default_rng(5)
+    N, K = 7, 48
+    W = (0.02 * rng.standard_normal((N, K))).astype(np.float32)
+    s_ch = rng.uniform(0.5, 2, K).astype(np.float32)
+    Wq, s_w = oracle.gps_fold(W, s_ch, 4)
+    assert Wq.min() >= -8 and Wq.max() <= 7 and np.abs(Wq).max(axis=1).min() >= 7
+    Wp = oracle.pack4(Wq)
+    assert Wp.shape == (N, K // 2)
+    for n in (0, N - 1):
+        for j in (0, 5, K // 2 - 1):
+            assert Wp[n, j] == (int(Wq[n, 2 * j]) % 16) + 16 * (int(Wq[n, 2 * j + 1]) % 16)
+    np.testing.assert_array_equal(oracle.unpack4(Wp), Wq)
+    Xq = rng.integers(-128, 128, (5, K)).astype(np.int8)
+    np.testing.assert_array_equal(oracle.igemm(Xq, oracle.unpack4(Wp)), Xq.astype(np.int64) @ Wq.astype(np.int64).T)
