@@ -86,12 +86,13 @@ int stwq_create(stwq_ctx** out, int device);
 void stwq_destroy(stwq_ctx* ctx);
 
 /*
- * Workspace. A context keeps four buffers: the int8 copy of X, per-row scratch (row scales of
+ * Workspace. A context keeps five buffers: the int8 copy of X, the int8 copy of packed 4-bit
+ * weights (qlinear_w4), per-row scratch (row scales of
  * qlinear_dtwq, row corrections of qlinear_asym, column statistics of gps_scales), calibration
  * histograms, and int32 partial sums for the calls that split K. Each is allocated on first use and
  * re-allocated (cudaFree + cudaMalloc, which synchronise the device) when a call needs more.
  *  - stwq_reserve sizes the first and third for an [M,K] activation and P positions;
- *    stwq_reserve_layer sizes all four for every call this header declares on an [M,K] x [N,K] layer
+ *    stwq_reserve_layer sizes all five for every call this header declares on an [M,K] x [N,K] layer
  *    with P positions. After either, calls within those sizes allocate nothing.
  *  - A call that would have to grow a buffer while its stream is being captured into a CUDA graph
  *    returns STWQ_ERR_CAPTURE and enqueues nothing (an allocation would invalidate the capture).
@@ -152,6 +153,25 @@ int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const floa
  */
 int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
              float* s_w, void* stream);
+
+/*
+ * 4-bit weights stored two per byte (the W4A8 setting of Appendix J, Table 11: 4-bit weights, 8-bit
+ * activations). The paper fixes the bit width, not a storage format; this one is the plain one:
+ *     byte[n, j] = (Wq[n, 2j] & 0xF) | ((Wq[n, 2j+1] & 0xF) << 4)
+ * i.e. two's complement nibbles, the even input channel in the low nibble, codes in [-8, 7], with
+ * Wq and s_w exactly those of gps_fold(bits = 4). A weight matrix then takes N K / 2 bytes of HBM.
+ *  - gps_fold_packed4: W [N,K] fp32 -> Wp [N, K/2] bytes, s_w [N]. K a multiple of 32.
+ *  - stwq_unpack4: Wp -> Wq [N,K] int8 (for callers that want the containers back).
+ *  - qlinear_w4: qlinear on packed weights: same arithmetic and results as qlinear on the unpacked
+ *    codes (the activations keep `bits` in {8, 6}). The codes are widened to int8 on the GPU before
+ *    the tensor cores read them; the widened copy lives in context workspace.
+ */
+int gps_fold_packed4(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, uint8_t* Wp, float* s_w,
+                     void* stream);
+int stwq_unpack4(stwq_ctx* ctx, const uint8_t* Wp, int N, int K, int8_t* Wq, void* stream);
+int qlinear_w4(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N, const uint8_t* Wp,
+               const float* s_w, const float* s_tok, int P, const float* s_ch, const float* bias, int bits, int act,
+               int out_dtype, void* Y, void* stream);
 
 /*
  * Activation quantization with static per-position scales (Eq. 1 on the left factor of

@@ -23,7 +23,8 @@ _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gp
             "qlinear", "qlinear_q", "stwq_device_status", "stwq_set_option", "stwq_launch_count",
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
             "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16", "stwq_reserve_layer",
-            "stwq_workspace_generation", "stwq_selftest_wait_expiry", "stwq_probe_int8_peak"]
+            "stwq_workspace_generation", "stwq_selftest_wait_expiry", "stwq_probe_int8_peak", "gps_fold_packed4", "stwq_unpack4",
+            "qlinear_w4"]
 
 _lib = None
 
@@ -65,6 +66,9 @@ def load_library():
     L.stwq_probe_int8_peak.argtypes = [vp, i32, i32, C.POINTER(i64), vp]
     L.stwq_calibrate.argtypes = [vp, vp, vp, i64, i32, i32, vp, i32, u32, vp, vp]
     L.gps_fold.argtypes = [vp, vp, i32, i32, vp, i32, vp, vp, vp]
+    L.gps_fold_packed4.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
+    L.stwq_unpack4.argtypes = [vp, vp, i32, i32, vp, vp]
+    L.qlinear_w4.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
     L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
@@ -98,7 +102,7 @@ def _p(t):
 
 
 ERR_NULL, ERR_DIM, ERR_ALIGN, ERR_BITS, ERR_CUDA = -1, -2, -3, -4, -6
-_F32, _BF16, _I8, _I32 = "torch.float32", "torch.bfloat16", "torch.int8", "torch.int32"
+_F32, _BF16, _I8, _I32, _U8 = "torch.float32", "torch.bfloat16", "torch.int8", "torch.int32", "torch.uint8"
 _OUT_DTYPES = {OUT_F32: _F32, OUT_BF16: _BF16, OUT_INT32: _I32}
 
 
@@ -238,6 +242,29 @@ class Context:
                    ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), False))
         self._check(self._L.gps_fold(self._h, _p(W), N, K, _p(s_ch), bits, _p(Wq), _p(s_w),
                                      self._stream(stream)), "gps_fold")
+
+    def gps_fold_packed4(self, W, s_ch, Wp, s_w, stream=None):
+        N, K = _mk(W, "W")
+        self._args("gps_fold_packed4", ("W", W, _F32, (N, K), False), ("s_ch", s_ch, _F32, (K,), True),
+                   ("Wp", Wp, _U8, (N, K // 2), False), ("s_w", s_w, _F32, (N,), False))
+        self._check(self._L.gps_fold_packed4(self._h, _p(W), N, K, _p(s_ch), _p(Wp), _p(s_w), self._stream(stream)),
+                    "gps_fold_packed4")
+
+    def stwq_unpack4(self, Wp, Wq, stream=None):
+        N, K = _mk(Wq, "Wq")
+        self._args("stwq_unpack4", ("Wp", Wp, _U8, (N, K // 2), False), ("Wq", Wq, _I8, (N, K), False))
+        self._check(self._L.stwq_unpack4(self._h, _p(Wp), N, K, _p(Wq), self._stream(stream)), "stwq_unpack4")
+
+    def qlinear_w4(self, X, pos_ids, Wp, s_w, s_tok, s_ch, bias, bits, act, out_dtype, Y, stream=None):
+        M, K = _mk(X)
+        N, _ = _mk(Wp, "Wp")
+        P = int(s_tok.numel()) if s_tok is not None else 1
+        self._args("qlinear_w4", ("X", X, _F32, (M, K), False), ("pos_ids", pos_ids, _I32, (M,), False),
+                   ("Wp", Wp, _U8, (N, K // 2), False), ("s_w", s_w, _F32, (N,), False), ("s_tok", s_tok, _F32, (P,), False),
+                   ("s_ch", s_ch, _F32, (K,), True), ("bias", bias, _F32, (N,), True),
+                   ("Y", Y, _out_dtype("qlinear_w4", out_dtype), (M, N), False))
+        self._check(self._L.qlinear_w4(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wp), _p(s_w), _p(s_tok), P, _p(s_ch),
+                                       _p(bias), bits, act, out_dtype, _p(Y), self._stream(stream)), "qlinear_w4")
 
     def _quantize_specs(self, X, x_dtype, pos_ids, s_ch, s_tok, Xq):
         M, K = _mk(X)

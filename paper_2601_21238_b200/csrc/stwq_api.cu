@@ -169,6 +169,7 @@ void stwq_destroy(stwq_ctx* ctx)
     if (ctx->ws_cal) cudaFree(ctx->ws_cal);
     if (ctx->ws_dec) cudaFree(ctx->ws_dec);
     if (ctx->ws_dyn) cudaFree(ctx->ws_dyn);
+    if (ctx->ws_w4) cudaFree(ctx->ws_w4);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }
@@ -195,6 +196,9 @@ int stwq_reserve_layer(stwq_ctx* ctx, int64_t M, int K, int N, int P)
     size_t dyn = (size_t)M * 8;
     if (stwq_gps_ws_bytes(K, N) > dyn) dyn = stwq_gps_ws_bytes(K, N);
     if (rc == STWQ_OK) rc = ensure_dyn(ctx, dyn, nullptr);
+    // int8 copy of packed 4-bit weights (qlinear_w4)
+    if (rc == STWQ_OK)
+        rc = stwq_ensure_ws(ctx, reinterpret_cast<void**>(&ctx->ws_w4), &ctx->ws_w4_bytes, (size_t)N * (size_t)K, nullptr, 0);
     // int32 partial sums of the few-row path when it splits K
     if (rc == STWQ_OK && M <= 256) {
         const size_t split = stwq_decode_split_bytes(ctx, K, N);
@@ -270,6 +274,50 @@ int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int
     if (check_wbits(bits) != STWQ_OK) return STWQ_ERR_BITS;
     DeviceGuard g(ctx->device);
     return stwq_launch_fold(ctx, W, N, K, s_ch, bits, Wq, s_w, static_cast<cudaStream_t>(stream));
+}
+
+int gps_fold_packed4(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, uint8_t* Wp, float* s_w,
+                     void* stream)
+{
+    if (!ctx || !W || !Wp || !s_w) return STWQ_ERR_NULL;
+    if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
+    if ((K & 31) != 0 || !aligned16(Wp)) return STWQ_ERR_ALIGN;     // rows of K / 2 bytes stay 16-byte aligned
+    DeviceGuard g(ctx->device);
+    return stwq_launch_fold_packed4(ctx, W, N, K, s_ch, Wp, s_w, static_cast<cudaStream_t>(stream));
+}
+
+int stwq_unpack4(stwq_ctx* ctx, const uint8_t* Wp, int N, int K, int8_t* Wq, void* stream)
+{
+    if (!ctx || !Wp || !Wq) return STWQ_ERR_NULL;
+    if (N <= 0 || K <= 0) return STWQ_ERR_DIM;
+    if ((K & 31) != 0 || !aligned16(Wp) || !aligned16(Wq)) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    return stwq_launch_unpack4(ctx, Wp, (int64_t)N * (K / 2), Wq, static_cast<cudaStream_t>(stream));
+}
+
+int qlinear_w4(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K, int N, const uint8_t* Wp,
+               const float* s_w, const float* s_tok, int P, const float* s_ch, const float* bias, int bits, int act,
+               int out_dtype, void* Y, void* stream)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (!pos_ids || !s_tok || !s_w) return STWQ_ERR_NULL;
+    int rc = check_gemm_args(X, pos_ids, M, K, N, reinterpret_cast<const int8_t*>(Wp), s_w, s_tok, P, act, out_dtype, Y);
+    if (rc != STWQ_OK) return rc;
+    if (check_bits(bits) != STWQ_OK) return STWQ_ERR_BITS;
+    if ((K & 31) != 0) return STWQ_ERR_ALIGN;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    rc = ensure_xq(ctx, (size_t)M * (size_t)K, st);
+    if (rc == STWQ_OK)
+        rc = stwq_ensure_ws(ctx, reinterpret_cast<void**>(&ctx->ws_w4), &ctx->ws_w4_bytes, (size_t)N * (size_t)K, st, 0);
+    if (rc != STWQ_OK) return rc;
+    // the weights travel through HBM as half a byte per code; the tensor cores take int8, so the
+    // codes are widened into workspace first (N K bytes written once, then read from L2 / HBM by the GEMM)
+    rc = stwq_launch_unpack4(ctx, Wp, (int64_t)N * (K / 2), ctx->ws_w4, st);
+    if (rc != STWQ_OK) return rc;
+    rc = stwq_launch_quantize(ctx, X, pos_ids, M, K, s_ch, s_tok, P, bits, ctx->ws_xq, false, st);
+    if (rc != STWQ_OK) return rc;
+    return run_gemm(ctx, ctx->ws_xq, pos_ids, M, K, N, ctx->ws_w4, s_w, s_tok, P, bias, act, out_dtype, Y, ctx->debug != 5, st);
 }
 
 int stwq_quantize(stwq_ctx* ctx, const float* X, const int32_t* pos_ids, int64_t M, int K,

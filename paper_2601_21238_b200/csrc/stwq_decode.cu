@@ -2,18 +2,22 @@
 // decode step in which a whole batch advances one token position (Section 2: "one token at a
 // time"). The arithmetic is that of qgemm2 (int8 x int8 -> int32 on the tensor cores, then the
 // Appendix A.1 dequantizer with bias and activation); what differs is the decomposition. With so
-// few rows the weights dominate the traffic (Wq is read once, 16.8 MB at the decode shapes), so
-// the aim is to have every SM pull its share of Wq from HBM from the first cycle:
+// few rows the weights dominate the traffic (Wq is read once, 16.8 MB at the decode shapes):
 //
 //   * one CTA pair (tcgen05 cta_group::2) per work item; the pair's 256 accumulator rows cover
 //     all of M, so Wq is staged exactly once on the whole GPU;
 //   * a work item is a 128-column slice of N and, when N alone does not give one item per pair,
 //     one of `ksplit` ranges of K (split-K);
-//   * the two operands have separate rings. The Wq ring holds 16 k-blocks (128 KB per pair
-//     member), normally the item's whole slab, and its loads are issued before anything else.
-//     The kernel can be launched as a programmatic dependent of the quantize kernel: it then
-//     starts while that kernel still runs, streams Wq, and only waits for the codes of X
-//     (griddepcontrol.wait) before the first load of Xq, which comes from L2 through a 4-stage ring;
+//   * the two operands have separate 8-stage rings. Each ring has its own producer warp, and the
+//     lanes of a producer warp issue the loads of different stages in the same instruction: one
+//     thread alone needs about 160 ns per request (wait, expect, issue are a dependent chain),
+//     2.6 us for a 16-k-block slab before its last byte is even asked for. The kernel can be
+//     launched as a programmatic dependent of the quantize kernel: it then starts while that
+//     kernel still runs, streams Wq, and only waits for the codes of X (griddepcontrol.wait)
+//     before the first load of Xq, which comes from L2;
+//   * two threads (in two warps) issue the MMAs, each into its own accumulator, because one thread
+//     cannot issue tcgen05.mma faster than one per ~61 ns whatever the instruction's width, and a
+//     256 x 128 x 32 instruction occupies the pipe for only 33 ns; the epilogue adds the accumulators;
 //   * split-K partials are exact int32 sums. Every epilogue warp writes its 32 x 64 piece of the
 //     pair's partial accumulator to scratch memory (lane-interleaved, so that each instruction
 //     moves 512 contiguous bytes) and then bumps a counter that belongs to that piece; the warp
@@ -39,9 +43,11 @@ constexpr int kBM = 128;       // rows per CTA (256 per pair)
 constexpr int kBK = 128;       // bytes of K per k-block
 constexpr int kBN = 128;       // columns per work item
 constexpr int kEpi = 8;        // epilogue warps per CTA: 4 lane quarters x 2 column halves
-constexpr int kStagesA = 4;    // Xq ring
-constexpr int kStagesB = 16;   // Wq ring
-constexpr int kFirstEpiWarp = 3;
+constexpr int kStagesA = 8;    // Xq ring (128 KB; doubles as output staging)
+constexpr int kStagesB = 8;    // Wq ring (64 KB)
+constexpr int kIssuers = 2;            // MMA-issuing threads, one accumulator each (4 measured no faster: with 2 the
+                                       // loop already runs at what L2 delivers, and every accumulator costs the epilogue a read)
+constexpr int kFirstEpiWarp = 2 + kIssuers;   // warps: 0 Wq producer, 1 Xq producer, 2.. MMA issuers, then the epilogue
 constexpr int kThreads = 32 * (kFirstEpiWarp + kEpi);
 constexpr int kPieceInts = 2 * 32 * 32;   // one warp's piece of a partial: 32 rows x 64 columns
 
@@ -71,6 +77,7 @@ struct SmemDec {
     static constexpr int kDynamic = kTotal + 1024;
     static_assert(kDynamic <= 227 * 1024, "shared memory budget");
     static_assert(kStagesA * kABytes >= kEpi * 8192, "the Xq ring doubles as output staging");
+    static_assert(kIssuers * kBN <= 512 && kStagesA % kIssuers == 0 && kStagesB % kIssuers == 0, "issuers own fixed ring stages");
 };
 
 __device__ __forceinline__ uint4 ld_cg_v4(const void* p)
@@ -122,78 +129,94 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             mbar_init(bar_full_b(s), 1);
             mbar_init(bar_empty_b(s), 1);
         }
-        mbar_init(bar_tfull, 1);
+        mbar_init(bar_tfull, kIssuers);                  // one commit from each MMA issuer
         *abort_flag = 0u;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
+    __syncthreads();
+    // The cluster barrier is split: arrive now, wait just before the first access to the peer
+    // (a load that signals the leader's barrier, a commit that arrives in both CTAs). Tensor memory
+    // is allocated in between, and the producers do not wait for it at all.
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
     if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"(kBN)
+                     "r"(kIssuers * kBN)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        tc_fence_before();
     }
-    tc_fence_before();
-    __syncthreads();
-    cluster_sync_all();                                  // barriers of both CTAs are initialised
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");        // barriers of both CTAs are initialised
     const unsigned long long limit = p.wait_limit_ns;
+    uint32_t tmem_base = 0;
+    if (warp >= 2) {
+        // the tensor-memory address, published by warp 2, is needed by warp 2 and the epilogue warps only
+        asm volatile("bar.sync 1, %0;" ::"r"(kThreads - 64) : "memory");
+        tc_fence_after();
+        tmem_base = *tmem_slot;
+    }
 
     if (warp == 0) {
         // ------------------------------------------------------------------ Wq producer
-        if (lane == 0) {
+        // Sixteen lanes, one per stage of the Wq ring, issue their loads in the same instruction:
+        // a single thread needs about 160 ns per request (wait, expect, issue form a dependent
+        // chain), which for the 16 k-blocks of a slab is 2.6 us before the last byte is even asked for.
+        if (lane < kStagesB) {
             bool ok = true;
             const uint32_t full0 = mapa_u32(bar_full_b(0), 0);
             const int n0 = nt * kBN + (int)rank * (kBN / 2);
-            int it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const int s = it % kStagesB;
+            const int s = lane;
+            int it = lane;
+            for (; kb0 + it < kb1; it += kStagesB) {
                 const uint32_t ph = (uint32_t)(it / kStagesB) & 1u;
                 if (!mbar_wait(bar_empty_b(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
                 if (rank == 0) mbar_expect_tx(bar_full_b(s), 2 * L::kBBytes);
-                tma_load_2d_pair(base + L::kOffB + s * L::kBBytes, &tmB, kb * kBK, n0, full0 + 8u * s);
+                tma_load_2d_pair(base + L::kOffB + s * L::kBBytes, &tmB, (kb0 + it) * kBK, n0, full0 + 8u * s);
             }
-            if (!ok && rank == 0) {
-                const int first = it > kStagesB ? it - kStagesB : 0;
-                for (int j = first; j < it; ++j) {
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar_full_b(j % kStagesB), (uint32_t)(j / kStagesB) & 1u))
-                        if (globaltimer_ns() - t0 > limit) break;
-                }
+            ok = __all_sync((1u << kStagesB) - 1u, ok);
+            if (!ok && rank == 0 && it >= kStagesB) {     // giving up: this lane's last load may still be in flight
+                const int j = it - kStagesB;
+                const unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_full_b(s), (uint32_t)(j / kStagesB) & 1u))
+                    if (globaltimer_ns() - t0 > limit) break;
             }
         }
     } else if (warp == 1) {
         // ------------------------------------------------------------------ Xq producer
-        if (lane == 0) {
+        if (lane < kStagesA) {
             grid_dependency_wait();                      // the codes of X come from the previous kernel
             bool ok = true;
             const uint32_t full0 = mapa_u32(bar_full_a(0), 0);
             const int m0 = (int)rank * kBM;
-            int it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
-                const int s = it % kStagesA;
+            const int s = lane;
+            int it = lane;
+            for (; kb0 + it < kb1; it += kStagesA) {
                 const uint32_t ph = (uint32_t)(it / kStagesA) & 1u;
                 if (!mbar_wait(bar_empty_a(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
                 if (rank == 0) mbar_expect_tx(bar_full_a(s), 2 * L::kABytes);
-                tma_load_2d_pair(base + s * L::kABytes, &tmA, kb * kBK, m0, full0 + 8u * s);
+                tma_load_2d_pair(base + s * L::kABytes, &tmA, (kb0 + it) * kBK, m0, full0 + 8u * s);
             }
-            if (!ok && rank == 0) {
-                const int first = it > kStagesA ? it - kStagesA : 0;
-                for (int j = first; j < it; ++j) {
-                    const unsigned long long t0 = globaltimer_ns();
-                    while (!mbar_try_wait(bar_full_a(j % kStagesA), (uint32_t)(j / kStagesA) & 1u))
-                        if (globaltimer_ns() - t0 > limit) break;
-                }
+            ok = __all_sync((1u << kStagesA) - 1u, ok);
+            if (!ok && rank == 0 && it >= kStagesA) {
+                const int j = it - kStagesA;
+                const unsigned long long t0 = globaltimer_ns();
+                while (!mbar_try_wait(bar_full_a(s), (uint32_t)(j / kStagesA) & 1u))
+                    if (globaltimer_ns() - t0 > limit) break;
             }
         }
-    } else if (warp == 2) {
-        // ------------------------------------------------------------------ MMA issuer (leader)
+    } else if (warp < kFirstEpiWarp) {
+        // ------------------------------------------------------------------ MMA issuers (leader)
+        // One thread cannot issue tcgen05.mma faster than about one per 61 ns, whatever the
+        // instruction's shape, and a 256 x 128 x 32 instruction keeps the pipe busy for only 33 ns.
+        // So kIssuers threads issue, each in a warp of its own: issuer i takes the k-blocks i,
+        // i + kIssuers, ... into accumulator i (tensor-memory columns 128 i ..); the epilogue adds
+        // the accumulators (int32, exact). Each issuer releases the ring stages of its own k-blocks.
         if (lane == 0 && rank == 0) {
             constexpr uint32_t idesc = make_idesc_i8(2 * kBM, kBN);
+            const int who = warp - 2;
+            const uint32_t d_tmem = tmem_base + (uint32_t)(who * kBN);
             bool ok = true;
-            int it = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++it) {
+            for (int it = who; kb0 + it < kb1; it += kIssuers) {
                 const int sa = it % kStagesA, sb = it % kStagesB;
                 if (!mbar_wait(bar_full_b(sb), (uint32_t)(it / kStagesB) & 1u, abort_flag, limit)) { ok = false; break; }
                 if (!mbar_wait(bar_full_a(sa), (uint32_t)(it / kStagesA) & 1u, abort_flag, limit)) { ok = false; break; }
@@ -202,7 +225,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const uint64_t b_desc = make_smem_desc(base + L::kOffB + sb * L::kBBytes);
 #pragma unroll
                 for (int k = 0; k < kBK / 32; ++k)
-                    tc_mma_i8_pair(tmem_base, a_desc + 2u * k, b_desc + 2u * k, idesc, (it | k) != 0 ? 1u : 0u);
+                    tc_mma_i8_pair(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (it >= kIssuers || k != 0) ? 1u : 0u);
                 tc_commit_pair(bar_empty_a(sa));
                 tc_commit_pair(bar_empty_b(sb));
             }
@@ -237,18 +260,31 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         if (ok) {
             tc_fence_after();
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(sub * 64);
-            uint32_t r0[32], r1[32];                      // this row's 64 accumulators
-            tmem_ld32(taddr, r0);
-            tmem_ld32(taddr + 32u, r1);
-            tmem_ld_wait();
+            // This row's 64 accumulators are handled as two halves of 32 columns, one after the other.
+            // 32 columns of this row: the sum of the issuers' accumulators (accumulator i exists only
+            // if the item has more than i k-blocks)
+            const int n_acc = min(kb1 - kb0, kIssuers);
+            auto load_acc = [&](uint32_t addr, uint32_t (&r)[32]) {
+                tmem_ld32(addr, r);
+                tmem_ld_wait();
+                for (int a = 1; a < n_acc; ++a) {
+                    uint32_t r2[32];
+                    tmem_ld32(addr + (uint32_t)(a * kBN), r2);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) r[j] += r2[j];
+                }
+            };
             bool finish = true;
             if (p.ksplit > 1) {
                 // publish this warp's piece of the partial sum, then see who is last
                 int32_t* piece = p.partial + ((((size_t)nt * p.ksplit + ks) * 2 + rank) * kEpi + ew) * kPieceInts;
+#pragma unroll 1
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t r[32];
+                    load_acc(taddr + 32u * h, r);
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {
-                    st_global_v4(piece + ((size_t)g * 32 + lane) * 4, r0 + g * 4);
-                    st_global_v4(piece + ((size_t)(8 + g) * 32 + lane) * 4, r1 + g * 4);
+                    for (int g = 0; g < 8; ++g) st_global_v4(piece + ((size_t)(h * 8 + g) * 32 + lane) * 4, r + g * 4);
                 }
                 __threadfence();
                 __syncwarp();
@@ -260,37 +296,38 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 }
                 old = __shfl_sync(0xffffffffu, old, 0);
                 finish = (old == (uint32_t)p.ksplit - 1u);
-                if (finish) {
-                    __threadfence();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) { r0[j] = 0u; r1[j] = 0u; }
-#pragma unroll 2
-                    for (int s2 = 0; s2 < p.ksplit; ++s2) {
-                        const int32_t* src = p.partial + ((((size_t)nt * p.ksplit + s2) * 2 + rank) * kEpi + ew) * kPieceInts;
-#pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            const uint4 a = ld_cg_v4(src + ((size_t)g * 32 + lane) * 4);
-                            const uint4 b = ld_cg_v4(src + ((size_t)(8 + g) * 32 + lane) * 4);
-                            r0[g * 4 + 0] += a.x; r0[g * 4 + 1] += a.y; r0[g * 4 + 2] += a.z; r0[g * 4 + 3] += a.w;
-                            r1[g * 4 + 0] += b.x; r1[g * 4 + 1] += b.y; r1[g * 4 + 2] += b.z; r1[g * 4 + 3] += b.w;
-                        }
-                    }
-                }
+                if (finish) __threadfence();
             }
             if (finish) {
                 // 32 rows x 64 columns -> this warp's staging tiles (8 KB of the idle Xq ring): one
                 // 32 x 128-byte tile for bf16, two for fp32 / int32, 128-byte swizzled as TMA expects
                 const uint32_t stage = base + (uint32_t)ew * 8192u;
                 const uint64_t st2 = pack_f2(st, st);
-#pragma unroll
+#pragma unroll 1
                 for (int h = 0; h < 2; ++h) {             // two halves of 32 columns
-                    const uint32_t* r = h == 0 ? r0 : r1;
+                    uint32_t r[32];
+                    if (p.ksplit > 1) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) r[j] = 0u;
+                        for (int s2 = 0; s2 < p.ksplit; ++s2) {
+                            const int32_t* src = p.partial + ((((size_t)nt * p.ksplit + s2) * 2 + rank) * kEpi + ew) * kPieceInts;
+#pragma unroll
+                            for (int g = 0; g < 8; ++g) {
+                                const uint4 a = ld_cg_v4(src + ((size_t)(h * 8 + g) * 32 + lane) * 4);
+                                r[g * 4 + 0] += a.x; r[g * 4 + 1] += a.y; r[g * 4 + 2] += a.z; r[g * 4 + 3] += a.w;
+                            }
+                        }
+                    } else {
+                        load_acc(taddr + 32u * h, r);
+                    }
+                    const float* hsw = my_sw + h * 32;
+                    const float* hbi = my_bias + h * 32;
                     if (OUT == STWQ_OUT_BF16) {
                         uint32_t w[16];
 #pragma unroll
                         for (int j = 0; j < 32; j += 2) {
-                            const uint64_t sw = pack_f2(my_sw[h * 32 + j], my_sw[h * 32 + j + 1]);
-                            const uint64_t bi = pack_f2(my_bias[h * 32 + j], my_bias[h * 32 + j + 1]);
+                            const uint64_t sw = pack_f2(hsw[j], hsw[j + 1]);
+                            const uint64_t bi = pack_f2(hbi[j], hbi[j + 1]);
                             uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
                             z = apply_act_f2<ACT>(z);
                             float v0, v1;
@@ -303,27 +340,23 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                             st_shared_v4(stage + (uint32_t)lane * 128u + piece16 * 16u, w[4 * g], w[4 * g + 1], w[4 * g + 2], w[4 * g + 3]);
                         }
                     } else {
-                        uint32_t w[32];
-                        if (OUT == STWQ_OUT_INT32) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) w[j] = r[j];
-                        } else {
+                        if (OUT != STWQ_OUT_INT32) {
 #pragma unroll
                             for (int j = 0; j < 32; j += 2) {
-                                const uint64_t sw = pack_f2(my_sw[h * 32 + j], my_sw[h * 32 + j + 1]);
-                                const uint64_t bi = pack_f2(my_bias[h * 32 + j], my_bias[h * 32 + j + 1]);
+                                const uint64_t sw = pack_f2(hsw[j], hsw[j + 1]);
+                                const uint64_t bi = pack_f2(hbi[j], hbi[j + 1]);
                                 const uint64_t z = fma_f2(pack_f2((float)(int32_t)r[j], (float)(int32_t)r[j + 1]), mul_f2(st2, sw), bi);
                                 float v0, v1;
                                 unpack_f2(z, v0, v1);
-                                w[j] = __float_as_uint(apply_act<ACT>(v0));
-                                w[j + 1] = __float_as_uint(apply_act<ACT>(v1));
+                                r[j] = __float_as_uint(apply_act<ACT>(v0));
+                                r[j + 1] = __float_as_uint(apply_act<ACT>(v1));
                             }
                         }
 #pragma unroll
                         for (int g = 0; g < 8; ++g) {
                             const uint32_t piece16 = (uint32_t)(g ^ (lane & 7));
-                            st_shared_v4(stage + (uint32_t)h * 4096u + (uint32_t)lane * 128u + piece16 * 16u, w[4 * g], w[4 * g + 1],
-                                         w[4 * g + 2], w[4 * g + 3]);
+                            st_shared_v4(stage + (uint32_t)h * 4096u + (uint32_t)lane * 128u + piece16 * 16u, r[4 * g], r[4 * g + 1],
+                                         r[4 * g + 2], r[4 * g + 3]);
                         }
                     }
                 }
@@ -337,7 +370,8 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                         if (n0 + 32 < p.N) tma_store_2d(&tmY, stage + 4096u, n0 + 32, row0);
                     }
                     bulk_commit();
-                    bulk_wait0();                         // the stores have completed before the CTA may exit
+                    bulk_wait_read0();                    // the staging tiles have been read before the CTA may exit;
+                                                          // the writes themselves complete with the grid
                 }
             }
         }
@@ -351,7 +385,7 @@ decode_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     tc_fence_after();
     if (warp == 2) {
         __syncwarp();
-        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kBN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kIssuers * kBN) : "memory");
     }
 }
 

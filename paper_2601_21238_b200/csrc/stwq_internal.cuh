@@ -37,6 +37,8 @@ struct stwq_ctx {
     void* ws_dec;              // split-K workspace: arrival counters, then int32 partial sums
     size_t ws_dec_bytes;
     uint64_t configured_decode;
+    int8_t* ws_w4;             // workspace: int8 copy of packed 4-bit weights (qlinear_w4 on the tiled route)
+    size_t ws_w4_bytes;
     int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
     uint64_t ws_generation;    // bumped whenever a workspace buffer is (re)allocated
     int probe_configured;      // the peak-probe kernel has its shared-memory attribute set
@@ -73,6 +75,9 @@ int stwq_launch_quantize_asym(stwq_ctx* ctx, const float* X, const int32_t* pos_
 int stwq_launch_calibrate_asym(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids, int64_t rows, int K,
                                int P, const float* s_ch, int bits, uint32_t pct_ppm, float* s_tok, int32_t* z_tok,
                                cudaStream_t st);
+int stwq_launch_fold_packed4(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, uint8_t* Wp, float* s_w,
+                             cudaStream_t st);
+int stwq_launch_unpack4(stwq_ctx* ctx, const uint8_t* Wp, int64_t packed_bytes, int8_t* Wq, cudaStream_t st);
 int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits,
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);

@@ -171,10 +171,17 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
 
     if (warp == 0) {
         // ------------------------------------------------------------------ TMA producer
-        if (lane == 0) {
+        // Two lanes issue the two loads of a stage in the same instruction: lane 0 the Xq rows,
+        // lane 1 the Wq rows. One thread issuing both one after the other needs about 160 ns per
+        // request (wait, expect, issue form a dependent chain), i.e. more than the 256 x 256 x 128
+        // tile's 260 ns of tensor-pipe time per k-block; side by side the chain is paid once.
+        if (lane < 2) {
             uint32_t it = 0;
             bool ok = true;
             const uint32_t full0 = mapa_u32(bar_full(0), 0);     // leader's barriers
+            const CUtensorMap* my_map = lane == 0 ? &tmA : &tmB;
+            const uint32_t my_dst0 = lane == 0 ? base : base + L::kOffB;
+            const uint32_t my_stage_bytes = lane == 0 ? L::kABytes : L::kBBytes;
             // launched as a programmatic dependent of the quantize kernel: everything up to here
             // (barriers, tensor memory, cluster handshake) may have run while that kernel drained;
             // its codes are read only from here on
@@ -184,16 +191,17 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 const int tile = w.tile;
                 const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
                 const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
+                const int my_row0 = lane == 0 ? m0 : n0;
                 for (int kb = w.kb0; kb < w.kb1; ++kb, ++it) {
                     const int s = it % STAGES;
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
-                    if (rank == 0) mbar_expect_tx(bar_full(s), 2 * L::kStageBytes);
-                    tma_load_2d_pair(base + s * L::kABytes, &tmA, kb * kBK, m0, full0 + 8u * s);
-                    tma_load_2d_pair(base + L::kOffB + s * L::kBBytes, &tmB, kb * kBK, n0, full0 + 8u * s);
+                    if (rank == 0 && lane == 0) mbar_expect_tx(bar_full(s), 2 * L::kStageBytes);
+                    tma_load_2d_pair(my_dst0 + s * my_stage_bytes, my_map, kb * kBK, my_row0, full0 + 8u * s);
                 }
             }
-            if (!ok && rank == 0) {
+            ok = __all_sync(0x3u, ok);
+            if (!ok && rank == 0 && lane == 0) {
                 const uint32_t first = it > (uint32_t)STAGES ? it - STAGES : 0u;
                 for (uint32_t j = first; j < it; ++j) {
                     const unsigned long long t0 = globaltimer_ns();

@@ -354,6 +354,40 @@ def test_qlinear_w4a8(gpu, act):
         assert_close(_run_qlinear(gpu, L, par4, X, pos, out), ref, RTOL[out], f"W4A8 act{act} {out}")
 
 
+@pytest.mark.parametrize("M", [37, 256, 700])
+@pytest.mark.parametrize("act", [0, 1])
+def test_packed_int4_weights(gpu, M, act):
+    """W4A8 with the weights stored two codes per byte (Table 11's setting): the packed bytes and the
+    scales equal the oracle's 4-bit fold packed by the oracle; unpacking on the GPU returns the
+    codes; qlinear_w4 gives the accumulators and outputs of qlinear on the unpacked codes, on the
+    few-row route (M <= 256) and on the tiled one."""
+    torch = gpu.torch
+    L = wl.scaled(wl.config_layers(1)[0], K=544, N=584, P=37, batch=19, bits=8, act=act)
+    par = prepare(L, samples=8, gps_n=64)
+    Wq4, sw4 = oracle.gps_fold(par["W"], par["s_ch"], 4)
+    Wp_ref = oracle.pack4(Wq4)
+    Wp = torch.full((L.N, L.K // 2), 0x5A, dtype=torch.uint8, device=gpu.dev)
+    sw = torch.zeros(L.N, device=gpu.dev)
+    gpu.ctx.gps_fold_packed4(gpu.T(par["W"]), gpu.T(par["s_ch"]), Wp, sw)
+    np.testing.assert_array_equal(Wp.cpu().numpy(), Wp_ref)
+    np.testing.assert_array_equal(sw.cpu().numpy(), sw4)
+    back = torch.full((L.N, L.K), 99, dtype=torch.int8, device=gpu.dev)
+    gpu.ctx.stwq_unpack4(Wp, back)
+    np.testing.assert_array_equal(back.cpu().numpy(), Wq4)
+    X, pos = wl.activations(L)[:M], wl.positions(L)[:M]
+    ref = oracle.qlinear(X, pos, oracle.unpack4(Wp_ref), sw4, par["s_tok"], par["s_ch"], par["bias"], 8, act)
+    d = {k: gpu.T(par[k]) for k in ("s_tok", "s_ch", "bias")}
+    for out in ("int32", "fp32", "bf16"):
+        Y = _out_tensor(gpu, M, L.N, out)
+        gpu.ctx.qlinear_w4(gpu.T(X), gpu.T(pos), Wp, sw, d["s_tok"], d["s_ch"], d["bias"], 8, 0 if out == "int32" else act,
+                           _out_code(gpu, out), Y)
+        assert gpu.ctx.stwq_device_status() == 0
+        if out == "int32":
+            np.testing.assert_array_equal(Y.cpu().numpy(), ref["acc"])
+        else:
+            assert_close(Y.float().cpu().numpy(), ref, RTOL[out], f"qlinear_w4 M={M} {out}")
+
+
 @pytest.mark.parametrize("out", ["fp32", "bf16"])
 def test_config1_full(gpu, out):
     """Config 1: one W8A8 linear over the 680-token VAR pyramid, K = N = 1024, every element."""
