@@ -105,6 +105,8 @@ def summarise_ncu(args):
         rows.append({"kernel": r[col["Kernel Name"]][:60], "grid": r[col["Grid Size"]],
                      "dram_read": val("dram__bytes_read.sum"), "dram_write": val("dram__bytes_write.sum"),
                      "ns": float(r[col["gpu__time_duration.sum"]].replace(",", "")) if "gpu__time_duration.sum" in col else None})
+    if args.profile_launches:
+        rows = [rows[int(i)] for i in args.profile_launches.split(",")]
     if not rows:
         raise SystemExit("no launch of that kernel in the csv")
     rec = {}
@@ -835,6 +837,7 @@ def main():
     ap.add_argument("--ncu-raw-csv", help="raw ncu csv export to summarise into profiles/roofline_traffic.json")
     ap.add_argument("--profile-key", default="qgemm2_kernel/config3", help="kernel/workload the csv belongs to")
     ap.add_argument("--profile-note", default="")
+    ap.add_argument("--profile-launches", default="", help="comma-separated indices of the launches (of that kernel) to use")
     args = ap.parse_args()
     if args.ncu_raw_csv:
         summarise_ncu(args)
