@@ -728,6 +728,30 @@ def other_configs(ctx, pk, torch, dev, peaks, args):
         rows.append(row)
         del X, W1, W2, H, Hq, Y
     out["ffn_fc1_fc2_chained"] = rows
+    # quantized attention of a VAR-d16-shaped layer (batch 16 x 16 heads, 680 positions, head dimension 64):
+    # filling the quantized KV cache, then both attention matmuls on int8 codes with the softmax-and-quantize
+    # pass in between (block-causal masks of the real model are replaced by a plain causal one)
+    G, T, d, Tmax = 256, 680, 64, 688
+    Q = torch.randn(G, T, d, device=dev)
+    Kn = torch.randn(G, T, d, device=dev)
+    Vn = torch.randn(G, T, d, device=dev)
+    pos_q = torch.arange(T, dtype=torch.int32, device=dev)
+    s_q = torch.full((T,), 4.0 * 2 / 255, device=dev)
+    s_k = torch.full((T,), 4.0 * 2 / 255, device=dev)
+    s_kcol = s_k * (1.0 / d ** 0.5)
+    s_v = torch.full((d,), 4.0 * 2 / 255, device=dev)
+    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=dev)
+    Vt = torch.zeros((G, d, Tmax), dtype=torch.int8, device=dev)
+    O = torch.empty((G, T, d), dtype=torch.bfloat16, device=dev)
+    ctx.stwq_reserve_attention(G, T, T, d)
+    t_app = graph_us(lambda: ctx.kv_append(Kn, Vn, 0, s_k, s_v, 8, Kc, Vt), 1)
+    t_att = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    out["attention_var_d16"] = {"heads": G, "positions": T, "head_dim": d, "kv_append_us": round(t_app, 1),
+                                "qattention_us": round(t_att, 1),
+                                "matmul_tops": round(2 * 2.0 * G * T * T * d / t_att / 1e6, 1),
+                                "note": "Q K^T and P V as batched int8 GEMMs (unfused: scores and probability codes "
+                                        "pass through workspace); ops counted for the full T x T matrices"}
+    del Q, Kn, Vn, Kc, Vt, O
     ctx.check_device_status()
     return out
 

@@ -295,6 +295,44 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
                  const float* s_ch, const float* bias, int bits, int act, int out_dtype, void* Y, void* stream);
 
 /*
+ * Quantized attention matmuls and the quantized KV cache (Section 5: "all linear layers and matrix
+ * multiplications" run in 6 or 8 bits; Appendix C: "including the KV cache"). G = batch x heads
+ * independent heads, head dimension d, Tq queries, Tk keys, token positions in [0, P).
+ * Readings, since the paper names the operands but not their quantizers:
+ *  - queries and keys: the static per-position quantizer of stwq_quantize without channel scales,
+ *    codes = clamp(round(x * (1 / s[pos]))); in S = Q K^T the two scales leave the integer sum:
+ *        S[i,j] = acc_qk[i,j] * (s_q[pos_q[i]] * s_kcol[j]),   s_kcol[j] = s_k[pos of key j] * softmax scale
+ *  - values: one static scale per head channel, codes = clamp(round(x * (1 / s_v[c]))) (a scale that varied
+ *    along the keys could not leave the sum over keys);
+ *  - probabilities: Eq. 1 on the fixed range [0, 1]: delta_p = 1 / (2^b - 1), zero point 0, UNSIGNED codes
+ *    0 .. 2^b - 1, P = softmax over the visible keys of row i (fp32); causal != 0 hides key j from query
+ *    i unless j <= i + (Tk - Tq);
+ *  - O[i,c] = acc_pv[i,c] * (delta_p * s_v[c]),  acc_pv = sum_j Pcode[i,j] Vq[j,c]   (unsigned x signed, int32).
+ * Cache layout: Kc [G, Tmax, d] int8 (row = position), Vt [G, d, Tmax] int8 (the value codes transposed,
+ * column = position), so that both matmuls read operands whose contraction index is contiguous.
+ * d and Tmax multiples of 16, d <= 256.
+ *  - kv_append: quantize t_new new key / value rows per head (Knew, Vnew [G, t_new, d] fp32, at positions
+ *    pos0 .. pos0 + t_new - 1) into the caches. s_k [P], s_v [d].
+ *  - qattention: Q [G, Tq, d] fp32, pos_q [Tq] (shared by all heads), keys / values = the first Tk
+ *    positions of the caches, s_q [P], s_kcol [Tk], s_v [d]; O [G, Tq, d] fp32 or bf16. Quantizes Q, runs
+ *    both matmuls as batched integer GEMMs on the tensor cores with the softmax-and-quantize pass in
+ *    between. The scores (fp32) and the codes live in context workspace (stwq_reserve_attention sizes
+ *    it ahead of time; growth during stream capture is refused like everywhere else).
+ *  - qattn_softmax_quantize, qattn_pv: the second and third stage on their own (S [rows, ld] fp32 with
+ *    rows = G Tq and ld >= Tk a multiple of 16; Pq [G, Tq, Tk_pad] codes; STWQ_OUT_INT32 stores acc_pv).
+ */
+int kv_append(stwq_ctx* ctx, const float* Knew, const float* Vnew, int G, int t_new, int d, int pos0, int Tmax,
+              const float* s_k, const float* s_v, int P, int bits, int8_t* Kc, int8_t* Vt, void* stream);
+int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
+               const int8_t* Kc, const int8_t* Vt, const float* s_q, const float* s_kcol, const float* s_v, int P,
+               int bits, int causal, int out_dtype, void* O, void* stream);
+int stwq_reserve_attention(stwq_ctx* ctx, int G, int Tq, int Tk, int d);
+int qattn_softmax_quantize(stwq_ctx* ctx, const float* S, int64_t rows, int Tq, int Tk, int ld, int causal, int bits,
+                           uint8_t* Pq, void* stream);
+int qattn_pv(stwq_ctx* ctx, const uint8_t* Pq, int G, int Tq, int Tk_pad, int d, int Tmax, const int8_t* Vt,
+             const float* s_v, const float* delta_p, int out_dtype, void* O, void* stream);
+
+/*
  * qlinear without any allocation. (The paper has no counterpart to this call; it exists for the
  * way the library gets embedded.) qlinear needs a context, whose creation allocates, and keeps
  * the int8 copy of X in workspace that may be (re)allocated during a call. Hosts that cannot

@@ -87,6 +87,8 @@ def lib():
             L.orc_pack4.restype = C.c_int
             L.orc_pack4.argtypes = [bp, C.c_int64, C.POINTER(C.c_uint8)]
             L.orc_unpack4.argtypes = [C.POINTER(C.c_uint8), C.c_int64, bp]
+            L.orc_softmax_quantize.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint8), dp]
+            L.orc_igemm_u8s8.argtypes = [C.POINTER(C.c_uint8), bp, C.c_int, C.c_int, C.c_int, ip]
             L.orc_gps_gain.restype = C.c_double
             L.orc_gps_gain.argtypes = [C.c_double] * 4
             _lib = L
@@ -373,3 +375,46 @@ def unpack4(packed):
     out = np.empty(packed.shape[:-1] + (packed.shape[-1] * 2,), np.int8)
     lib().orc_unpack4(_ptr(packed, C.c_uint8), packed.size, _ptr(out, C.c_int8))
     return out
+
+
+def softmax_quantize(S, causal, bits):
+    """Row softmax of S [Tq, Tk] (fp32) then the probability quantizer (unsigned codes, delta = 1/(2^b - 1)).
+    Returns (codes uint8 [Tq, Tk], u float64: the value before rounding)."""
+    S = _f32(S)
+    Tq, Tk = S.shape
+    codes = np.empty((Tq, Tk), np.uint8)
+    u = np.empty((Tq, Tk), np.float64)
+    lib().orc_softmax_quantize(_ptr(S, C.c_float), Tq, Tk, int(bool(causal)), bits, _ptr(codes, C.c_uint8),
+                               _ptr(u, C.c_double))
+    return codes, u
+
+
+def igemm_u8s8(P, Vq):
+    """acc[i,c] = sum_j P[i,j] Vq[j,c]: unsigned probability codes [Tq, Tk] times signed value codes [Tk, C]."""
+    P = np.ascontiguousarray(P, np.uint8)
+    Vq = np.ascontiguousarray(Vq, np.int8)
+    Tq, Tk = P.shape
+    assert Vq.shape[0] == Tk
+    acc = np.empty((Tq, Vq.shape[1]), np.int32)
+    lib().orc_igemm_u8s8(_ptr(P, C.c_uint8), _ptr(Vq, C.c_int8), Tq, Tk, Vq.shape[1], _ptr(acc, C.c_int32))
+    return acc
+
+
+def qattention(Q, K, V, pos_q, pos_k, s_q, s_k, s_v, softmax_scale, bits, causal):
+    """One head of quantized attention, composed of the steps above (queries / keys with per-position
+    scales, values per channel, unsigned probability codes). Q [Tq,d], K, V [Tk,d]. Returns a dict with
+    every intermediate: Qq, Kq, Vq, acc_qk, S (fp32), Pq, u, acc_pv, O (float64), mag."""
+    ones = np.ones(1, np.float32)
+    Qq = quantize(Q, pos_q, None, s_q, bits)
+    Kq = quantize(K, pos_k, None, s_k, bits)
+    Vq = quantize(V, np.zeros(V.shape[0], np.int32), s_v, ones, bits)
+    acc_qk = igemm(Qq, Kq)
+    s_kcol = (_f32(s_k)[np.asarray(pos_k)] * np.float32(softmax_scale)).astype(np.float32)
+    S, _ = epilogue(acc_qk, pos_q, s_q, s_kcol, None, 0)
+    S32 = S.astype(np.float32)
+    Pq, u = softmax_quantize(S32, causal, bits)
+    acc_pv = igemm_u8s8(Pq, Vq)
+    delta_p = np.array([np.float32(1.0) / np.float32((1 << bits) - 1)], np.float32)
+    O, mag = epilogue(acc_pv, np.zeros(Q.shape[0], np.int32), delta_p, s_v, None, 0)
+    return {"Qq": Qq, "Kq": Kq, "Vq": Vq, "acc_qk": acc_qk, "s_kcol": s_kcol, "S": S32, "Pq": Pq, "u": u,
+            "acc_pv": acc_pv, "delta_p": delta_p, "O": O, "mag": mag, "act": 0}

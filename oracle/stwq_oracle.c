@@ -749,3 +749,66 @@ void orc_unpack4(const uint8_t* bytes, int64_t n_pairs, int8_t* codes)
         codes[2 * j + 1] = (int8_t)(hi >= 8 ? hi - 16 : hi);
     }
 }
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Quantized attention matmuls and the quantized KV cache (Section 5: 6- or 8-bit
+ * quantization of "all linear layers and matrix multiplications"; Appendix C: the
+ * KV cache is quantized too). The paper gives no quantizer for these operands
+ * beyond static, calibrated parameters (Appendix B; Section 4.2), so the reading
+ * is stated here and in the design notes:
+ *   - queries and keys: static scale per token position (the STWQ quantizer of
+ *     orc_quantize with s_ch = NULL); in S = Q K^T the scale of a query row and of
+ *     a key column factor out of the integer sum, so
+ *       S[i,j] = acc_qk[i,j] * (s_q[pos_i] * s_kcol[j]),  s_kcol[j] = s_k[pos_j] * softmax_scale
+ *     which is orc_epilogue with s_w = s_kcol, no bias, no activation;
+ *   - values: one static scale per head channel (orc_quantize with s_ch = s_v and
+ *     unit position scales): a scale that varied along the keys could not be taken
+ *     out of the sum over keys;
+ *   - attention probabilities: Eq. 1 on the fixed range [0, 1]: delta_p = 1/(2^b - 1),
+ *     zero point 0, UNSIGNED codes 0 .. 2^b - 1 (orc_softmax_quantize);
+ *   - O[i,c] = acc_pv[i,c] * (delta_p * s_v[c]) with acc_pv = sum_j P[i,j] Vq[j,c]
+ *     (orc_igemm_u8s8), again orc_epilogue (one "position" with scale delta_p).
+ */
+
+/*
+ * Row softmax followed by the quantizer of the probabilities. S is [Tq, Tk] fp32
+ * (the dequantized scores). causal != 0 masks key j for query i unless
+ * j <= i + (Tk - Tq) (the last query sees every key). Computed in double:
+ *   m_i = max_j S[i,j],  e_ij = exp(S[i,j] - m_i),  P_ij = e_ij / sum_j e_ij   (masked: 0)
+ *   u = P_ij * (2^b - 1),  code = clamp(round(u), 0, 2^b - 1)
+ * A row with every key masked gives zeros. u_out (optional) receives u.
+ */
+void orc_softmax_quantize(const float* S, int Tq, int Tk, int causal, int bits, uint8_t* codes, double* u_out)
+{
+    const double D = (double)((1 << bits) - 1);
+    for (int i = 0; i < Tq; ++i) {
+        const int last = causal ? i + (Tk - Tq) : Tk - 1;      /* last visible key */
+        double m = -INFINITY;
+        for (int j = 0; j < Tk && j <= last; ++j)
+            if ((double)S[(int64_t)i * Tk + j] > m) m = (double)S[(int64_t)i * Tk + j];
+        double sum = 0.0;
+        for (int j = 0; j < Tk && j <= last; ++j) sum += exp((double)S[(int64_t)i * Tk + j] - m);
+        for (int j = 0; j < Tk; ++j) {
+            double u = 0.0;
+            if (j <= last && sum > 0.0) u = exp((double)S[(int64_t)i * Tk + j] - m) / sum * D;
+            double r = nearbyint(u);
+            if (r < 0.0) r = 0.0;
+            if (r > D) r = D;
+            codes[(int64_t)i * Tk + j] = (uint8_t)r;
+            if (u_out) u_out[(int64_t)i * Tk + j] = u;
+        }
+    }
+}
+
+/* acc[i,c] = sum_j P[i,j] * Vq[j,c], P unsigned 8-bit codes, Vq signed; int32 exact
+ * (|acc| <= Tk * 255 * 128). P is [Tq, Tk], Vq is [Tk, C] (key-major, as the values are produced). */
+void orc_igemm_u8s8(const uint8_t* P, const int8_t* Vq, int Tq, int Tk, int C, int32_t* acc)
+{
+    for (int i = 0; i < Tq; ++i)
+        for (int c = 0; c < C; ++c) {
+            int32_t s = 0;
+            for (int j = 0; j < Tk; ++j) s += (int32_t)P[(int64_t)i * Tk + j] * (int32_t)Vq[(int64_t)j * C + c];
+            acc[(int64_t)i * C + c] = s;
+        }
+}

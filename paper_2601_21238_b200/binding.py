@@ -24,7 +24,7 @@ _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gp
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
             "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16", "stwq_reserve_layer",
             "stwq_workspace_generation", "stwq_selftest_wait_expiry", "stwq_probe_int8_peak", "gps_fold_packed4", "stwq_unpack4",
-            "qlinear_w4"]
+            "qlinear_w4", "kv_append", "qattention", "stwq_reserve_attention", "qattn_softmax_quantize", "qattn_pv"]
 
 _lib = None
 
@@ -69,6 +69,11 @@ def load_library():
     L.gps_fold_packed4.argtypes = [vp, vp, i32, i32, vp, vp, vp, vp]
     L.stwq_unpack4.argtypes = [vp, vp, i32, i32, vp, vp]
     L.qlinear_w4.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
+    L.kv_append.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
+    L.qattention.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, vp, vp]
+    L.stwq_reserve_attention.argtypes = [vp, i32, i32, i32, i32]
+    L.qattn_softmax_quantize.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp]
+    L.qattn_pv.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp]
     L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
@@ -265,6 +270,46 @@ class Context:
                    ("Y", Y, _out_dtype("qlinear_w4", out_dtype), (M, N), False))
         self._check(self._L.qlinear_w4(self._h, _p(X), _p(pos_ids), M, K, N, _p(Wp), _p(s_w), _p(s_tok), P, _p(s_ch),
                                        _p(bias), bits, act, out_dtype, _p(Y), self._stream(stream)), "qlinear_w4")
+
+    def kv_append(self, Knew, Vnew, pos0, s_k, s_v, bits, Kc, Vt, stream=None):
+        G, t_new, d = (int(v) for v in Knew.shape)
+        Tmax = int(Kc.shape[1])
+        P = int(s_k.numel())
+        self._args("kv_append", ("Knew", Knew, _F32, (G, t_new, d), False), ("Vnew", Vnew, _F32, (G, t_new, d), False),
+                   ("s_k", s_k, _F32, (P,), False), ("s_v", s_v, _F32, (d,), False), ("Kc", Kc, _I8, (G, Tmax, d), False),
+                   ("Vt", Vt, _I8, (G, d, Tmax), False))
+        self._check(self._L.kv_append(self._h, _p(Knew), _p(Vnew), G, t_new, d, pos0, Tmax, _p(s_k), _p(s_v), P, bits,
+                                      _p(Kc), _p(Vt), self._stream(stream)), "kv_append")
+
+    def qattention(self, Q, pos_q, Tk, Kc, Vt, s_q, s_kcol, s_v, bits, causal, out_dtype, O, stream=None):
+        G, Tq, d = (int(v) for v in Q.shape)
+        Tmax = int(Kc.shape[1])
+        P = int(s_q.numel())
+        self._args("qattention", ("Q", Q, _F32, (G, Tq, d), False), ("pos_q", pos_q, _I32, (Tq,), False),
+                   ("Kc", Kc, _I8, (G, Tmax, d), False), ("Vt", Vt, _I8, (G, d, Tmax), False), ("s_q", s_q, _F32, (P,), False),
+                   ("s_kcol", s_kcol, _F32, (Tk,), False), ("s_v", s_v, _F32, (d,), False),
+                   ("O", O, _out_dtype("qattention", out_dtype), (G, Tq, d), False))
+        self._check(self._L.qattention(self._h, _p(Q), _p(pos_q), G, Tq, Tk, d, Tmax, _p(Kc), _p(Vt), _p(s_q), _p(s_kcol),
+                                       _p(s_v), P, bits, int(bool(causal)), out_dtype, _p(O), self._stream(stream)),
+                    "qattention")
+
+    def stwq_reserve_attention(self, G, Tq, Tk, d):
+        self._check(self._L.stwq_reserve_attention(self._h, G, Tq, Tk, d), "stwq_reserve_attention")
+
+    def qattn_softmax_quantize(self, S, Tq, Tk, causal, bits, Pq, stream=None):
+        rows, ld = _mk(S, "S")
+        self._args("qattn_softmax_quantize", ("S", S, _F32, (rows, ld), False), ("Pq", Pq, _U8, (rows, ld), False))
+        self._check(self._L.qattn_softmax_quantize(self._h, _p(S), rows, Tq, Tk, ld, int(bool(causal)), bits, _p(Pq),
+                                                   self._stream(stream)), "qattn_softmax_quantize")
+
+    def qattn_pv(self, Pq, Vt, s_v, delta_p, out_dtype, O, stream=None):
+        G, Tq, Tk_pad = (int(v) for v in Pq.shape)
+        d, Tmax = int(Vt.shape[1]), int(Vt.shape[2])
+        self._args("qattn_pv", ("Pq", Pq, _U8, (G, Tq, Tk_pad), False), ("Vt", Vt, _I8, (G, d, Tmax), False),
+                   ("s_v", s_v, _F32, (d,), out_dtype == OUT_INT32), ("delta_p", delta_p, _F32, (1,), out_dtype == OUT_INT32),
+                   ("O", O, _out_dtype("qattn_pv", out_dtype), (G, Tq, d), False))
+        self._check(self._L.qattn_pv(self._h, _p(Pq), G, Tq, Tk_pad, d, Tmax, _p(Vt), _p(s_v), _p(delta_p), out_dtype,
+                                     _p(O), self._stream(stream)), "qattn_pv")
 
     def _quantize_specs(self, X, x_dtype, pos_ids, s_ch, s_tok, Xq):
         M, K = _mk(X)

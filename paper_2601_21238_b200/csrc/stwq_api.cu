@@ -170,6 +170,7 @@ void stwq_destroy(stwq_ctx* ctx)
     if (ctx->ws_dec) cudaFree(ctx->ws_dec);
     if (ctx->ws_dyn) cudaFree(ctx->ws_dyn);
     if (ctx->ws_w4) cudaFree(ctx->ws_w4);
+    if (ctx->ws_attn) cudaFree(ctx->ws_attn);
     if (ctx->d_status) cudaFree(ctx->d_status);
     delete ctx;
 }

@@ -1,0 +1,249 @@
+// Quantized attention matmuls and the quantized KV cache (Section 5: all linear layers and matrix
+// multiplications run in 6 or 8 bits; Appendix C: so does the KV cache). The two matmuls of a head,
+// S = Q K^T and O = P V, run on the tensor cores as batched integer GEMMs (qgemm2 with one matrix
+// per head); this file holds what surrounds them:
+//
+//   rowq_kernel               rows of Q, K or V -> int8 codes with static scales (the quantizer of
+//                             Eq. 1 as the linear layers use it: (x * rc[c]) * rt[pos], round to nearest
+//                             even, clamp), written densely (Q), at their position in the key cache, or
+//                             transposed into the value cache;
+//   softmax_quantize_kernel   row softmax of the dequantized scores and the quantizer of the
+//                             probabilities: Eq. 1 on the fixed range [0, 1], delta = 1 / (2^b - 1), zero
+//                             point 0, unsigned codes.
+//
+// Readings (the paper names the operands but not their quantizers): queries and keys carry one
+// static scale per token position, which factors out of the sum over channels; values carry one
+// static scale per channel, because a scale that varied along the keys could not leave the sum over
+// keys; the caches hold codes: K as [G, Tmax, d] and V transposed as [G, d, Tmax], so that both
+// matmuls read K-major operands.
+#include "stwq_internal.cuh"
+
+namespace {
+
+constexpr int kRowThreads = 128;
+
+// One block per row. out index = g * out_gstride + out_row * out_row_stride + c * out_col_stride,
+// out_row = the row's position (caches) or its index within the matrix (dense output).
+__global__ void __launch_bounds__(kRowThreads)
+rowq_kernel(const float* __restrict__ X, int d, const int32_t* __restrict__ pos_ids, int rows_per_g, int pos0,
+            const float* __restrict__ s_tok, int P, const float* __restrict__ s_ch, int qmin, int qmax,
+            int8_t* __restrict__ out, int64_t out_gstride, int64_t out_row_stride, int64_t out_col_stride,
+            int out_row_from_pos, uint32_t* __restrict__ status)
+{
+    const int64_t r = blockIdx.x;
+    const int g = (int)(r / rows_per_g);
+    const int t = (int)(r - (int64_t)g * rows_per_g);
+    const int pos = pos_ids != nullptr ? pos_ids[t] : pos0 + t;
+    const bool ok = pos >= 0 && pos < P;
+    if (!ok && threadIdx.x == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+    const float rt = (s_tok != nullptr && ok) ? __frcp_rn(s_tok[pos]) : 1.0f;
+    const int out_row = out_row_from_pos ? pos : t;
+    if (out_row_from_pos && !ok) return;                  // no slot in the cache for a position outside [0, P)
+    const float* x = X + r * d;
+    int8_t* o = out + (int64_t)g * out_gstride + (int64_t)out_row * out_row_stride;
+    for (int c = threadIdx.x; c < d; c += kRowThreads) {
+        const float rc = s_ch != nullptr ? __frcp_rn(s_ch[c]) : 1.0f;
+        const float u = __fmul_rn(__fmul_rn(x[c], rc), rt);
+        o[(int64_t)c * out_col_stride] = ok ? (int8_t)stwq_code(u, qmin, qmax) : (int8_t)0;
+    }
+}
+
+// One warp per row of S [rows, ld] (ld >= Tk, padding columns are written as code 0). Causal: query
+// i of a matrix (i = row % Tq) sees the keys j <= i + (Tk - Tq).
+__global__ void __launch_bounds__(256)
+softmax_quantize_kernel(const float* __restrict__ S, int64_t rows, int Tq, int Tk, int ld, int causal, float levels,
+                        uint8_t* __restrict__ Pq, float* __restrict__ delta_out)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0 && delta_out != nullptr) *delta_out = __fdiv_rn(1.0f, levels);
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (row >= rows) return;
+    const int i = (int)(row % Tq);
+    const int last = causal ? min(Tk - 1, i + (Tk - Tq)) : Tk - 1;       // last visible key
+    const float* s = S + row * ld;
+    uint8_t* p = Pq + row * ld;
+    float m = -INFINITY;
+    for (int j = lane; j <= last; j += 32) m = fmaxf(m, s[j]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    float sum = 0.0f;
+    for (int j = lane; j <= last; j += 32) sum += exp2f((s[j] - m) * 1.4426950408889634f);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+    const float scale = sum > 0.0f ? __fdiv_rn(levels, sum) : 0.0f;
+    for (int j = lane; j < ld; j += 32) {
+        float u = 0.0f;
+        if (j <= last) u = exp2f((s[j] - m) * 1.4426950408889634f) * scale;
+        p[j] = (uint8_t)min(max(__float2int_rn(u), 0), (int)levels);
+    }
+}
+
+int launch_rowq(stwq_ctx* ctx, const float* X, int64_t rows, int d, const int32_t* pos_ids, int rows_per_g, int pos0,
+                const float* s_tok, int P, const float* s_ch, int bits, int8_t* out, int64_t gs, int64_t rs, int64_t cs,
+                int from_pos, cudaStream_t st)
+{
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    rowq_kernel<<<(unsigned)rows, kRowThreads, 0, st>>>(X, d, pos_ids, rows_per_g, pos0, s_tok, P, s_ch, qmin, qmax, out, gs,
+                                                        rs, cs, from_pos, ctx->d_status);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int64_t round_up(int64_t v, int64_t m) { return (v + m - 1) / m * m; }
+
+struct DevGuard {
+    int prev = -1;
+    bool switched = false;
+    explicit DevGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) == cudaSuccess && prev != dev) {
+            cudaSetDevice(dev);
+            switched = true;
+        }
+    }
+    ~DevGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+// Workspace of one qattention call: codes of Q, scores, probability codes, the padded key-column
+// scales and the probability step.
+struct AttnWs {
+    int8_t* Qq;
+    float* S;
+    uint8_t* Pq;
+    float* skcol;
+    float* delta_p;
+    size_t bytes;
+};
+AttnWs attn_layout(void* base, int64_t G, int64_t Tq, int64_t Tk_pad, int64_t d)
+{
+    AttnWs w;
+    size_t off = 0;
+    auto take = [&](size_t n) { size_t o = off; off = (size_t)round_up((int64_t)(off + n), 256); return o; };
+    const size_t oq = take((size_t)(G * Tq * d));
+    const size_t os = take((size_t)(G * Tq * Tk_pad) * 4);
+    const size_t op = take((size_t)(G * Tq * Tk_pad));
+    const size_t ok = take((size_t)Tk_pad * 4);
+    const size_t od = take(256);
+    uint8_t* b = static_cast<uint8_t*>(base);
+    w.Qq = reinterpret_cast<int8_t*>(b + oq);
+    w.S = reinterpret_cast<float*>(b + os);
+    w.Pq = b + op;
+    w.skcol = reinterpret_cast<float*>(b + ok);
+    w.delta_p = reinterpret_cast<float*>(b + od);
+    w.bytes = off;
+    return w;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kv_append(stwq_ctx* ctx, const float* Knew, const float* Vnew, int G, int t_new, int d, int pos0, int Tmax,
+              const float* s_k, const float* s_v, int P, int bits, int8_t* Kc, int8_t* Vt, void* stream)
+{
+    if (!ctx || !Knew || !Vnew || !s_k || !s_v || !Kc || !Vt) return STWQ_ERR_NULL;
+    if (G <= 0 || t_new <= 0 || d <= 0 || Tmax <= 0 || P <= 0 || pos0 < 0) return STWQ_ERR_DIM;
+    if ((int64_t)pos0 + t_new > Tmax || (int64_t)pos0 + t_new > P) return STWQ_ERR_DIM;
+    if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
+    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Kc) || !aligned16(Vt)) return STWQ_ERR_ALIGN;
+    DevGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t rows = (int64_t)G * t_new;
+    int rc = launch_rowq(ctx, Knew, rows, d, nullptr, t_new, pos0, s_k, P, nullptr, bits, Kc, (int64_t)Tmax * d, d, 1, 1, st);
+    if (rc != STWQ_OK) return rc;
+    return launch_rowq(ctx, Vnew, rows, d, nullptr, t_new, pos0, nullptr, P, s_v, bits, Vt, (int64_t)d * Tmax, 1, Tmax, 1, st);
+}
+
+int stwq_reserve_attention(stwq_ctx* ctx, int G, int Tq, int Tk, int d)
+{
+    if (!ctx) return STWQ_ERR_NULL;
+    if (G <= 0 || Tq <= 0 || Tk <= 0 || d <= 0) return STWQ_ERR_DIM;
+    DevGuard g(ctx->device);
+    const AttnWs w = attn_layout(nullptr, G, Tq, round_up(Tk, 16), d);
+    return stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, nullptr, 0);
+}
+
+int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
+               const int8_t* Kc, const int8_t* Vt, const float* s_q, const float* s_kcol, const float* s_v, int P,
+               int bits, int causal, int out_dtype, void* O, void* stream)
+{
+    if (!ctx || !Q || !pos_q || !Kc || !Vt || !s_q || !s_kcol || !s_v || !O) return STWQ_ERR_NULL;
+    if (G <= 0 || Tq <= 0 || Tk <= 0 || d <= 0 || Tmax <= 0 || P <= 0) return STWQ_ERR_DIM;
+    if (Tk > Tmax || (causal && Tq > Tk) || d > 256) return STWQ_ERR_DIM;
+    if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
+    if (out_dtype != STWQ_OUT_F32 && out_dtype != STWQ_OUT_BF16) return STWQ_ERR_BITS;
+    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Q) || !aligned16(Kc) || !aligned16(Vt) || !aligned16(O) ||
+        !aligned16(s_v))
+        return STWQ_ERR_ALIGN;
+    DevGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t Tk_pad = round_up(Tk, 16);
+    AttnWs w = attn_layout(nullptr, G, Tq, Tk_pad, d);
+    int rc = stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, st, 0);
+    if (rc != STWQ_OK) return rc;
+    w = attn_layout(ctx->ws_attn, G, Tq, Tk_pad, d);
+
+    // queries -> codes with their per-position scales
+    rc = launch_rowq(ctx, Q, (int64_t)G * Tq, d, pos_q, Tq, 0, s_q, P, nullptr, bits, w.Qq, (int64_t)Tq * d, d, 1, 0, st);
+    if (rc != STWQ_OK) return rc;
+    // key-column scales, padded with zeros to the 16-column pitch of the score matrix
+    cudaError_t e = cudaMemsetAsync(w.skcol, 0, (size_t)Tk_pad * 4, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(w.skcol, s_kcol, (size_t)Tk * 4, cudaMemcpyDeviceToDevice, st);
+    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    // S = dequantized Q K^T, one matrix per head: rows scaled by s_q[pos], columns by s_kcol
+    stwq_batch bq = {G, (int64_t)d, (int64_t)Tmax * d, 0, 1, 0};
+    rc = stwq_launch_qgemm2(ctx, w.Qq, pos_q, Tq, d, (int)Tk_pad, Kc, w.skcol, s_q, P, nullptr, STWQ_ACT_NONE, STWQ_OUT_F32,
+                            w.S, false, nullptr, st, nullptr, &bq);
+    if (rc != STWQ_OK) return rc;
+    // probabilities -> unsigned codes (and the step 1 / (2^b - 1) for the second dequantizer)
+    const float levels = (float)((1 << bits) - 1);
+    const int64_t rows = (int64_t)G * Tq;
+    softmax_quantize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(w.S, rows, Tq, Tk, (int)Tk_pad, causal ? 1 : 0, levels,
+                                                                       w.Pq, w.delta_p);
+    ctx->launches += 1;
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    // O = dequantized P V: unsigned probability codes times the transposed value cache, scaled by
+    // delta_p (one "position") and the value channels' scales
+    stwq_batch bp = {G, (int64_t)Tmax, (int64_t)d * Tmax, 0, 1, 1};
+    return stwq_launch_qgemm2(ctx, reinterpret_cast<const int8_t*>(w.Pq), nullptr, Tq, (int)Tk_pad, d, Vt, s_v, w.delta_p, 1,
+                              nullptr, STWQ_ACT_NONE, out_dtype, O, false, nullptr, st, nullptr, &bp);
+}
+
+// The stages of qattention on their own (tests compare each with the CPU definition).
+int qattn_softmax_quantize(stwq_ctx* ctx, const float* S, int64_t rows, int Tq, int Tk, int ld, int causal, int bits,
+                           uint8_t* Pq, void* stream)
+{
+    if (!ctx || !S || !Pq) return STWQ_ERR_NULL;
+    if (rows <= 0 || Tq <= 0 || Tk <= 0 || ld < Tk || (causal && Tq > Tk)) return STWQ_ERR_DIM;
+    if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
+    DevGuard g(ctx->device);
+    softmax_quantize_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        S, rows, Tq, Tk, ld, causal ? 1 : 0, (float)((1 << bits) - 1), Pq, nullptr);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+int qattn_pv(stwq_ctx* ctx, const uint8_t* Pq, int G, int Tq, int Tk_pad, int d, int Tmax, const int8_t* Vt,
+             const float* s_v, const float* delta_p, int out_dtype, void* O, void* stream)
+{
+    if (!ctx || !Pq || !Vt || !O) return STWQ_ERR_NULL;
+    if (out_dtype != STWQ_OUT_INT32 && (!s_v || !delta_p)) return STWQ_ERR_NULL;
+    if (G <= 0 || Tq <= 0 || Tk_pad <= 0 || d <= 0 || Tk_pad > Tmax || d > 256) return STWQ_ERR_DIM;
+    if (out_dtype < STWQ_OUT_F32 || out_dtype > STWQ_OUT_INT32) return STWQ_ERR_BITS;
+    if ((d & 15) != 0 || (Tmax & 15) != 0 || (Tk_pad & 15) != 0 || !aligned16(Pq) || !aligned16(Vt) || !aligned16(O) ||
+        (s_v && !aligned16(s_v)))
+        return STWQ_ERR_ALIGN;
+    DevGuard g(ctx->device);
+    stwq_batch bp = {G, (int64_t)Tmax, (int64_t)d * Tmax, 0, 1, 1};
+    return stwq_launch_qgemm2(ctx, reinterpret_cast<const int8_t*>(Pq), nullptr, Tq, Tk_pad, d, Vt, s_v, delta_p, 1, nullptr,
+                              STWQ_ACT_NONE, out_dtype, O, false, nullptr, static_cast<cudaStream_t>(stream), nullptr, &bp);
+}
+
+}  // extern "C"

@@ -37,6 +37,8 @@ struct stwq_ctx {
     void* ws_dec;              // split-K workspace: arrival counters, then int32 partial sums
     size_t ws_dec_bytes;
     uint64_t configured_decode;
+    void* ws_attn;             // workspace of qattention: codes of Q, scores, probability codes
+    size_t ws_attn_bytes;
     int8_t* ws_w4;             // workspace: int8 copy of packed 4-bit weights (qlinear_w4 on the tiled route)
     size_t ws_w4_bytes;
     int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
@@ -59,6 +61,16 @@ struct stwq_asym {
     const int32_t* z_w;        // [N] signed zero point per output channel
     const int32_t* colsum;     // [N] sum_k Wq[n,k]
     const int32_t* rowcorr;    // [M] sum_k Xq[m,k] - K z_tok[pos[m]]
+};
+
+// Batched operands of the CTA-pair GEMM (one matrix per attention head): A [G, M, K] and Y [G, M, N]
+// dense; B [G, N, K] with rows ldb bytes apart and matrices b_gstride bytes apart.
+struct stwq_batch {
+    int G;
+    int64_t ldb, b_gstride;
+    int64_t sw_gstride;        // elements between the column-scale vectors of two matrices (0 = one vector for all)
+    int pos_shared;            // pos_ids has M entries shared by all matrices (else G * M)
+    int a_unsigned;            // A holds unsigned 8-bit codes (attention probabilities)
 };
 
 // Launchers (host). Each returns STWQ_OK or STWQ_ERR_CUDA and bumps ctx->launches.
@@ -94,7 +106,8 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize,
-                       const struct stwq_chain* chain, cudaStream_t st, const struct stwq_asym* asym = nullptr);
+                       const struct stwq_chain* chain, cudaStream_t st, const struct stwq_asym* asym = nullptr,
+                       const struct stwq_batch* batch = nullptr);
 int stwq_launch_decode(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K,
                        int N, const int8_t* Wq, const float* s_w, const float* s_tok, int P,
                        const float* bias, int act, int out_dtype, void* Y, bool after_quantize, cudaStream_t st);

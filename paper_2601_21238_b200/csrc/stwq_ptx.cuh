@@ -151,6 +151,22 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
         : "memory");
 }
+// The same with a third coordinate (batched operands: one matrix per head).
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int c0, int c1, int c2,
+                                                 uint32_t bar_cluster_addr)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4}], [%5];"
+        ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(bar_cluster_addr)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+                 : "memory");
+}
 __device__ __forceinline__ void tc_mma_i8_pair(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                                uint32_t accumulate)
 {
@@ -362,3 +378,8 @@ __device__ __forceinline__ float apply_act(float z)
 // 2-D tensor map over a dense row-major [rows, cols] matrix with 128-byte swizzle (host side).
 int stwq_encode_2d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* ptr,
                    int64_t rows, int64_t cols, int box_cols, int box_rows);
+// 3-D tensor map over `batch` row-major [rows, cols] matrices, rows row_pitch bytes apart, matrices
+// batch_pitch bytes apart; the box is one matrix deep.
+int stwq_encode_3d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* ptr,
+                   int64_t rows, int64_t cols, int64_t batch, int64_t row_pitch, int64_t batch_pitch, int box_cols,
+                   int box_rows);

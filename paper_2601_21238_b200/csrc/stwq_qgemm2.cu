@@ -63,6 +63,11 @@ struct Gemm2Params {
     int qmin_next, qmax_next;
     void* Y;                   // used by the direct-store epilogue
     int y_vec32;               // Y base and row pitch are 32-byte aligned: 256-bit stores are legal
+    // batched operands (attention heads): tile index = g * tiles_per_g + tile within matrix g
+    int tiles_per_g;
+    int pos_shared;            // pos_ids indexed by the row within the matrix (else by g * M + row)
+    int64_t sw_gstride;        // s_w of matrix g starts at s_w + g * sw_gstride
+    uint32_t idesc;            // instruction descriptor (signed or unsigned A)
 };
 
 // STORE = 0: the epilogue stages 32 x 128-byte pieces in shared memory and writes them with TMA
@@ -188,7 +193,8 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
             asm volatile("griddepcontrol.wait;" ::: "memory");
             for (int u = pair; ok && u < p.num_units; u += num_pairs) {
                 const Unit w = decode_unit(p, u);
-                const int tile = w.tile;
+                const int g = w.tile / p.tiles_per_g;
+                const int tile = w.tile - g * p.tiles_per_g;
                 const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
                 const int n0 = (tile % p.tiles_n) * BN + (int)rank * (BN / 2);
                 const int my_row0 = lane == 0 ? m0 : n0;
@@ -197,7 +203,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const uint32_t ph = (it / STAGES) & 1u;
                     if (!mbar_wait(bar_empty(s), ph ^ 1u, abort_flag, limit)) { ok = false; break; }
                     if (rank == 0 && lane == 0) mbar_expect_tx(bar_full(s), 2 * L::kStageBytes);
-                    tma_load_2d_pair(my_dst0 + s * my_stage_bytes, my_map, kb * kBK, my_row0, full0 + 8u * s);
+                    tma_load_3d_pair(my_dst0 + s * my_stage_bytes, my_map, kb * kBK, my_row0, g, full0 + 8u * s);
                 }
             }
             ok = __all_sync(0x3u, ok);
@@ -213,7 +219,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
     } else if (warp == 1) {
         // ------------------------------------------------------------------ MMA issuer (leader)
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = make_idesc_i8(2 * kBM, BN);
+            const uint32_t idesc = p.idesc;
             uint32_t it = 0, t = 0;
             bool ok = true;
             for (int u = pair; ok && u < p.num_units; u += num_pairs, ++t) {
@@ -261,12 +267,16 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
         bool ok = true;
         for (int u = pair; u < p.num_units; u += num_pairs, ++t) {
             const Unit wu = decode_unit(p, u);
-            const int tile = wu.tile;
+            const int g = wu.tile / p.tiles_per_g;
+            const int tile = wu.tile - g * p.tiles_per_g;
             const int acc = t & 1;
             const uint32_t aph = (t >> 1) & 1u;
             const int m0 = (tile / p.tiles_n) * (2 * kBM) + (int)rank * kBM;
             const int n0 = (tile % p.tiles_n) * BN;
-            const int64_t row = (int64_t)m0 + q * 32 + lane;
+            const int64_t row = (int64_t)m0 + q * 32 + lane;              // row within matrix g
+            const int64_t grow = (int64_t)g * p.M + row;                  // row of the stacked output
+            const int64_t prow = p.pos_shared ? row : grow;               // index into pos_ids
+            const float* g_sw = p.s_w + (int64_t)g * p.sw_gstride;
             float st = 0.0f, rtn = 0.0f;
             int zx = 0, Rm = 0;
             if (ASYM) {
@@ -283,8 +293,8 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     *reinterpret_cast<int4*>(my_cs + i) = cs;
                 }
                 if (row < p.M) {
-                    const int pos = p.pos_ids[row];
-                    Rm = p.rowcorr[row];
+                    const int pos = p.pos_ids[prow];
+                    Rm = p.rowcorr[grow];
                     if (pos >= 0 && pos < p.P) zx = p.z_tok[pos];
                 }
                 __syncwarp();
@@ -298,7 +308,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     const int col = n0 + (sub + k * kSubs) * kChunkCols + (i % kChunkCols);
                     float4 sw = make_float4(0.f, 0.f, 0.f, 0.f), bi = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (col < p.N) {                      // N is a multiple of 4: the float4 is in range
-                        sw = __ldg(reinterpret_cast<const float4*>(p.s_w + col));
+                        sw = __ldg(reinterpret_cast<const float4*>(g_sw + col));
                         if (p.bias != nullptr) bi = __ldg(reinterpret_cast<const float4*>(p.bias + col));
                     }
                     *reinterpret_cast<float4*>(my_sw + i) = sw;
@@ -313,7 +323,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     }
                 }
                 if (row < p.M) {
-                    const int pos = p.pos_ids[row];
+                    const int pos = p.pos_ids != nullptr ? p.pos_ids[prow] : 0;      // no positions: one scale for all rows
                     if (pos >= 0 && pos < p.P) {
                         st = p.s_tok[pos];
                         if (OUT == kOutCodes) rtn = __fdiv_rn(1.0f, p.s_tok_next[pos]);
@@ -491,7 +501,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                 if (STORE == 1) {
                     // straight from registers: this thread's 128 contiguous bytes of row `row`
                     if (row < p.M && col0 < p.N) {
-                        uint8_t* y = reinterpret_cast<uint8_t*>(p.Y) + ((size_t)row * (size_t)p.N + (size_t)col0) * kElem;
+                        uint8_t* y = reinterpret_cast<uint8_t*>(p.Y) + ((size_t)grow * (size_t)p.N + (size_t)col0) * kElem;
                         if (p.y_vec32 && col0 + kChunkCols <= p.N) {
 #pragma unroll
                             for (int g = 0; g < 4; ++g) st_global_v8(y + g * 32, w + g * 8);
@@ -516,7 +526,7 @@ qgemm2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ C
                     fence_async_smem();
                     __syncwarp();
                     if (lane == 0) {
-                        if (col0 < p.N && (int64_t)m0 + q * 32 < p.M) tma_store_2d(&tmY, stage_tile, col0, m0 + q * 32);
+                        if (col0 < p.N && (int64_t)m0 + q * 32 < p.M) tma_store_3d(&tmY, stage_tile, col0, m0 + q * 32, g);
                         bulk_commit();    // one group per chunk, even an empty one: wait_group.read 1 counts groups
                     }
                 }
@@ -554,6 +564,26 @@ int stwq_encode_2d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int 
     cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, dt, 2, const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        ctx->last_cuda_error = (int)r;
+        return STWQ_ERR_CUDA;
+    }
+    return STWQ_OK;
+}
+
+int stwq_encode_3d(stwq_ctx* ctx, CUtensorMap* map, CUtensorMapDataType dt, int elem_bytes, const void* ptr,
+                   int64_t rows, int64_t cols, int64_t batch, int64_t row_pitch, int64_t batch_pitch, int box_cols,
+                   int box_rows)
+{
+    EncodeTiledFn fn = reinterpret_cast<EncodeTiledFn>(ctx->encode_tiled);
+    cuuint64_t gdim[3] = {(cuuint64_t)cols, (cuuint64_t)rows, (cuuint64_t)batch};
+    cuuint64_t gstride[2] = {(cuuint64_t)row_pitch, (cuuint64_t)batch_pitch};
+    cuuint32_t box[3] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    (void)elem_bytes;
+    CUresult r = fn(map, dt, 3, const_cast<void*>(ptr), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -675,8 +705,9 @@ bool stwq_qgemm2_supported(int N, int out_dtype, const float* s_w, const float* 
 int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, int64_t M, int K, int N,
                        const int8_t* Wq, const float* s_w, const float* s_tok, int P, const float* bias,
                        int act, int out_dtype, void* Y, bool after_quantize, const stwq_chain* chain, cudaStream_t st,
-                       const stwq_asym* asym)
+                       const stwq_asym* asym, const stwq_batch* batch)
 {
+    const int G = batch ? batch->G : 1;
     // 256-wide tiles whenever N has more than 128 columns: a 128-wide tile needs 1.5x the
     // L2 -> shared-memory bytes per multiply-accumulate and is bound by that feed.
     const int tiles_m = (int)((M + 2 * kBM - 1) / (2 * kBM));
@@ -699,7 +730,12 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.M = M; p.N = N; p.K = K; p.P = P;
     p.pos_ids = pos_ids; p.s_w = s_w; p.s_tok = s_tok; p.bias = bias;
     p.tiles_n = (N + bn - 1) / bn;
-    p.num_tiles = tiles_m * p.tiles_n;
+    p.tiles_per_g = tiles_m * p.tiles_n;
+    p.num_tiles = G * p.tiles_per_g;
+    p.pos_shared = batch ? batch->pos_shared : 1;
+    p.sw_gstride = batch ? batch->sw_gstride : 0;
+    p.idesc = stwq_ptx::make_idesc_i8(2 * kBM, bn);
+    if (batch && batch->a_unsigned) p.idesc &= ~(1u << 7);         // A format field: 0 = unsigned 8-bit
     p.num_kb = (K + kBK - 1) / kBK;
     p.status = ctx->d_status;
     p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
@@ -719,7 +755,7 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     p.counters = nullptr;
     const int pairs = ctx->max_pairs > 0 ? ctx->max_pairs : ctx->sm_count / 2;
     const int tail = p.num_tiles % pairs;
-    if (bn == 256 && tail > 0 && 2 * tail <= pairs && ctx->force_ksplit > 0) {
+    if (bn == 256 && tail > 0 && 2 * tail <= pairs && ctx->force_ksplit > 0 && G == 1) {
         int nsplit = ctx->force_ksplit < p.num_kb ? ctx->force_ksplit : p.num_kb;
         if (nsplit >= 2) {
             const int kbps = (p.num_kb + nsplit - 1) / nsplit;
@@ -739,18 +775,21 @@ int stwq_launch_qgemm2(stwq_ctx* ctx, const int8_t* Xq, const int32_t* pos_ids, 
     }
 
     CUtensorMap tmA, tmB, tmY;
-    int rc = stwq_encode_2d(ctx, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, kBK, kBM);
+    const int64_t ldb = batch ? batch->ldb : K;
+    const int64_t bgs = batch ? batch->b_gstride : (int64_t)N * K;
+    int rc = stwq_encode_3d(ctx, &tmA, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Xq, M, K, G, K, M * (int64_t)K, kBK, kBM);
     if (rc != STWQ_OK) return rc;
-    rc = stwq_encode_2d(ctx, &tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, N, K, kBK, bn / 2);
+    rc = stwq_encode_3d(ctx, &tmB, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Wq, N, K, G, ldb, bgs, kBK, bn / 2);
     if (rc != STWQ_OK) return rc;
+    const int64_t ypitch = (int64_t)N * elem, ygs = M * ypitch;
     if (out_dtype == STWQ_OUT_BF16)
-        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, M, N, 64, 32);
+        rc = stwq_encode_3d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, Y, M, N, G, ypitch, ygs, 64, 32);
     else if (out_dtype == STWQ_OUT_F32)
-        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Y, M, N, 32, 32);
+        rc = stwq_encode_3d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, Y, M, N, G, ypitch, ygs, 32, 32);
     else if (out_dtype == kOutCodes)
-        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Y, M, N, 128, 32);
+        rc = stwq_encode_3d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Y, M, N, G, ypitch, ygs, 128, 32);
     else
-        rc = stwq_encode_2d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, 32, 32);
+        rc = stwq_encode_3d(ctx, &tmY, CU_TENSOR_MAP_DATA_TYPE_INT32, 4, Y, M, N, G, ypitch, ygs, 32, 32);
     if (rc != STWQ_OK) return rc;
     if (bn == 128) return launch_bn<128, 6, 8, 0>(ctx, tmA, tmB, tmY, p, act, out_dtype, after_quantize, st);
     // Long main loops hide the epilogue anyway and gain from the deeper ring that the

@@ -1,0 +1,154 @@
+"""Quantized attention matmuls and the quantized KV cache on the GPU against the CPU oracle: cache
+codes, integer accumulators and probability codes of every stage, then the composite call.
+Integer results bit-exact; the probability codes (an integer decided by a floating-point softmax)
+may differ by one where the oracle's value before rounding lies within fp32 noise of a tie."""
+import numpy as np
+import pytest
+
+import oracle
+from layer_setup import assert_close
+
+pytestmark = pytest.mark.gpu
+
+rng = np.random.default_rng(31)
+
+
+@pytest.fixture(scope="module")
+def gpu():
+    import torch
+
+    import paper_2601_21238_b200 as pk
+    from paper_2601_21238_b200 import binding as B
+    from paper_2601_21238_b200 import build as pkbuild
+    pkbuild.build()
+    ctx = pk.Context(0)
+    dev = torch.device("cuda:0")
+
+    class G:
+        pass
+    g = G()
+    g.torch, g.ctx, g.dev, g.B = torch, ctx, dev, B
+    g.T = lambda a: None if a is None else torch.from_numpy(np.ascontiguousarray(a)).to(dev)
+    yield g
+    ctx.close()
+
+
+def _head_data(G, T, d, P):
+    """Seeded heads with per-position magnitude and a few outlier channels, and static scales sized
+    like a calibration would (ranges near the data's abs-max per position / per channel)."""
+    sig = rng.uniform(0.5, 3.0, (1, T, 1)).astype(np.float32)
+    Q = (rng.standard_normal((G, T, d)).astype(np.float32) * sig)
+    K = (rng.standard_normal((G, T, d)).astype(np.float32) * sig)
+    V = rng.standard_normal((G, T, d)).astype(np.float32)
+    V[:, :, :2] *= 6.0
+    s_q = np.ones(P, np.float32)
+    s_k = np.ones(P, np.float32)
+    s_q[:T] = (np.abs(Q).max(axis=(0, 2)) * 2 / 255 * 0.9).astype(np.float32)      # a little saturation
+    s_k[:T] = (np.abs(K).max(axis=(0, 2)) * 2 / 255).astype(np.float32)
+    s_v = (np.abs(V).max(axis=(0, 1)) * 2 / 255).astype(np.float32)
+    return Q, K, V, s_q, s_k, s_v
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+def test_kv_append_writes_the_oracles_codes_into_both_cache_layouts(gpu, bits):
+    torch = gpu.torch
+    G, T, d, P, Tmax = 3, 21, 48, 24, 32
+    _, K, V, _, s_k, s_v = _head_data(G, T, d, P)
+    Kc = torch.full((G, Tmax, d), 77, dtype=torch.int8, device=gpu.dev)
+    Vt = torch.full((G, d, Tmax), 77, dtype=torch.int8, device=gpu.dev)
+    # prefill of 16 positions, then five single-position steps
+    gpu.ctx.kv_append(gpu.T(K[:, :16]), gpu.T(V[:, :16]), 0, gpu.T(s_k), gpu.T(s_v), bits, Kc, Vt)
+    for t in range(16, T):
+        gpu.ctx.kv_append(gpu.T(K[:, t:t + 1]), gpu.T(V[:, t:t + 1]), t, gpu.T(s_k), gpu.T(s_v), bits, Kc, Vt)
+    assert gpu.ctx.stwq_device_status() == 0
+    pos = np.arange(T, dtype=np.int32)
+    for g in range(G):
+        want_k = oracle.quantize(K[g], pos, None, s_k, bits)
+        want_v = oracle.quantize(V[g], np.zeros(T, np.int32), s_v, np.ones(1, np.float32), bits)
+        np.testing.assert_array_equal(Kc[g, :T].cpu().numpy(), want_k)
+        np.testing.assert_array_equal(Vt[g, :, :T].cpu().numpy(), want_v.T)
+    assert (Kc[:, T:].cpu().numpy() == 77).all() and (Vt[:, :, T:].cpu().numpy() == 77).all()   # untouched slots
+    # a position beyond the cache or the scale table is refused on the host
+    with pytest.raises(Exception):
+        gpu.ctx.kv_append(gpu.T(K[:, :4]), gpu.T(V[:, :4]), Tmax - 2, gpu.T(s_k), gpu.T(s_v), bits, Kc, Vt)
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(5, 37, 37, True), (3, 1, 50, False), (2, 300, 300, True), (4, 20, 129, True)])
+def test_softmax_quantizer_codes(gpu, shape, bits):
+    torch = gpu.torch
+    G, Tq, Tk, causal = shape
+    ld = (Tk + 15) // 16 * 16
+    S = (rng.standard_normal((G * Tq, ld)) * 4).astype(np.float32)
+    Pq = torch.full((G * Tq, ld), 9, dtype=torch.uint8, device=gpu.dev)
+    gpu.ctx.qattn_softmax_quantize(gpu.T(S), Tq, Tk, causal, bits, Pq)
+    got = Pq.cpu().numpy().astype(np.int32)
+    assert (got[:, Tk:] == 0).all()                       # padding columns
+    flips = 0
+    for g in range(G):
+        want, u = oracle.softmax_quantize(S[g * Tq:(g + 1) * Tq, :Tk], causal, bits)
+        diff = got[g * Tq:(g + 1) * Tq, :Tk] != want
+        assert np.abs(got[g * Tq:(g + 1) * Tq, :Tk] - want.astype(np.int32)).max() <= 1
+        # fp32 softmax: relative error of a probability below 2e-6 (exp2 of a rounded argument, a sum of Tk terms)
+        assert (np.abs(u - np.floor(u) - 0.5)[diff] <= 2e-6 * np.maximum(1.0, u[diff]) * 8).all()
+        flips += int(diff.sum())
+    assert flips <= 1e-3 * got.size + 2
+
+
+@pytest.mark.parametrize("shape", [(3, 37, 48, 64, 64), (2, 300, 304, 128, 320), (5, 1, 80, 64, 96), (1, 680, 688, 64, 688)])
+def test_probability_value_matmul_is_exact(gpu, shape):
+    """Unsigned probability codes times the transposed value cache: int32 accumulators bit-exact
+    (a code above 127 must be read as unsigned), outputs within tolerance."""
+    torch = gpu.torch
+    G, Tq, Tk_pad, d, Tmax = shape
+    Pc = rng.integers(0, 256, (G, Tq, Tk_pad)).astype(np.uint8)
+    Vq = rng.integers(-128, 128, (G, Tmax, d)).astype(np.int8)          # columns beyond Tk_pad are never read
+    s_v = rng.uniform(1e-3, 1e-2, d).astype(np.float32)
+    delta = np.array([1.0 / 255.0], np.float32)
+    Vt = np.ascontiguousarray(Vq.transpose(0, 2, 1))
+    acc = torch.full((G, Tq, d), -3, dtype=torch.int32, device=gpu.dev)
+    gpu.ctx.qattn_pv(gpu.T(Pc), gpu.T(Vt), None, None, gpu.B.OUT_INT32, acc)
+    assert gpu.ctx.stwq_device_status() == 0
+    for out, dt, rtol in (("fp32", torch.float32, 1e-5), ("bf16", torch.bfloat16, 1e-2)):
+        O = torch.full((G, Tq, d), -3, dtype=dt, device=gpu.dev)
+        gpu.ctx.qattn_pv(gpu.T(Pc), gpu.T(Vt), gpu.T(s_v), gpu.T(delta), gpu.B.OUT_F32 if out == "fp32" else gpu.B.OUT_BF16, O)
+        for g in range(G):
+            want = oracle.igemm_u8s8(Pc[g], Vq[g, :Tk_pad])
+            np.testing.assert_array_equal(acc[g].cpu().numpy(), want)
+            Y, mag = oracle.epilogue(want, np.zeros(Tq, np.int32), delta, s_v, None, 0)
+            assert_close(O[g].float().cpu().numpy(), {"Y": Y, "mag": mag, "act": 0}, rtol, f"P V {out}")
+
+
+@pytest.mark.parametrize("bits", [8, 6])
+@pytest.mark.parametrize("shape", [(4, 37, 37, 64, True), (2, 1, 50, 64, False), (3, 129, 129, 128, True), (2, 40, 200, 48, True)])
+def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits):
+    """The composite call against the oracle's head: the output differs from the oracle's only through
+    probability codes that sit on a rounding tie (each such code moves O by delta_p |Vq| s_v), so O is
+    compared with the usual tolerance plus that allowance for a handful of flips per row."""
+    torch = gpu.torch
+    G, Tq, Tk, d, causal = shape
+    P, Tmax = Tk + 3, (Tk + 15) // 16 * 16 + 16
+    Q, K, V, s_q, s_k, s_v = _head_data(G, Tk, d, P)
+    Q = Q[:, Tk - Tq:]                                    # the queries are the last Tq positions
+    pos_q = np.arange(Tk - Tq, Tk, dtype=np.int32)
+    pos_k = np.arange(Tk, dtype=np.int32)
+    scale = np.float32(1.0 / np.sqrt(d))
+    s_kcol = (s_k[pos_k] * scale).astype(np.float32)
+    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=gpu.dev)
+    Vt = torch.full((G, d, Tmax), 55, dtype=torch.int8, device=gpu.dev)      # stale codes beyond Tk must not matter
+    gpu.ctx.kv_append(gpu.T(K), gpu.T(V), 0, gpu.T(s_k), gpu.T(s_v), bits, Kc, Vt)
+    levels = 2 ** bits - 1
+    for out, dt, rtol in (("fp32", torch.float32, 1e-5), ("bf16", torch.bfloat16, 1e-2)):
+        O = torch.full((G, Tq, d), -3, dtype=dt, device=gpu.dev)
+        gpu.ctx.qattention(gpu.T(Q), gpu.T(pos_q), Tk, Kc, Vt, gpu.T(s_q), gpu.T(s_kcol), gpu.T(s_v), bits, causal,
+                           gpu.B.OUT_F32 if out == "fp32" else gpu.B.OUT_BF16, O)
+        assert gpu.ctx.stwq_device_status() == 0
+        got = O.float().cpu().numpy().astype(np.float64)
+        for g in range(G):
+            r = oracle.qattention(Q[g], K[g], V[g], pos_q, pos_k, s_q, s_k, s_v, scale, bits, causal)
+            np.testing.assert_array_equal(Kc[g, :Tk].cpu().numpy(), r["Kq"])
+            flip = 4 * (1.0 / levels) * (2 ** (bits - 1)) * s_v[None, :].astype(np.float64)     # four flipped codes per row
+            tol = rtol * (np.abs(r["O"]) + r["mag"]) + flip
+            assert (np.abs(got[g] - r["O"]) <= tol).all(), f"{out} head {g}: worst {np.abs(got[g] - r['O']).max()}"
+            # and it is a sensible attention: close to the float head computed from the same inputs
+        assert np.isfinite(got).all()

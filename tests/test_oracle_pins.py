@@ -620,3 +620,78 @@ def test_packed_rows_keep_the_channel_order_and_the_4bit_fold_fits():
     np.testing.assert_array_equal(oracle.unpack4(Wp), Wq)
     Xq = rng.integers(-128, 128, (5, K)).astype(np.int8)
     np.testing.assert_array_equal(oracle.igemm(Xq, oracle.unpack4(Wp)), Xq.astype(np.int64) @ Wq.astype(np.int64).T)
+
+
+# ----------------------------------------------------------------------------- quantized attention
+def test_softmax_quantizer_against_numpy_and_its_invariants():
+    """Probability codes: the textbook softmax (numpy, float64) scaled by 2^b - 1 and rounded; rows of
+    codes sum to 2^b - 1 within Tk / 2 (each code is within 1/2 of its exact value); a one-hot row gives
+    the code 2^b - 1; equal scores give equal codes; the causal mask zeroes exactly the keys after the
+    query; shifting a row by a constant changes nothing."""
+    rng = np.random.default_rng(21)
+    Tq, Tk = 9, 23
+    S = (rng.standard_normal((Tq, Tk)) * 3).astype(np.float32)
+    for bits in (8, 6):
+        D = 2 ** bits - 1
+        codes, u = oracle.softmax_quantize(S, False, bits)
+        e = np.exp(S.astype(np.float64) - S.astype(np.float64).max(axis=1, keepdims=True))
+        Pn = e / e.sum(axis=1, keepdims=True)
+        np.testing.assert_allclose(u, Pn * D, rtol=1e-12, atol=1e-12)
+        np.testing.assert_array_equal(codes, np.rint(Pn * D).astype(np.uint8))
+        assert np.abs(codes.astype(np.int64).sum(axis=1) - D).max() <= Tk / 2
+        shifted, _ = oracle.softmax_quantize(S + np.float32(8.0), False, bits)
+        assert np.abs(shifted.astype(int) - codes.astype(int)).max() <= 1      # fp32 rounding of S + 8 only
+        hot = np.full((1, Tk), -1e4, np.float32)
+        hot[0, 5] = 0.0
+        c1, _ = oracle.softmax_quantize(hot, False, bits)
+        assert c1[0, 5] == D and c1.sum() == D
+        flat, _ = oracle.softmax_quantize(np.zeros((1, 4), np.float32), False, bits)
+        assert (flat == np.rint(D / 4)).all()
+        # causal: Tq = Tk -> lower triangle; Tq < Tk -> the last query sees all keys
+        cc, _ = oracle.softmax_quantize(S[:, :Tq], True, bits)
+        assert (np.triu(cc, 1) == 0).all() and cc[0, 0] == D
+        cc2, _ = oracle.softmax_quantize(S, True, bits)
+        for i in range(Tq):
+            assert (cc2[i, i + Tk - Tq + 1:] == 0).all()
+        np.testing.assert_array_equal(cc2[Tq - 1], codes[Tq - 1])
+
+
+def test_unsigned_signed_integer_gemm_against_int64_and_a_hand_case():
+    rng = np.random.default_rng(22)
+    P = rng.integers(0, 256, (7, 40)).astype(np.uint8)
+    V = rng.integers(-128, 128, (40, 11)).astype(np.int8)
+    P[0], V[:, 0] = 255, -128                              # extreme: 40 * 255 * -128
+    np.testing.assert_array_equal(oracle.igemm_u8s8(P, V), P.astype(np.int64) @ V.astype(np.int64))
+    assert oracle.igemm_u8s8(P, V)[0, 0] == -40 * 255 * 128
+    # hand case: [200, 3] . [[-2], [100]] = -400 + 300; an unsigned 200 must not be read as -56
+    assert oracle.igemm_u8s8(np.array([[200, 3]], np.uint8), np.array([[-2], [100]], np.int8))[0, 0] == -100
+
+
+def test_quantized_attention_approaches_float_attention_and_factors_its_scales():
+    """The composition: with fine scales the quantized head is close to float attention (error bounded
+    by the quantization steps), the per-position query / key scales and the per-channel value scales
+    factor out of the integer sums exactly (the dequantized scores equal Qhat Khat^T), and a key
+    that is masked contributes nothing."""
+    rng = np.random.default_rng(23)
+    Tq, Tk, d, P = 12, 12, 16, 12
+    Q = rng.standard_normal((Tq, d)).astype(np.float32)
+    K = rng.standard_normal((Tk, d)).astype(np.float32)
+    V = rng.standard_normal((Tk, d)).astype(np.float32)
+    pos = np.arange(Tq, dtype=np.int32)
+    s_q = (np.abs(Q).max(axis=1) * 2 / 255).astype(np.float32)
+    s_k = (np.abs(K).max(axis=1) * 2 / 255).astype(np.float32)
+    s_v = (np.abs(V).max(axis=0) * 2 / 255).astype(np.float32)
+    scale = 1.0 / np.sqrt(d)
+    r = oracle.qattention(Q, K, V, pos, pos, s_q, s_k, s_v, scale, 8, True)
+    Qh = r["Qq"].astype(np.float64) * s_q[:, None]
+    Kh = r["Kq"].astype(np.float64) * s_k[:, None]
+    np.testing.assert_allclose(r["S"], (Qh @ Kh.T) * scale, rtol=2e-6, atol=1e-6)
+    Sf = (Q.astype(np.float64) @ K.astype(np.float64).T) * scale
+    Sf = np.where(np.tril(np.ones((Tq, Tk))) > 0, Sf, -np.inf)
+    Pf = np.exp(Sf - Sf.max(axis=1, keepdims=True))
+    Pf /= Pf.sum(axis=1, keepdims=True)
+    Of = Pf @ V.astype(np.float64)
+    assert np.abs(r["O"] - Of).max() < 0.05 and np.abs(r["O"] - Of).mean() < 0.01
+    Vh = r["Vq"].astype(np.float64) * s_v[None, :]
+    np.testing.assert_allclose(r["O"], (r["Pq"].astype(np.float64) / 255.0) @ Vh, rtol=1e-6, atol=1e-7)
+    assert (np.triu(r["Pq"], 1) == 0).all()
