@@ -142,6 +142,20 @@ int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const floa
                uint32_t pct_ppm, int variant, float* s_ch, int32_t* k_star, void* stream);
 
 /*
+ * Distribution-Guided Calibration (Section 4.3, Eq. 17): the Mahalanobis distance of every sample of a
+ * set to the set's own distribution, rho(x) = sqrt((x - u)^T S^-1 (x - u)) with u the mean and S the
+ * (population) covariance of the set, and the choice of the ceil(keep_ppm n / 1e6) samples with the
+ * largest rho (the paper keeps the top 50 %) as the calibration set. The paper does not say which
+ * vector stands for a sample: F [n, D] fp32 holds one feature vector per sample, D <= 1024.
+ * ridge >= 0: ridge * trace(S) / D is added to the diagonal of S before it is factorised (0 = Eq. 17 as
+ * printed; a covariance that is then not positive definite, e.g. D >= n, gives rho = 0 for every
+ * sample). rho [n] fp64 out; selected (int32, ceil(keep n) entries, may be NULL) receives the indices
+ * of the kept samples, largest rho first, equal rho in index order. All in fp64 on the GPU.
+ */
+int dgc_select(stwq_ctx* ctx, const float* F, int n, int D, uint32_t keep_ppm, double ridge, double* rho,
+               int32_t* selected, void* stream);
+
+/*
  * Equivalent scaling, weight side (Eq. 2: Y = (X / s)(s * W)), then per-output-channel
  * min-max weight quantization with the symmetric form of Eq. 1:
  *     W'[n,k] = W[n,k] * s_ch[k]                  (s_ch == NULL: W' = W)

@@ -89,6 +89,8 @@ def lib():
             L.orc_unpack4.argtypes = [C.POINTER(C.c_uint8), C.c_int64, bp]
             L.orc_softmax_quantize.argtypes = [fp, C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(C.c_uint8), dp]
             L.orc_igemm_u8s8.argtypes = [C.POINTER(C.c_uint8), bp, C.c_int, C.c_int, C.c_int, ip]
+            L.orc_dgc_select.restype = C.c_int
+            L.orc_dgc_select.argtypes = [fp, C.c_int, C.c_int, C.c_uint32, C.c_double, dp, ip]
             L.orc_gps_gain.restype = C.c_double
             L.orc_gps_gain.argtypes = [C.c_double] * 4
             _lib = L
@@ -418,3 +420,16 @@ def qattention(Q, K, V, pos_q, pos_k, s_q, s_k, s_v, softmax_scale, bits, causal
     O, mag = epilogue(acc_pv, np.zeros(Q.shape[0], np.int32), delta_p, s_v, None, 0)
     return {"Qq": Qq, "Kq": Kq, "Vq": Vq, "acc_qk": acc_qk, "s_kcol": s_kcol, "S": S32, "Pq": Pq, "u": u,
             "acc_pv": acc_pv, "delta_p": delta_p, "O": O, "mag": mag, "act": 0}
+
+
+def dgc_select(F, keep_ppm=500000, ridge=0.0):
+    """Mahalanobis distance of every sample (rows of F [n, D]) to the set, and the indices of the kept
+    fraction, largest distance first. Returns (rho float64 [n], selected int32 [k])."""
+    F = _f32(F)
+    n, D = F.shape
+    k = min(n, max(1, (keep_ppm * n + 999999) // 1000000))
+    rho = np.empty(n, np.float64)
+    sel = np.empty(k, np.int32)
+    if lib().orc_dgc_select(_ptr(F, C.c_float), n, D, keep_ppm, float(ridge), _ptr(rho, C.c_double), _ptr(sel, C.c_int32)) != 0:
+        raise ValueError("covariance not positive definite (use a ridge)")
+    return rho, sel

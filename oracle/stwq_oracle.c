@@ -812,3 +812,82 @@ void orc_igemm_u8s8(const uint8_t* P, const int8_t* Vq, int Tq, int Tk, int C, i
             acc[(int64_t)i * C + c] = s;
         }
 }
+
+/* ------------------------------------------------------------------------- */
+/*
+ * Distribution-Guided Calibration (Section 4.3, Eq. 17): the Mahalanobis distance of every
+ * sample of a set to the set's own distribution,
+ *     rho(x) = sqrt((x - u)^T S^-1 (x - u)),   u = mean, S = covariance of the set,
+ * and the selection of the fraction of samples with the largest rho (the paper keeps the top
+ * 50 %) as the calibration set. The paper does not say which vector represents a sample; the
+ * caller supplies one feature vector per sample, F [n, D].
+ * Readings: S is the population covariance (divide by n; the ranking does not depend on the
+ * factor); S may be singular (D >= n, constant features), so ridge * trace(S) / D is added to its
+ * diagonal (ridge = 0 gives Eq. 17 as printed; a zero-variance set gives rho = 0); S^-1 is applied
+ * through the Cholesky factor S = L L^T: rho^2 = |L^-1 (x - u)|^2. k = ceil(keep_ppm * n / 1e6)
+ * samples are kept, the largest rho first, equal rho in index order. All in double.
+ * Returns 0, or -1 if the (ridged) covariance is not positive definite.
+ */
+int orc_dgc_select(const float* F, int n, int D, uint32_t keep_ppm, double ridge, double* rho, int32_t* selected)
+{
+    double* u = (double*)calloc((size_t)D, sizeof(double));
+    double* S = (double*)calloc((size_t)D * D, sizeof(double));
+    double* y = (double*)malloc(sizeof(double) * (size_t)D);
+    int status = 0;
+    for (int i = 0; i < n; ++i)
+        for (int a = 0; a < D; ++a) u[a] += (double)F[(int64_t)i * D + a];
+    for (int a = 0; a < D; ++a) u[a] /= (double)n;
+    for (int i = 0; i < n; ++i)
+        for (int a = 0; a < D; ++a)
+            for (int b = 0; b <= a; ++b)
+                S[(int64_t)a * D + b] += ((double)F[(int64_t)i * D + a] - u[a]) * ((double)F[(int64_t)i * D + b] - u[b]);
+    double tr = 0.0;
+    for (int a = 0; a < D; ++a) {
+        for (int b = 0; b <= a; ++b) S[(int64_t)a * D + b] /= (double)n;
+        tr += S[(int64_t)a * D + a];
+    }
+    for (int a = 0; a < D; ++a) S[(int64_t)a * D + a] += ridge * tr / (double)D;
+    if (!(tr > 0.0)) {                                   /* every sample equals the mean */
+        for (int i = 0; i < n; ++i) rho[i] = 0.0;
+    } else {
+        /* Cholesky, lower triangle in place: L[a][b] for b <= a */
+        for (int k = 0; k < D && status == 0; ++k) {
+            double dkk = S[(int64_t)k * D + k];
+            for (int b = 0; b < k; ++b) dkk -= S[(int64_t)k * D + b] * S[(int64_t)k * D + b];
+            if (!(dkk > 0.0)) { status = -1; break; }
+            const double lkk = sqrt(dkk);
+            S[(int64_t)k * D + k] = lkk;
+            for (int a = k + 1; a < D; ++a) {
+                double v = S[(int64_t)a * D + k];
+                for (int b = 0; b < k; ++b) v -= S[(int64_t)a * D + b] * S[(int64_t)k * D + b];
+                S[(int64_t)a * D + k] = v / lkk;
+            }
+        }
+        for (int i = 0; i < n && status == 0; ++i) {     /* forward substitution L y = x - u */
+            double r2 = 0.0;
+            for (int a = 0; a < D; ++a) {
+                double v = (double)F[(int64_t)i * D + a] - u[a];
+                for (int b = 0; b < a; ++b) v -= S[(int64_t)a * D + b] * y[b];
+                y[a] = v / S[(int64_t)a * D + a];
+                r2 += y[a] * y[a];
+            }
+            rho[i] = sqrt(r2);
+        }
+    }
+    if (status == 0 && selected) {
+        int64_t k = ((int64_t)keep_ppm * n + 999999) / 1000000;
+        if (k < 1) k = 1;
+        if (k > n) k = n;
+        /* selection by rank: sample i is kept if fewer than k samples come before it */
+        for (int i = 0; i < n; ++i) {
+            int64_t before = 0;
+            for (int j = 0; j < n; ++j)
+                if (rho[j] > rho[i] || (rho[j] == rho[i] && j < i)) ++before;
+            if (before < k) selected[before] = i;
+        }
+    }
+    free(u);
+    free(S);
+    free(y);
+    return status;
+}

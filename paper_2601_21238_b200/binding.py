@@ -24,7 +24,8 @@ _SYMBOLS = ["stwq_create", "stwq_destroy", "stwq_reserve", "stwq_calibrate", "gp
             "stwq_strerror", "stwq_last_cuda_error", "qlinear_static", "dtwq_quantize", "qlinear_dtwq", "qlinear_chain", "qlinear_chain_q", "stwq_quantize_bf16", "stwq_calibrate_asym", "gps_fold_asym",
             "stwq_quantize_asym", "qlinear_asym", "gps_scales", "qlinear_bf16", "stwq_reserve_layer",
             "stwq_workspace_generation", "stwq_selftest_wait_expiry", "stwq_probe_int8_peak", "gps_fold_packed4", "stwq_unpack4",
-            "qlinear_w4", "kv_append", "qattention", "stwq_reserve_attention", "qattn_softmax_quantize", "qattn_pv"]
+            "qlinear_w4", "kv_append", "qattention", "stwq_reserve_attention", "qattn_softmax_quantize", "qattn_pv",
+            "dgc_select"]
 
 _lib = None
 
@@ -74,6 +75,7 @@ def load_library():
     L.stwq_reserve_attention.argtypes = [vp, i32, i32, i32, i32]
     L.qattn_softmax_quantize.argtypes = [vp, vp, i64, i32, i32, i32, i32, i32, vp, vp]
     L.qattn_pv.argtypes = [vp, vp, i32, i32, i32, i32, i32, vp, vp, vp, i32, vp, vp]
+    L.dgc_select.argtypes = [vp, vp, i32, i32, u32, C.c_double, vp, vp, vp]
     L.gps_scales.argtypes = [vp, vp, i64, i32, vp, i32, i32, u32, i32, vp, vp, vp]
     L.stwq_quantize.argtypes = [vp, vp, vp, i64, i32, vp, vp, i32, i32, vp, vp]
     L.qlinear.argtypes = [vp, vp, vp, i64, i32, i32, vp, vp, vp, i32, vp, vp, i32, i32, i32, vp, vp]
@@ -247,6 +249,14 @@ class Context:
                    ("Wq", Wq, _I8, (N, K), False), ("s_w", s_w, _F32, (N,), False))
         self._check(self._L.gps_fold(self._h, _p(W), N, K, _p(s_ch), bits, _p(Wq), _p(s_w),
                                      self._stream(stream)), "gps_fold")
+
+    def dgc_select(self, F, keep_ppm, ridge, rho, selected=None, stream=None):
+        n, D = _mk(F, "F")
+        k = min(n, max(1, (keep_ppm * n + 999999) // 1000000))
+        self._args("dgc_select", ("F", F, _F32, (n, D), False), ("rho", rho, "torch.float64", (n,), False),
+                   ("selected", selected, _I32, (k,), True))
+        self._check(self._L.dgc_select(self._h, _p(F), n, D, keep_ppm, float(ridge), _p(rho), _p(selected),
+                                       self._stream(stream)), "dgc_select")
 
     def gps_fold_packed4(self, W, s_ch, Wp, s_w, stream=None):
         N, K = _mk(W, "W")

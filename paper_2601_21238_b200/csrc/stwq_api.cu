@@ -267,6 +267,22 @@ int gps_scales(stwq_ctx* ctx, const float* Xcal, int64_t rows, int K, const floa
                            static_cast<cudaStream_t>(stream));
 }
 
+int dgc_select(stwq_ctx* ctx, const float* F, int n, int D, uint32_t keep_ppm, double ridge, double* rho,
+               int32_t* selected, void* stream)
+{
+    if (!ctx || !F || !rho) return STWQ_ERR_NULL;
+    if (n <= 0 || D <= 0 || D > 1024 || n > (1 << 20)) return STWQ_ERR_DIM;
+    if (keep_ppm < 1u || keep_ppm > 1000000u || !(ridge >= 0.0)) return STWQ_ERR_BITS;
+    DeviceGuard g(ctx->device);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int rc = ensure_dyn(ctx, stwq_dgc_ws_bytes(D), st);
+    if (rc != STWQ_OK) return rc;
+    int64_t k = ((int64_t)keep_ppm * n + 999999) / 1000000;
+    if (k < 1) k = 1;
+    if (k > n) k = n;
+    return stwq_launch_dgc(ctx, ctx->ws_dyn, F, n, D, (int)k, ridge, rho, selected, st);
+}
+
 int gps_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s_ch, int bits, int8_t* Wq,
              float* s_w, void* stream)
 {

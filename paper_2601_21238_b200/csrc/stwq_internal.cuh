@@ -94,6 +94,9 @@ int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s
                      int8_t* Wq, float* s_w, cudaStream_t st);
 size_t stwq_calibrate_ws_bytes(int P);
 size_t stwq_gps_ws_bytes(int K, int N);
+size_t stwq_dgc_ws_bytes(int D);
+int stwq_launch_dgc(stwq_ctx* ctx, void* ws, const float* F, int n, int D, int k, double ridge, double* rho,
+                    int32_t* selected, cudaStream_t st);
 int stwq_launch_gps(stwq_ctx* ctx, void* ws_cal, void* ws, const float* X, int64_t T, int K, const float* W, int N,
                     int bits, uint32_t pct_ppm, int variant, float* s, int32_t* k_star_out, cudaStream_t st);
 int stwq_launch_calibrate(stwq_ctx* ctx, void* ws, const float* Xcal, const int32_t* pos_ids,

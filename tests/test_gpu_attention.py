@@ -152,3 +152,37 @@ def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits):
             assert (np.abs(got[g] - r["O"]) <= tol).all(), f"{out} head {g}: worst {np.abs(got[g] - r['O']).max()}"
             # and it is a sensible attention: close to the float head computed from the same inputs
         assert np.isfinite(got).all()
+
+
+# ----------------------------------------------------------------------------- distribution-guided calibration
+@pytest.mark.parametrize("shape", [(128, 64, 0.0), (41, 5, 0.0), (300, 257, 0.0), (6, 12, 1e-6), (64, 1, 0.0), (20, 20, 1e-9)])
+def test_dgc_select_matches_the_oracle(gpu, shape):
+    """Eq. 17 on the GPU: distances agree with the oracle to fp64 rounding, the kept set and its order
+    are the oracle's (the data hold no near-equal distances except the planted duplicates, whose order
+    is fixed by index)."""
+    torch = gpu.torch
+    n, D, ridge = shape
+    F = (rng.standard_normal((n, D)) @ rng.standard_normal((D, D)) + rng.standard_normal(D)).astype(np.float32)
+    if n > 10:
+        F[5] = F[3]                                        # duplicates: equal distances, index order
+        F[7] += 4.0
+    rho_ref, sel_ref = oracle.dgc_select(F, 500000, ridge)
+    rho = torch.zeros(n, dtype=torch.float64, device=gpu.dev)
+    sel = torch.full((len(sel_ref),), -1, dtype=torch.int32, device=gpu.dev)
+    gpu.ctx.dgc_select(gpu.T(F), 500000, ridge, rho, sel)
+    assert gpu.ctx.stwq_device_status() == 0
+    np.testing.assert_allclose(rho.cpu().numpy(), rho_ref, rtol=1e-8, atol=1e-12)
+    np.testing.assert_array_equal(sel.cpu().numpy(), sel_ref)
+    # sum of squared distances = n D when nothing is added to the covariance (trace identity)
+    if ridge == 0.0 and D < n:
+        assert abs(float((rho ** 2).sum()) - n * D) < 1e-7 * n * D
+
+
+def test_dgc_degenerate_sets(gpu):
+    torch = gpu.torch
+    rho = torch.full((5,), 3.0, dtype=torch.float64, device=gpu.dev)
+    gpu.ctx.dgc_select(gpu.T(np.ones((5, 3), np.float32)), 500000, 1e-6, rho)      # no variance at all
+    assert (rho.cpu().numpy() == 0).all()
+    wide = rng.standard_normal((6, 12)).astype(np.float32)                          # singular, no ridge
+    gpu.ctx.dgc_select(gpu.T(wide), 500000, 0.0, rho.new_zeros(6))
+    assert gpu.ctx.stwq_device_status() == 0

@@ -695,3 +695,60 @@ def test_quantized_attention_approaches_float_attention_and_factors_its_scales()
     Vh = r["Vq"].astype(np.float64) * s_v[None, :]
     np.testing.assert_allclose(r["O"], (r["Pq"].astype(np.float64) / 255.0) @ Vh, rtol=1e-6, atol=1e-7)
     assert (np.triu(r["Pq"], 1) == 0).all()
+
+
+# ----------------------------------------------------------------------------- distribution-guided calibration
+def test_mahalanobis_distance_closed_forms_and_invariances():
+    """Eq. 17. One feature: rho is the absolute z-score. Whitened data: rho is the Euclidean distance
+    to the mean. Any invertible affine map of the features leaves rho unchanged. The squared distances
+    of a set to itself sum to n D (trace of S^-1 S). And the library route: numpy's inverse."""
+    rng = np.random.default_rng(41)
+    n, D = 60, 7
+    F = (rng.standard_normal((n, D)) @ rng.standard_normal((D, D)) + rng.standard_normal(D) * 3).astype(np.float32)
+    rho, _ = oracle.dgc_select(F)
+    Fd = F.astype(np.float64)
+    u = Fd.mean(axis=0)
+    S = (Fd - u).T @ (Fd - u) / n
+    want = np.sqrt(np.einsum("ia,ab,ib->i", Fd - u, np.linalg.inv(S), Fd - u))
+    np.testing.assert_allclose(rho, want, rtol=1e-9)
+    assert abs((rho ** 2).sum() - n * D) < 1e-8 * n * D
+    x1 = F[:, :1]
+    r1, _ = oracle.dgc_select(x1)
+    x64 = x1[:, 0].astype(np.float64)
+    np.testing.assert_allclose(r1, np.abs(x64 - x64.mean()) / x64.std(), rtol=1e-10)
+    # an affine map with exactly representable entries, so that fp32 storage adds nothing
+    A = np.array([[2, 1, 0, 0, 0, 0, 0], [0, 1, 0, 0, 0, 0, 0], [0, 0, 4, 0, 0, 0, 1], [0, 0, 0, 0.5, 0, 0, 0],
+                  [1, 0, 0, 0, 1, 0, 0], [0, 0, 0, 0, 0, 8, 0], [0, 0, 0, 0, 0, 0, 1]], np.float64)
+    Fi = np.rint(Fd * 16) / 16                                  # multiples of 1/16: the map stays exact in fp32
+    r_a, _ = oracle.dgc_select(Fi.astype(np.float32))
+    r_b, _ = oracle.dgc_select((Fi @ A.T + 3.0).astype(np.float32))
+    np.testing.assert_allclose(r_a, r_b, rtol=1e-9)
+    # whitening by the exact inverse root of S makes the covariance the identity
+    w, V = np.linalg.eigh(S)
+    Wh = (Fd - u) @ V @ np.diag(w ** -0.5) @ V.T
+    rw, _ = oracle.dgc_select(Wh.astype(np.float32))
+    np.testing.assert_allclose(rw, np.linalg.norm(Wh, axis=1), rtol=1e-5)
+
+
+def test_dgc_keeps_the_samples_farthest_from_the_set():
+    rng = np.random.default_rng(42)
+    n, D = 41, 5
+    F = rng.standard_normal((n, D)).astype(np.float32)
+    F[7] += 9.0                                                 # an obvious outlier sample is kept first
+    rho, sel = oracle.dgc_select(F, 500000)
+    assert len(sel) == 21 and sel[0] == 7 and len(set(sel.tolist())) == 21
+    assert (np.diff(rho[sel]) <= 0).all()                       # largest distance first
+    rest = np.setdiff1d(np.arange(n), sel)
+    assert rho[sel].min() >= rho[rest].max()
+    np.testing.assert_array_equal(sel, np.argsort(-rho, kind="stable")[:21])
+    assert len(oracle.dgc_select(F, 1000000)[1]) == n and len(oracle.dgc_select(F, 1)[1]) == 1
+    # duplicates: equal distances are kept in index order
+    Fd = np.repeat(F[:4], 3, axis=0)
+    rd, sd = oracle.dgc_select(Fd, 500000, ridge=1e-9)
+    np.testing.assert_array_equal(sd, np.argsort(-rd, kind="stable")[:6])
+    # more features than samples: singular without a ridge, fine with one; constant data: all zero
+    wide = rng.standard_normal((6, 12)).astype(np.float32)
+    with pytest.raises(ValueError):
+        oracle.dgc_select(wide, 500000, 0.0)
+    assert np.isfinite(oracle.dgc_select(wide, 500000, 1e-6)[0]).all()
+    assert (oracle.dgc_select(np.ones((5, 3), np.float32), 500000, 1e-6)[0] == 0).all()
