@@ -1,5 +1,6 @@
 """Quantized attention matmuls and the quantized KV cache on the GPU against the CPU oracle: cache
-codes, integer accumulators and probability codes of every stage, then the composite call.
+codes, integer accumulators and probability codes of every stage, then the composite call; and the
+calibration-set selection by Mahalanobis distance (Section 4.3).
 Integer results bit-exact; the probability codes (an integer decided by a floating-point softmax)
 may differ by one where the oracle's value before rounding lies within fp32 noise of a tie."""
 import numpy as np

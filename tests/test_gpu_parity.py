@@ -606,6 +606,26 @@ def test_options_reject_values_they_do_not_name(gpu):
         assert L.stwq_set_option(h, opt, 0) == 0
 
 
+def test_peak_probe_and_reserve_layer(gpu):
+    """The int8 peak probe launches, reports the operations it performs and leaves no error behind;
+    stwq_reserve_layer makes a later call allocation-free (the workspace generation stays put)."""
+    torch = gpu.torch
+    ops = gpu.ctx.stwq_probe_int8_peak(64, 3)
+    assert ops == 3 * 64 * 4 * 2 * 256 * 256 * 32
+    ops_all = gpu.ctx.stwq_probe_int8_peak(16)
+    assert ops_all % (16 * 4 * 2 * 256 * 256 * 32) == 0 and ops_all > 0
+    assert gpu.ctx.stwq_device_status() == 0
+    gpu.ctx.stwq_reserve_layer(200, 4096, 1024, 8)
+    gen = gpu.ctx.stwq_workspace_generation()
+    L = wl.scaled(wl.config_layers(4)[1], K=4096, N=1024, P=8)
+    par = prepare(L, samples=2, gps_n=32)
+    X = wl.activations(wl.scaled(L, batch=256))[:200]
+    pos = rng.integers(0, L.P, 200).astype(np.int32)
+    ref = oracle.qlinear(X, pos, par["Wq"], par["s_w"], par["s_tok"], par["s_ch"], par["bias"], 8, 0)
+    np.testing.assert_array_equal(_run_qlinear(gpu, L, par, X, pos, "int32", act=0), ref["acc"])     # splits K: uses the scratch
+    assert gpu.ctx.stwq_workspace_generation() == gen
+
+
 # ----------------------------------------------------------------------------- failure handling
 def test_bounded_wait_expires_and_the_context_stays_usable(gpu):
     """The wait every GEMM kernel uses gives up after the limit, the kernel reports the timeout and
