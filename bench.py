@@ -849,7 +849,7 @@ def main():
     ap.add_argument("--config", type=int, default=3, help="workload family 2..5 (default: the VAR-d30 block)")
     ap.add_argument("--inner", type=int, default=32, help="micro-batches per step (even)")
     ap.add_argument("--calib-samples", type=int, default=32)
-    ap.add_argument("--cpu-rows", type=int, default=4096)
+    ap.add_argument("--cpu-rows", type=int, default=16384)
     ap.add_argument("--ref-rows", type=int, default=128)
     ap.add_argument("--kernel-seconds", type=float, default=0.2, help="timed seconds per kernel in the per-kernel section")
     ap.add_argument("--probe-seconds", type=float, default=0.5)

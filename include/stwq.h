@@ -9,6 +9,9 @@
  *   online    stwq_quantize    X -> int8 codes with the static scales     (Eq. 1, Eq. 2, Section 4.2)
  *   online    qlinear          quantize -> int8 GEMM -> dequantize (+bias, +GELU)
  *   online    qlinear_q        the same from precomputed codes
+ * and, beside the path: chained layers, bf16 activations, the asymmetric quantizer, the dynamic
+ * token-wise baseline, packed 4-bit weights, quantized attention with a quantized KV cache, and the
+ * selection of calibration samples (each documented at its declaration below).
  *
  * Notation: M rows (tokens x batch), K input channels (the paper's n), N output
  * channels (the paper's m), P token positions (the paper's T), b in {8, 6} bits,
