@@ -406,10 +406,24 @@ def decode_rows(ctx, pk, torch, dev, peaks, seconds):
                 ctx.qlinear(Xs[i], pos, Ws[i], s_w, s_tok, s_ch, b, 8, 0, pk.OUT_BF16, Ys[i])
         g = capture(torch, side, rot)
         us = timed_replays(torch, side, g, seconds) / copies * 1e3
+        # the same calls from codes a producer layer has already emitted (no quantize step in the chain)
+        Xqs = [torch.randint(-128, 128, (L.M, L.K), dtype=torch.int8, device=dev) for _ in range(copies)]
+
+        def rot_q():
+            for i in range(copies):
+                ctx.qlinear_q(Xqs[i], pos, Ws[i], s_w, s_tok, b, 0, pk.OUT_BF16, Ys[i])
+        gq = capture(torch, side, rot_q)
+        us_q = timed_replays(torch, side, gq, seconds) / copies * 1e3
+        byts_q = 1.0 * L.M * L.K + L.N * L.K + 2.0 * L.M * L.N
+        del gq, Xqs
         byts = 4.0 * L.M * L.K + L.N * L.K + 2.0 * L.M * L.N
         traffic, note = recorded_traffic("decode_kernel", L.name)
         rows.append({"layer": L.name, "M": L.M, "K": L.K, "N": L.N, "qlinear_us": round(us, 2),
                      "tops": round(L.ops / us / 1e6, 1), "timing": f"CUDA graph, {copies} weight copies rotated (HBM-cold)",
+                     "from_codes": {"qlinear_q_us": round(us_q, 2), "gbs": round(byts_q / us_q / 1e3, 1),
+                                    "frac_of_hbm": round(byts_q / us_q / 1e3 / peaks["hbm_gbs"], 4),
+                                    "note": "qlinear_q on int8 codes (what a chained producer layer emits): the few-row "
+                                            "kernel alone, algorithmic bytes Xq + Wq + Y"},
                      "roofline": {"kernel": "quantize_kernel + decode_kernel (one qlinear call)", "bound": "hbm",
                                   "achieved": round(byts / us / 1e3, 1), "peak": peaks["hbm_gbs"], "unit": "GB/s",
                                   "frac": round(byts / us / 1e3 / peaks["hbm_gbs"], 4),

@@ -329,7 +329,8 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
  * column = position), so that both matmuls read operands whose contraction index is contiguous.
  * d and Tmax multiples of 16, d <= 256.
  *  - kv_append: quantize t_new new key / value rows per head (Knew, Vnew [G, t_new, d] fp32, at positions
- *    pos0 .. pos0 + t_new - 1) into the caches. s_k [P], s_v [d].
+ *    pos0 .. pos0 + t_new - 1) into the caches. s_k [P], s_v [d]. Knew, Kc and Vt 16-byte aligned;
+ *    G <= 65535 (STWQ_ERR_DIM beyond).
  *  - qattention: Q [G, Tq, d] fp32, pos_q [Tq] (shared by all heads), keys / values = the first Tk
  *    positions of the caches, s_q [P], s_kcol [Tk], s_v [d]; O [G, Tq, d] fp32 or bf16. Quantizes Q, runs
  *    both matmuls as batched integer GEMMs on the tensor cores with the softmax-and-quantize pass in

@@ -3,8 +3,8 @@
 // S = Q K^T and O = P V, run on the tensor cores as batched integer GEMMs (qgemm2 with one matrix
 // per head); this file holds what surrounds them:
 //
-//   rowq_kernel               rows of Q, K or V -> int8 codes with static scales (the quantizer of
-//                             Eq. 1 as the linear layers use it: (x * rc[c]) * rt[pos], round to nearest
+//   rowq_rows_kernel,         rows of Q, K or V -> int8 codes with static scales (the quantizer of
+//   rowq_transpose_kernel     Eq. 1 as the linear layers use it: (x * rc[c]) * rt[pos], round to nearest
 //                             even, clamp), written densely (Q), at their position in the key cache, or
 //                             transposed into the value cache;
 //   softmax_quantize_kernel   row softmax of the dequantized scores and the quantizer of the
@@ -20,32 +20,60 @@
 
 namespace {
 
-constexpr int kRowThreads = 128;
+constexpr int kRowThreads = 256;
 
-// One block per row. out index = g * out_gstride + out_row * out_row_stride + c * out_col_stride,
-// out_row = the row's position (caches) or its index within the matrix (dense output).
+// Row-major output (Q codes, key cache): one warp per row, a lane per group of four channels
+// (16-byte loads, 4-byte stores). out index = g * out_gstride + out_row * d + c, out_row = the
+// row's position (key cache) or its index within the matrix (dense output).
 __global__ void __launch_bounds__(kRowThreads)
-rowq_kernel(const float* __restrict__ X, int d, const int32_t* __restrict__ pos_ids, int rows_per_g, int pos0,
-            const float* __restrict__ s_tok, int P, const float* __restrict__ s_ch, int qmin, int qmax,
-            int8_t* __restrict__ out, int64_t out_gstride, int64_t out_row_stride, int64_t out_col_stride,
-            int out_row_from_pos, uint32_t* __restrict__ status)
+rowq_rows_kernel(const float* __restrict__ X, int64_t rows, int d, const int32_t* __restrict__ pos_ids, int rows_per_g,
+                 int pos0, const float* __restrict__ s_tok, int P, int qmin, int qmax, int8_t* __restrict__ out,
+                 int64_t out_gstride, int out_row_from_pos, uint32_t* __restrict__ status)
 {
-    const int64_t r = blockIdx.x;
+    const int lane = threadIdx.x & 31;
+    const int64_t r = (int64_t)blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
+    if (r >= rows) return;
     const int g = (int)(r / rows_per_g);
     const int t = (int)(r - (int64_t)g * rows_per_g);
     const int pos = pos_ids != nullptr ? pos_ids[t] : pos0 + t;
     const bool ok = pos >= 0 && pos < P;
-    if (!ok && threadIdx.x == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
-    const float rt = (s_tok != nullptr && ok) ? __frcp_rn(s_tok[pos]) : 1.0f;
-    const int out_row = out_row_from_pos ? pos : t;
+    if (!ok && lane == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
     if (out_row_from_pos && !ok) return;                  // no slot in the cache for a position outside [0, P)
-    const float* x = X + r * d;
-    int8_t* o = out + (int64_t)g * out_gstride + (int64_t)out_row * out_row_stride;
-    for (int c = threadIdx.x; c < d; c += kRowThreads) {
-        const float rc = s_ch != nullptr ? __frcp_rn(s_ch[c]) : 1.0f;
-        const float u = __fmul_rn(__fmul_rn(x[c], rc), rt);
-        o[(int64_t)c * out_col_stride] = ok ? (int8_t)stwq_code(u, qmin, qmax) : (int8_t)0;
+    const float rt = ok ? __frcp_rn(s_tok[pos]) : 0.0f;
+    const float4* x = reinterpret_cast<const float4*>(X + r * d);
+    uint32_t* o = reinterpret_cast<uint32_t*>(out + (int64_t)g * out_gstride + (int64_t)(out_row_from_pos ? pos : t) * d);
+    for (int c4 = lane; c4 < (d >> 2); c4 += 32) {
+        const float4 v = x[c4];
+        // (x * 1) * rt: no channel scale on queries and keys
+        const int q0 = ok ? stwq_code(__fmul_rn(v.x, rt), qmin, qmax) : 0;
+        const int q1 = ok ? stwq_code(__fmul_rn(v.y, rt), qmin, qmax) : 0;
+        const int q2 = ok ? stwq_code(__fmul_rn(v.z, rt), qmin, qmax) : 0;
+        const int q3 = ok ? stwq_code(__fmul_rn(v.w, rt), qmin, qmax) : 0;
+        o[c4] = (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)(q3 & 0xFF) << 24);
     }
+}
+
+// Value cache, transposed: a block takes 32 consecutive new positions of one head, reads their
+// rows along the channels, and writes each channel's 32 codes as one contiguous run of the cache
+// row Vt[g, c, pos0 + t0 ...]. Per-channel scales, no position scale: (x * rc[c]) * 1.
+__global__ void __launch_bounds__(kRowThreads)
+rowq_transpose_kernel(const float* __restrict__ V, int d, int t_new, int pos0, const float* __restrict__ s_v, int qmin,
+                      int qmax, int8_t* __restrict__ Vt, int Tmax)
+{
+    extern __shared__ int8_t tile[];                      // [d][33]
+    const int g = blockIdx.y;
+    const int t0 = blockIdx.x * 32;
+    const int nt = min(32, t_new - t0);
+    for (int i = threadIdx.x; i < nt * d; i += kRowThreads) {
+        const int tt = i / d, c = i - tt * d;
+        const float rc = __frcp_rn(s_v[c]);
+        const float x = V[((int64_t)g * t_new + t0 + tt) * d + c];
+        tile[c * 33 + tt] = (int8_t)stwq_code(__fmul_rn(x, rc), qmin, qmax);
+    }
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    for (int c = threadIdx.x >> 5; c < d; c += kRowThreads / 32)
+        if (lane < nt) Vt[((int64_t)g * d + c) * Tmax + pos0 + t0 + lane] = tile[c * 33 + lane];
 }
 
 // One warp per row of S [rows, ld] (ld >= Tk, padding columns are written as code 0). Causal: query
@@ -78,13 +106,24 @@ softmax_quantize_kernel(const float* __restrict__ S, int64_t rows, int Tq, int T
     }
 }
 
-int launch_rowq(stwq_ctx* ctx, const float* X, int64_t rows, int d, const int32_t* pos_ids, int rows_per_g, int pos0,
-                const float* s_tok, int P, const float* s_ch, int bits, int8_t* out, int64_t gs, int64_t rs, int64_t cs,
-                int from_pos, cudaStream_t st)
+int launch_rows(stwq_ctx* ctx, const float* X, int64_t rows, int d, const int32_t* pos_ids, int rows_per_g, int pos0,
+                const float* s_tok, int P, int bits, int8_t* out, int64_t gs, int from_pos, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    rowq_kernel<<<(unsigned)rows, kRowThreads, 0, st>>>(X, d, pos_ids, rows_per_g, pos0, s_tok, P, s_ch, qmin, qmax, out, gs,
-                                                        rs, cs, from_pos, ctx->d_status);
+    const int64_t blocks = (rows + kRowThreads / 32 - 1) / (kRowThreads / 32);
+    rowq_rows_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(X, rows, d, pos_ids, rows_per_g, pos0, s_tok, P, qmin, qmax, out,
+                                                               gs, from_pos, ctx->d_status);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
+}
+
+int launch_transpose(stwq_ctx* ctx, const float* V, int G, int t_new, int d, int pos0, const float* s_v, int bits, int8_t* Vt,
+                     int Tmax, cudaStream_t st)
+{
+    const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+    rowq_transpose_kernel<<<dim3((unsigned)((t_new + 31) / 32), (unsigned)G), kRowThreads, (size_t)d * 33, st>>>(
+        V, d, t_new, pos0, s_v, qmin, qmax, Vt, Tmax);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
@@ -148,15 +187,15 @@ int kv_append(stwq_ctx* ctx, const float* Knew, const float* Vnew, int G, int t_
 {
     if (!ctx || !Knew || !Vnew || !s_k || !s_v || !Kc || !Vt) return STWQ_ERR_NULL;
     if (G <= 0 || t_new <= 0 || d <= 0 || Tmax <= 0 || P <= 0 || pos0 < 0) return STWQ_ERR_DIM;
-    if ((int64_t)pos0 + t_new > Tmax || (int64_t)pos0 + t_new > P) return STWQ_ERR_DIM;
+    if ((int64_t)pos0 + t_new > Tmax || (int64_t)pos0 + t_new > P || G > 65535) return STWQ_ERR_DIM;
     if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
-    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Kc) || !aligned16(Vt)) return STWQ_ERR_ALIGN;
+    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Knew) || !aligned16(Kc) || !aligned16(Vt)) return STWQ_ERR_ALIGN;
     DevGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)G * t_new;
-    int rc = launch_rowq(ctx, Knew, rows, d, nullptr, t_new, pos0, s_k, P, nullptr, bits, Kc, (int64_t)Tmax * d, d, 1, 1, st);
+    int rc = launch_rows(ctx, Knew, rows, d, nullptr, t_new, pos0, s_k, P, bits, Kc, (int64_t)Tmax * d, 1, st);
     if (rc != STWQ_OK) return rc;
-    return launch_rowq(ctx, Vnew, rows, d, nullptr, t_new, pos0, nullptr, P, s_v, bits, Vt, (int64_t)d * Tmax, 1, Tmax, 1, st);
+    return launch_transpose(ctx, Vnew, G, t_new, d, pos0, s_v, bits, Vt, Tmax, st);
 }
 
 int stwq_reserve_attention(stwq_ctx* ctx, int G, int Tq, int Tk, int d)
@@ -189,7 +228,7 @@ int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int T
     w = attn_layout(ctx->ws_attn, G, Tq, Tk_pad, d);
 
     // queries -> codes with their per-position scales
-    rc = launch_rowq(ctx, Q, (int64_t)G * Tq, d, pos_q, Tq, 0, s_q, P, nullptr, bits, w.Qq, (int64_t)Tq * d, d, 1, 0, st);
+    rc = launch_rows(ctx, Q, (int64_t)G * Tq, d, pos_q, Tq, 0, s_q, P, bits, w.Qq, (int64_t)Tq * d, 0, st);
     if (rc != STWQ_OK) return rc;
     // key-column scales, padded with zeros to the 16-column pitch of the score matrix
     cudaError_t e = cudaMemsetAsync(w.skcol, 0, (size_t)Tk_pad * 4, st);

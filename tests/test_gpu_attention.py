@@ -74,6 +74,29 @@ def test_kv_append_writes_the_oracles_codes_into_both_cache_layouts(gpu, bits):
         gpu.ctx.kv_append(gpu.T(K[:, :4]), gpu.T(V[:, :4]), Tmax - 2, gpu.T(s_k), gpu.T(s_v), bits, Kc, Vt)
 
 
+@pytest.mark.parametrize("case", [(2, 70, 64, 3, 96), (1, 33, 16, 31, 64), (5, 256, 128, 0, 256)])
+def test_kv_append_blocks_of_positions_at_an_odd_offset(gpu, case):
+    """Several 32-position tiles with a ragged last one, starting at a cache column that is not a
+    multiple of 4: the transposed value cache is written in runs along the positions."""
+    torch = gpu.torch
+    G, t_new, d, pos0, Tmax = case
+    P = Tmax
+    _, K, V, _, _, s_v = _head_data(G, t_new, d, P)
+    s_k = rng.uniform(0.01, 0.05, P).astype(np.float32)
+    Kc = torch.full((G, Tmax, d), -5, dtype=torch.int8, device=gpu.dev)
+    Vt = torch.full((G, d, Tmax), -5, dtype=torch.int8, device=gpu.dev)
+    gpu.ctx.kv_append(gpu.T(K), gpu.T(V), pos0, gpu.T(s_k), gpu.T(s_v), 8, Kc, Vt)
+    assert gpu.ctx.stwq_device_status() == 0
+    pos = np.arange(pos0, pos0 + t_new, dtype=np.int32)
+    kc, vt = Kc.cpu().numpy(), Vt.cpu().numpy()
+    for g in range(G):
+        np.testing.assert_array_equal(kc[g, pos0:pos0 + t_new], oracle.quantize(K[g], pos, None, s_k, 8))
+        want_v = oracle.quantize(V[g], np.zeros(t_new, np.int32), s_v, np.ones(1, np.float32), 8)
+        np.testing.assert_array_equal(vt[g, :, pos0:pos0 + t_new], want_v.T)
+    assert (kc[:, :pos0] == -5).all() and (kc[:, pos0 + t_new:] == -5).all()
+    assert (vt[:, :, :pos0] == -5).all() and (vt[:, :, pos0 + t_new:] == -5).all()
+
+
 @pytest.mark.parametrize("bits", [8, 6])
 @pytest.mark.parametrize("shape", [(5, 37, 37, True), (3, 1, 50, False), (2, 300, 300, True), (4, 20, 129, True)])
 def test_softmax_quantizer_codes(gpu, shape, bits):
