@@ -760,11 +760,25 @@ def other_configs(ctx, pk, torch, dev, peaks, args):
     ctx.stwq_reserve_attention(G, T, T, d)
     t_app = graph_us(lambda: ctx.kv_append(Kn, Vn, 0, s_k, s_v, 8, Kc, Vt), 1)
     t_att = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    ctx.stwq_set_option(pk.OPT_VARIANT, 9)
+    try:
+        ctx.stwq_reserve_attention(G, T, T, d)
+        t_staged = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    finally:
+        ctx.stwq_set_option(pk.OPT_VARIANT, 0)
+    # what a head must move: Q (fp32 in, codes out and back in), both code caches once, O
+    att_bytes = G * T * d * (4 + 1 + 1 + 2) + 2 * G * T * d
+    app_bytes = 2 * G * T * d * (4 + 1)
     out["attention_var_d16"] = {"heads": G, "positions": T, "head_dim": d, "kv_append_us": round(t_app, 1),
+                                "kv_append_frac_of_hbm": round(app_bytes / t_app / 1e3 / peaks["hbm_gbs"], 3),
                                 "qattention_us": round(t_att, 1),
+                                "qattention_three_stages_us": round(t_staged, 1),
                                 "matmul_tops": round(2 * 2.0 * G * T * T * d / t_att / 1e6, 1),
-                                "note": "Q K^T and P V as batched int8 GEMMs (unfused: scores and probability codes "
-                                        "pass through workspace); ops counted for the full T x T matrices"}
+                                "min_bytes_frac_of_hbm": round(att_bytes / t_att / 1e3 / peaks["hbm_gbs"], 3),
+                                "note": "one kernel per 128 queries of a head: Q K^T, softmax, probability codes and P V "
+                                        "on the SM (keys walked twice); three_stages = batched int8 GEMMs with scores and "
+                                        "codes in workspace; ops counted for the full T x T matrices, bytes = Q fp32 + "
+                                        "Q codes twice + both code caches + O bf16"}
     del Q, Kn, Vn, Kc, Vt, O
     ctx.check_device_status()
     return out

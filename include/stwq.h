@@ -329,13 +329,17 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
  * column = position), so that both matmuls read operands whose contraction index is contiguous.
  * d and Tmax multiples of 16, d <= 256.
  *  - kv_append: quantize t_new new key / value rows per head (Knew, Vnew [G, t_new, d] fp32, at positions
- *    pos0 .. pos0 + t_new - 1) into the caches. s_k [P], s_v [d]. Knew, Kc and Vt 16-byte aligned;
- *    G <= 65535 (STWQ_ERR_DIM beyond).
+ *    pos0 .. pos0 + t_new - 1) into the caches. s_k [P], s_v [d]. Knew, Vnew, s_v, Kc and Vt
+ *    16-byte aligned (STWQ_ERR_ALIGN otherwise).
  *  - qattention: Q [G, Tq, d] fp32, pos_q [Tq] (shared by all heads), keys / values = the first Tk
- *    positions of the caches, s_q [P], s_kcol [Tk], s_v [d]; O [G, Tq, d] fp32 or bf16. Quantizes Q, runs
- *    both matmuls as batched integer GEMMs on the tensor cores with the softmax-and-quantize pass in
- *    between. The scores (fp32) and the codes live in context workspace (stwq_reserve_attention sizes
- *    it ahead of time; growth during stream capture is refused like everywhere else).
+ *    positions of the caches, s_q [P], s_kcol [Tk], s_v [d]; O [G, Tq, d] fp32 or bf16. Quantizes Q, then
+ *    one kernel per 128 queries of a head runs both matmuls on the tensor cores with the softmax and the
+ *    quantizer of the probabilities in between, scores and probability codes staying on the SM (the keys
+ *    are walked twice: row maxima and sums first, codes second). STWQ_OPT_VARIANT 9 runs the three stages
+ *    as separate kernels instead (batched integer GEMMs with the scores, fp32, and the codes in context
+ *    workspace). The two differ only where a probability sits on a rounding tie of its code.
+ *    stwq_reserve_attention sizes the workspace ahead of time for the variant in force; growth during
+ *    stream capture is refused like everywhere else.
  *  - qattn_softmax_quantize, qattn_pv: the second and third stage on their own (S [rows, ld] fp32 with
  *    rows = G Tq and ld >= Tk a multiple of 16; Pq [G, Tq, Tk_pad] codes; STWQ_OUT_INT32 stores acc_pv).
  */
@@ -405,7 +409,8 @@ int stwq_selftest_wait_expiry(stwq_ctx* ctx, uint64_t* waited_ns, void* stream);
  * STWQ_OPT_TILE_N: 128 or 256 = tile width of the CTA-pair GEMM.
  * STWQ_OPT_VARIANT: 1 / 2 = CTA-pair GEMM epilogue through staged TMA stores / straight from
  *   registers; 5 = ordinary launches instead of programmatic dependent ones; 7 / 8 = the
- *   register-streaming / the TMA-ring quantize kernel.
+ *   register-streaming / the TMA-ring quantize kernel; 9 = qattention as three separate stages (batched
+ *   GEMM, softmax-and-quantize pass, batched GEMM) instead of the one-kernel head.
  * STWQ_OPT_KSPLIT (-1 .. 64): n > 0 = cut the tiles of the last wave of the CTA-pair GEMM (every work item of
  *   the few-row kernel) into n ranges of K; -1 = the few-row kernel never cuts. The CTA-pair GEMM
  *   cuts only on request.

@@ -228,7 +228,7 @@ int stwq_set_option(stwq_ctx* ctx, int option, int value)
         ctx->force_bn = value;
         return STWQ_OK;
     }
-    if (option == STWQ_OPT_VARIANT && (value == 0 || value == 1 || value == 2 || value == 5 || value == 7 || value == 8)) {
+    if (option == STWQ_OPT_VARIANT && (value == 0 || value == 1 || value == 2 || value == 5 || value == 7 || value == 8 || value == 9)) {
         ctx->debug = value;
         return STWQ_OK;
     }

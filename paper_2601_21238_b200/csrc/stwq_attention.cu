@@ -22,58 +22,88 @@ namespace {
 
 constexpr int kRowThreads = 256;
 
-// Row-major output (Q codes, key cache): one warp per row, a lane per group of four channels
-// (16-byte loads, 4-byte stores). out index = g * out_gstride + out_row * d + c, out_row = the
-// row's position (key cache) or its index within the matrix (dense output).
+__device__ __forceinline__ uint32_t pack_codes(int q0, int q1, int q2, int q3)
+{
+    return (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)(q3 & 0xFF) << 24);
+}
+
+// Row-major output (Q codes, key cache): a thread per group of four channels (a 16-byte load, a
+// 4-byte store), consecutive threads along the row and on into the next one.
+// out index = g * out_gstride + out_row * d + c, out_row = the row's position (key cache) or its
+// index within the matrix (dense output).
 __global__ void __launch_bounds__(kRowThreads)
-rowq_rows_kernel(const float* __restrict__ X, int64_t rows, int d, const int32_t* __restrict__ pos_ids, int rows_per_g,
+rowq_rows_kernel(const float4* __restrict__ X, int64_t n_vec, int d4, const int32_t* __restrict__ pos_ids, int rows_per_g,
                  int pos0, const float* __restrict__ s_tok, int P, int qmin, int qmax, int8_t* __restrict__ out,
                  int64_t out_gstride, int out_row_from_pos, uint32_t* __restrict__ status)
 {
-    const int lane = threadIdx.x & 31;
-    const int64_t r = (int64_t)blockIdx.x * (kRowThreads / 32) + (threadIdx.x >> 5);
-    if (r >= rows) return;
+    const int64_t i = (int64_t)blockIdx.x * kRowThreads + threadIdx.x;
+    if (i >= n_vec) return;
+    const int64_t r = i / d4;
+    const int c4 = (int)(i - r * d4);
     const int g = (int)(r / rows_per_g);
     const int t = (int)(r - (int64_t)g * rows_per_g);
     const int pos = pos_ids != nullptr ? pos_ids[t] : pos0 + t;
     const bool ok = pos >= 0 && pos < P;
-    if (!ok && lane == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+    if (!ok && c4 == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
     if (out_row_from_pos && !ok) return;                  // no slot in the cache for a position outside [0, P)
-    const float rt = ok ? __frcp_rn(s_tok[pos]) : 0.0f;
-    const float4* x = reinterpret_cast<const float4*>(X + r * d);
-    uint32_t* o = reinterpret_cast<uint32_t*>(out + (int64_t)g * out_gstride + (int64_t)(out_row_from_pos ? pos : t) * d);
-    for (int c4 = lane; c4 < (d >> 2); c4 += 32) {
-        const float4 v = x[c4];
+    uint32_t packed = 0;
+    if (ok) {
+        const float rt = __frcp_rn(s_tok[pos]);
+        const float4 v = X[i];
         // (x * 1) * rt: no channel scale on queries and keys
-        const int q0 = ok ? stwq_code(__fmul_rn(v.x, rt), qmin, qmax) : 0;
-        const int q1 = ok ? stwq_code(__fmul_rn(v.y, rt), qmin, qmax) : 0;
-        const int q2 = ok ? stwq_code(__fmul_rn(v.z, rt), qmin, qmax) : 0;
-        const int q3 = ok ? stwq_code(__fmul_rn(v.w, rt), qmin, qmax) : 0;
-        o[c4] = (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)(q3 & 0xFF) << 24);
+        packed = pack_codes(stwq_code(__fmul_rn(v.x, rt), qmin, qmax), stwq_code(__fmul_rn(v.y, rt), qmin, qmax),
+                            stwq_code(__fmul_rn(v.z, rt), qmin, qmax), stwq_code(__fmul_rn(v.w, rt), qmin, qmax));
     }
+    uint32_t* o = reinterpret_cast<uint32_t*>(out + (int64_t)g * out_gstride + (int64_t)(out_row_from_pos ? pos : t) * (d4 * 4));
+    o[c4] = packed;
 }
 
-// Value cache, transposed: a block takes 32 consecutive new positions of one head, reads their
-// rows along the channels, and writes each channel's 32 codes as one contiguous run of the cache
-// row Vt[g, c, pos0 + t0 ...]. Per-channel scales, no position scale: (x * rc[c]) * 1.
+// Value cache, transposed: a thread takes four consecutive new positions and four consecutive
+// channels (four 16-byte loads), turns the 4 x 4 block of codes in registers, and writes each
+// channel's four positions as one word of the cache row Vt[g, c, pos0 + t ...] (single bytes at a
+// ragged end or when the run does not start on a 4-byte boundary). Eight consecutive threads
+// cover 32 positions of the same channels, so a warp writes full 32-byte sectors.
+// Per-channel scales, no position scale: (x * rc[c]) * 1.
 __global__ void __launch_bounds__(kRowThreads)
-rowq_transpose_kernel(const float* __restrict__ V, int d, int t_new, int pos0, const float* __restrict__ s_v, int qmin,
-                      int qmax, int8_t* __restrict__ Vt, int Tmax)
+rowq_transpose_kernel(const float4* __restrict__ V, int G, int d4, int t_new, int pos0, const float4* __restrict__ s_v,
+                      int qmin, int qmax, int8_t* __restrict__ Vt, int Tmax)
 {
-    extern __shared__ int8_t tile[];                      // [d][33]
-    const int g = blockIdx.y;
-    const int t0 = blockIdx.x * 32;
-    const int nt = min(32, t_new - t0);
-    for (int i = threadIdx.x; i < nt * d; i += kRowThreads) {
-        const int tt = i / d, c = i - tt * d;
-        const float rc = __frcp_rn(s_v[c]);
-        const float x = V[((int64_t)g * t_new + t0 + tt) * d + c];
-        tile[c * 33 + tt] = (int8_t)stwq_code(__fmul_rn(x, rc), qmin, qmax);
+    const int tiles = (t_new + 31) >> 5;
+    const int64_t i = (int64_t)blockIdx.x * kRowThreads + threadIdx.x;
+    if (i >= (int64_t)G * tiles * d4 * 8) return;
+    const int tq = (int)(i & 7);
+    int64_t rest = i >> 3;
+    const int c4 = (int)(rest % d4);
+    rest /= d4;
+    const int tile = (int)(rest % tiles);
+    const int g = (int)(rest / tiles);
+    const int t = tile * 32 + tq * 4;                     // first of this thread's four positions
+    if (t >= t_new) return;
+    const int nt = min(4, t_new - t);
+    const float4 sv = s_v[c4];
+    const float rc[4] = {__frcp_rn(sv.x), __frcp_rn(sv.y), __frcp_rn(sv.z), __frcp_rn(sv.w)};
+    int q[4][4];                                          // [position][channel]
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nt) v = V[((int64_t)g * t_new + t + r) * d4 + c4];
+        q[r][0] = stwq_code(__fmul_rn(v.x, rc[0]), qmin, qmax);
+        q[r][1] = stwq_code(__fmul_rn(v.y, rc[1]), qmin, qmax);
+        q[r][2] = stwq_code(__fmul_rn(v.z, rc[2]), qmin, qmax);
+        q[r][3] = stwq_code(__fmul_rn(v.w, rc[3]), qmin, qmax);
     }
-    __syncthreads();
-    const int lane = threadIdx.x & 31;
-    for (int c = threadIdx.x >> 5; c < d; c += kRowThreads / 32)
-        if (lane < nt) Vt[((int64_t)g * d + c) * Tmax + pos0 + t0 + lane] = tile[c * 33 + lane];
+    int8_t* o = Vt + ((int64_t)g * d4 * 4 + c4 * 4) * Tmax + pos0 + t;
+    const bool word = nt == 4 && ((pos0 + t) & 3) == 0;   // Tmax is a multiple of 16, the base 16-byte aligned
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+        if (word) {
+            *reinterpret_cast<uint32_t*>(o + (int64_t)c * Tmax) = pack_codes(q[0][c], q[1][c], q[2][c], q[3][c]);
+        } else {
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (r < nt) o[(int64_t)c * Tmax + r] = (int8_t)q[r][c];
+        }
+    }
 }
 
 // One warp per row of S [rows, ld] (ld >= Tk, padding columns are written as code 0). Causal: query
@@ -110,9 +140,12 @@ int launch_rows(stwq_ctx* ctx, const float* X, int64_t rows, int d, const int32_
                 const float* s_tok, int P, int bits, int8_t* out, int64_t gs, int from_pos, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    const int64_t blocks = (rows + kRowThreads / 32 - 1) / (kRowThreads / 32);
-    rowq_rows_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(X, rows, d, pos_ids, rows_per_g, pos0, s_tok, P, qmin, qmax, out,
-                                                               gs, from_pos, ctx->d_status);
+    const int64_t n_vec = rows * (d / 4);
+    const int64_t blocks = (n_vec + kRowThreads - 1) / kRowThreads;
+    if (blocks > 0x7fffffff) return STWQ_ERR_DIM;
+    rowq_rows_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(reinterpret_cast<const float4*>(X), n_vec, d / 4, pos_ids,
+                                                               rows_per_g, pos0, s_tok, P, qmin, qmax, out, gs, from_pos,
+                                                               ctx->d_status);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
@@ -122,8 +155,11 @@ int launch_transpose(stwq_ctx* ctx, const float* V, int G, int t_new, int d, int
                      int Tmax, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    rowq_transpose_kernel<<<dim3((unsigned)((t_new + 31) / 32), (unsigned)G), kRowThreads, (size_t)d * 33, st>>>(
-        V, d, t_new, pos0, s_v, qmin, qmax, Vt, Tmax);
+    const int64_t n_thr = (int64_t)G * ((t_new + 31) / 32) * (d / 4) * 8;
+    const int64_t blocks = (n_thr + kRowThreads - 1) / kRowThreads;
+    if (blocks > 0x7fffffff) return STWQ_ERR_DIM;
+    rowq_transpose_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(reinterpret_cast<const float4*>(V), G, d / 4, t_new, pos0,
+                                                                    reinterpret_cast<const float4*>(s_v), qmin, qmax, Vt, Tmax);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
@@ -158,15 +194,16 @@ struct AttnWs {
     float* delta_p;
     size_t bytes;
 };
-AttnWs attn_layout(void* base, int64_t G, int64_t Tq, int64_t Tk_pad, int64_t d)
+// staged = false: the one-kernel head keeps scores and probability codes on the SM
+AttnWs attn_layout(void* base, int64_t G, int64_t Tq, int64_t Tk_pad, int64_t d, bool staged)
 {
     AttnWs w;
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off = (size_t)round_up((int64_t)(off + n), 256); return o; };
     const size_t oq = take((size_t)(G * Tq * d));
-    const size_t os = take((size_t)(G * Tq * Tk_pad) * 4);
-    const size_t op = take((size_t)(G * Tq * Tk_pad));
-    const size_t ok = take((size_t)Tk_pad * 4);
+    const size_t os = take(staged ? (size_t)(G * Tq * Tk_pad) * 4 : 0);
+    const size_t op = take(staged ? (size_t)(G * Tq * Tk_pad) : 0);
+    const size_t ok = take((size_t)round_up(Tk_pad, 128) * 4);
     const size_t od = take(256);
     uint8_t* b = static_cast<uint8_t*>(base);
     w.Qq = reinterpret_cast<int8_t*>(b + oq);
@@ -187,9 +224,10 @@ int kv_append(stwq_ctx* ctx, const float* Knew, const float* Vnew, int G, int t_
 {
     if (!ctx || !Knew || !Vnew || !s_k || !s_v || !Kc || !Vt) return STWQ_ERR_NULL;
     if (G <= 0 || t_new <= 0 || d <= 0 || Tmax <= 0 || P <= 0 || pos0 < 0) return STWQ_ERR_DIM;
-    if ((int64_t)pos0 + t_new > Tmax || (int64_t)pos0 + t_new > P || G > 65535) return STWQ_ERR_DIM;
+    if ((int64_t)pos0 + t_new > Tmax || (int64_t)pos0 + t_new > P) return STWQ_ERR_DIM;
     if (bits != 8 && bits != 6) return STWQ_ERR_BITS;
-    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Knew) || !aligned16(Kc) || !aligned16(Vt)) return STWQ_ERR_ALIGN;
+    if ((d & 15) != 0 || (Tmax & 15) != 0 || !aligned16(Knew) || !aligned16(Vnew) || !aligned16(s_v) || !aligned16(Kc) || !aligned16(Vt))
+        return STWQ_ERR_ALIGN;
     DevGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t rows = (int64_t)G * t_new;
@@ -203,7 +241,7 @@ int stwq_reserve_attention(stwq_ctx* ctx, int G, int Tq, int Tk, int d)
     if (!ctx) return STWQ_ERR_NULL;
     if (G <= 0 || Tq <= 0 || Tk <= 0 || d <= 0) return STWQ_ERR_DIM;
     DevGuard g(ctx->device);
-    const AttnWs w = attn_layout(nullptr, G, Tq, round_up(Tk, 16), d);
+    const AttnWs w = attn_layout(nullptr, G, Tq, round_up(Tk, 16), d, ctx->debug == 9);
     return stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, nullptr, 0);
 }
 
@@ -222,18 +260,23 @@ int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int T
     DevGuard g(ctx->device);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t Tk_pad = round_up(Tk, 16);
-    AttnWs w = attn_layout(nullptr, G, Tq, Tk_pad, d);
+    const bool staged = ctx->debug == 9;                  // the three stages as separate kernels
+    AttnWs w = attn_layout(nullptr, G, Tq, Tk_pad, d, staged);
     int rc = stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, st, 0);
     if (rc != STWQ_OK) return rc;
-    w = attn_layout(ctx->ws_attn, G, Tq, Tk_pad, d);
+    w = attn_layout(ctx->ws_attn, G, Tq, Tk_pad, d, staged);
 
     // queries -> codes with their per-position scales
     rc = launch_rows(ctx, Q, (int64_t)G * Tq, d, pos_q, Tq, 0, s_q, P, bits, w.Qq, (int64_t)Tq * d, 0, st);
     if (rc != STWQ_OK) return rc;
-    // key-column scales, padded with zeros to the 16-column pitch of the score matrix
-    cudaError_t e = cudaMemsetAsync(w.skcol, 0, (size_t)Tk_pad * 4, st);
+    // key-column scales, padded with zeros (to the 16-column pitch of the score matrix; to whole
+    // chunks of 128 keys for the one-kernel head)
+    cudaError_t e = cudaMemsetAsync(w.skcol, 0, (size_t)round_up(Tk_pad, 128) * 4, st);
     if (e == cudaSuccess) e = cudaMemcpyAsync(w.skcol, s_kcol, (size_t)Tk * 4, cudaMemcpyDeviceToDevice, st);
     if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    if (!staged)
+        return stwq_launch_qattn_fused(ctx, w.Qq, pos_q, G, Tq, Tk, d, Tmax, Kc, Vt, s_q, w.skcol, s_v, P, bits, causal,
+                                       out_dtype, O, st);
     // S = dequantized Q K^T, one matrix per head: rows scaled by s_q[pos], columns by s_kcol
     stwq_batch bq = {G, (int64_t)d, (int64_t)Tmax * d, 0, 1, 0};
     rc = stwq_launch_qgemm2(ctx, w.Qq, pos_q, Tq, d, (int)Tk_pad, Kc, w.skcol, s_q, P, nullptr, STWQ_ACT_NONE, STWQ_OUT_F32,

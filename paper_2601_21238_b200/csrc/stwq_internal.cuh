@@ -44,6 +44,7 @@ struct stwq_ctx {
     int force_ksplit;          // tuning: 0 = choose, else the number of K ranges of the few-row path
     uint64_t ws_generation;    // bumped whenever a workspace buffer is (re)allocated
     int probe_configured;      // the peak-probe kernel has its shared-memory attribute set
+    int attn_configured;       // so has the one-kernel attention head
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
 };
 
@@ -95,6 +96,9 @@ int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s
 size_t stwq_calibrate_ws_bytes(int P);
 size_t stwq_gps_ws_bytes(int K, int N);
 size_t stwq_dgc_ws_bytes(int D);
+int stwq_launch_qattn_fused(stwq_ctx* ctx, const int8_t* Qq, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
+                            const int8_t* Kc, const int8_t* Vt, const float* s_q, const float* s_kcol_pad, const float* s_v,
+                            int P, int bits, int causal, int out_dtype, void* O, cudaStream_t st);
 int stwq_launch_dgc(stwq_ctx* ctx, void* ws, const float* F, int n, int D, int k, double ridge, double* rho,
                     int32_t* selected, cudaStream_t st);
 int stwq_launch_gps(stwq_ctx* ctx, void* ws_cal, void* ws, const float* X, int64_t T, int K, const float* W, int N,

@@ -143,12 +143,27 @@ def test_probability_value_matmul_is_exact(gpu, shape):
             assert_close(O[g].float().cpu().numpy(), {"Y": Y, "mag": mag, "act": 0}, rtol, f"P V {out}")
 
 
+@pytest.mark.parametrize("variant", [0, 9])
 @pytest.mark.parametrize("bits", [8, 6])
-@pytest.mark.parametrize("shape", [(4, 37, 37, 64, True), (2, 1, 50, 64, False), (3, 129, 129, 128, True), (2, 40, 200, 48, True)])
-def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits):
+@pytest.mark.parametrize("shape", [(4, 37, 37, 64, True), (2, 1, 50, 64, False), (3, 129, 129, 128, True), (2, 40, 200, 48, True),
+                                   (2, 680, 680, 64, True), (1, 300, 420, 128, False), (1, 200, 300, 256, True),
+                                   (2, 130, 260, 16, True), (3, 1, 300, 64, False), (1, 256, 256, 144, True)])
+def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits, variant):
     """The composite call against the oracle's head: the output differs from the oracle's only through
     probability codes that sit on a rounding tie (each such code moves O by delta_p |Vq| s_v), so O is
-    compared with the usual tolerance plus that allowance for a handful of flips per row."""
+    compared with the usual tolerance plus that allowance for a handful of flips per row. Both forms of
+    the call are held to it: the one-kernel head (several chunks of 128 keys, query tiles with a ragged
+    last one, head dimensions below, at and above one 128-byte block) and the three separate stages."""
+    torch = gpu.torch
+    G, Tq, Tk, d, causal = shape
+    gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
+    try:
+        _check_qattention(gpu, shape, bits)
+    finally:
+        gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, 0)
+
+
+def _check_qattention(gpu, shape, bits):
     torch = gpu.torch
     G, Tq, Tk, d, causal = shape
     P, Tmax = Tk + 3, (Tk + 15) // 16 * 16 + 16
@@ -176,6 +191,38 @@ def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits):
             assert (np.abs(got[g] - r["O"]) <= tol).all(), f"{out} head {g}: worst {np.abs(got[g] - r['O']).max()}"
             # and it is a sensible attention: close to the float head computed from the same inputs
         assert np.isfinite(got).all()
+
+
+@pytest.mark.parametrize("shape", [(3, 333, 333, 64, True), (2, 100, 700, 96, False)])
+def test_one_kernel_head_agrees_with_the_separate_stages(gpu, shape):
+    """Same codes except on rounding ties: the outputs of the two forms differ by at most a few
+    flipped probability codes per row, and most rows agree to the last rounding of the dequantizer."""
+    torch = gpu.torch
+    G, Tq, Tk, d, causal = shape
+    P, Tmax = Tk, (Tk + 15) // 16 * 16
+    Q, K, V, s_q, s_k, s_v = _head_data(G, Tk, d, P)
+    Q = Q[:, Tk - Tq:]
+    pos_q = np.arange(Tk - Tq, Tk, dtype=np.int32)
+    s_kcol = (s_k[:Tk] * np.float32(1.0 / np.sqrt(d))).astype(np.float32)
+    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=gpu.dev)
+    Vt = torch.zeros((G, d, Tmax), dtype=torch.int8, device=gpu.dev)
+    gpu.ctx.kv_append(gpu.T(K), gpu.T(V), 0, gpu.T(s_k), gpu.T(s_v), 8, Kc, Vt)
+    outs = []
+    for variant in (0, 9):
+        gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
+        try:
+            O = torch.full((G, Tq, d), -3, dtype=torch.float32, device=gpu.dev)
+            gpu.ctx.qattention(gpu.T(Q), gpu.T(pos_q), Tk, Kc, Vt, gpu.T(s_q), gpu.T(s_kcol), gpu.T(s_v), 8, causal,
+                               gpu.B.OUT_F32, O)
+            outs.append(O.cpu().numpy().astype(np.float64))
+        finally:
+            gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, 0)
+    assert gpu.ctx.stwq_device_status() == 0
+    diff = np.abs(outs[0] - outs[1])
+    flip = (1.0 / 255) * 128 * s_v[None, None, :].astype(np.float64)          # one code moved by one step
+    assert (diff <= 4 * flip + 1e-6 * np.abs(outs[1])).all()
+    rows_equal = (diff <= 1e-6 * np.abs(outs[1]) + 1e-12).all(axis=2).mean()
+    assert rows_equal > 0.9, rows_equal
 
 
 # ----------------------------------------------------------------------------- distribution-guided calibration

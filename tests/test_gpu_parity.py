@@ -598,7 +598,7 @@ def test_forced_kernel_variants_match_the_oracle(gpu, option, value):
 
 def test_options_reject_values_they_do_not_name(gpu):
     L, h = gpu.ctx.lib, gpu.ctx.handle
-    for opt, bad in ((gpu.B.OPT_TILE_N, 64), (gpu.B.OPT_TILE_N, 192), (gpu.B.OPT_VARIANT, 3), (gpu.B.OPT_VARIANT, 9),
+    for opt, bad in ((gpu.B.OPT_TILE_N, 64), (gpu.B.OPT_TILE_N, 192), (gpu.B.OPT_VARIANT, 3), (gpu.B.OPT_VARIANT, 10),
                      (gpu.B.OPT_KSPLIT, -2), (gpu.B.OPT_KSPLIT, 65), (gpu.B.OPT_GEMM_PATH, 4),
                      (gpu.B.OPT_WAIT_LIMIT_MS, 0)):
         assert L.stwq_set_option(h, opt, bad) == -2
