@@ -106,6 +106,13 @@ rowq_transpose_kernel(const float4* __restrict__ V, int G, int d4, int t_new, in
     }
 }
 
+// Column scales of the keys, followed by zeros up to the padded length.
+__global__ void pad_scales_kernel(const float* __restrict__ src, int n, int n_pad, float* __restrict__ dst)
+{
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_pad) dst[i] = i < n ? src[i] : 0.0f;
+}
+
 // One warp per row of S [rows, ld] (ld >= Tk, padding columns are written as code 0). Causal: query
 // i of a matrix (i = row % Tq) sees the keys j <= i + (Tk - Tq).
 __global__ void __launch_bounds__(256)
@@ -200,7 +207,7 @@ AttnWs attn_layout(void* base, int64_t G, int64_t Tq, int64_t Tk_pad, int64_t d,
     AttnWs w;
     size_t off = 0;
     auto take = [&](size_t n) { size_t o = off; off = (size_t)round_up((int64_t)(off + n), 256); return o; };
-    const size_t oq = take((size_t)(G * Tq * d));
+    const size_t oq = take(staged ? (size_t)(G * Tq * d) : 0);
     const size_t os = take(staged ? (size_t)(G * Tq * Tk_pad) * 4 : 0);
     const size_t op = take(staged ? (size_t)(G * Tq * Tk_pad) : 0);
     const size_t ok = take((size_t)round_up(Tk_pad, 128) * 4);
@@ -266,17 +273,19 @@ int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int T
     if (rc != STWQ_OK) return rc;
     w = attn_layout(ctx->ws_attn, G, Tq, Tk_pad, d, staged);
 
+    // key-column scales, padded with zeros (to the 16-column pitch of the score matrix; to whole
+    // chunks of 128 keys for the one-kernel head)
+    const int n_pad = (int)round_up(Tk_pad, 128);
+    pad_scales_kernel<<<(n_pad + 255) / 256, 256, 0, st>>>(s_kcol, Tk, n_pad, w.skcol);
+    ctx->launches += 1;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
+    if (!staged)                                          // quantizes its queries itself
+        return stwq_launch_qattn_fused(ctx, Q, pos_q, G, Tq, Tk, d, Tmax, Kc, Vt, s_q, w.skcol, s_v, P, bits, causal, out_dtype,
+                                       O, st);
     // queries -> codes with their per-position scales
     rc = launch_rows(ctx, Q, (int64_t)G * Tq, d, pos_q, Tq, 0, s_q, P, bits, w.Qq, (int64_t)Tq * d, 0, st);
     if (rc != STWQ_OK) return rc;
-    // key-column scales, padded with zeros (to the 16-column pitch of the score matrix; to whole
-    // chunks of 128 keys for the one-kernel head)
-    cudaError_t e = cudaMemsetAsync(w.skcol, 0, (size_t)round_up(Tk_pad, 128) * 4, st);
-    if (e == cudaSuccess) e = cudaMemcpyAsync(w.skcol, s_kcol, (size_t)Tk * 4, cudaMemcpyDeviceToDevice, st);
-    if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
-    if (!staged)
-        return stwq_launch_qattn_fused(ctx, w.Qq, pos_q, G, Tq, Tk, d, Tmax, Kc, Vt, s_q, w.skcol, s_v, P, bits, causal,
-                                       out_dtype, O, st);
     // S = dequantized Q K^T, one matrix per head: rows scaled by s_q[pos], columns by s_kcol
     stwq_batch bq = {G, (int64_t)d, (int64_t)Tmax * d, 0, 1, 0};
     rc = stwq_launch_qgemm2(ctx, w.Qq, pos_q, Tq, d, (int)Tk_pad, Kc, w.skcol, s_q, P, nullptr, STWQ_ACT_NONE, STWQ_OUT_F32,

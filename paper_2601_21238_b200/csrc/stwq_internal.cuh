@@ -96,7 +96,7 @@ int stwq_launch_fold(stwq_ctx* ctx, const float* W, int N, int K, const float* s
 size_t stwq_calibrate_ws_bytes(int P);
 size_t stwq_gps_ws_bytes(int K, int N);
 size_t stwq_dgc_ws_bytes(int D);
-int stwq_launch_qattn_fused(stwq_ctx* ctx, const int8_t* Qq, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
+int stwq_launch_qattn_fused(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
                             const int8_t* Kc, const int8_t* Vt, const float* s_q, const float* s_kcol_pad, const float* s_v,
                             int P, int bits, int causal, int out_dtype, void* O, cudaStream_t st);
 int stwq_launch_dgc(stwq_ctx* ctx, void* ws, const float* F, int n, int D, int k, double ridge, double* rho,

@@ -49,6 +49,8 @@ constexpr uint32_t kMagicBits = 0x4B400000u;
 
 struct FaParams {
     int Tq, Tk, d, causal, P, n_qt, dkb, out_bf16, kstages, vstages, nbuf;
+    const float* Q;               // [G, Tq, d] fp32: quantized by the CTA that owns the rows
+    int qmin, qmax;
     const int32_t* pos_q;
     const float* s_q;
     const float* s_kcol;          // padded to a multiple of 128 entries
@@ -126,7 +128,7 @@ __device__ __forceinline__ uint64_t acc_to_float2(uint32_t v0, uint32_t v1, uint
 }
 
 __global__ void __launch_bounds__(kThreads, 2)
-qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+qattn_fused_kernel(const __grid_constant__ CUtensorMap tmK,
                    const __grid_constant__ CUtensorMap tmV, const FaParams p)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -172,7 +174,7 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const int tmem_cols = p.d <= 128 ? 256 : 512;        // O follows them: columns 64 nbuf .. 64 nbuf + d - 1
 
     if (threadIdx.x == 0) {
-        mbar_init(bar_q, 1);
+        mbar_init(bar_q, kSoftWarps);                     // the row threads write the query codes
         for (int s = 0; s < kMaxStages; ++s) {
             mbar_init(bar_kfull(s), 1);
             mbar_init(bar_kempty(s), 1);
@@ -210,8 +212,6 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // One thread feeds both rings and never blocks on one of them while the other could take a
         // load: the value chunks of the second walk start arriving during the first.
         if (lane == 0) {
-            mbar_expect_tx(bar_q, (uint32_t)(p.dkb * kTile));
-            for (int kb = 0; kb < p.dkb; ++kb) tma_load_3d(base + kb * kTile, &tmQ, kb * 128, q0, g, bar_q);
             int ik = 0, iv = 0;                           // next key load (of 2 nch), next value load (of nch)
             bool ok = true;
             unsigned long long t0 = globaltimer_ns();
@@ -254,8 +254,6 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (!ok) {
                 // giving up: loads already issued may still be landing in this CTA's shared memory
                 t0 = globaltimer_ns();
-                while (!mbar_try_wait(bar_q, 0u))
-                    if (globaltimer_ns() - t0 > limit) break;
                 for (int b = 1; b <= kKStages && ik - b >= 0; ++b) {
                     const int jt = ik - b;
                     while (!mbar_try_wait(bar_kfull(jt % kKStages), (uint32_t)(jt / kKStages) & 1u))
@@ -337,6 +335,41 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         // first walk adds half a 3-input max and half a packed add, the second half a packed fma
         // (scale to codes and round) and three quarters of a byte permute.
         const int h = (warp - 2) >> 2;                    // which half of every chunk
+        // The queries of this tile -> codes (the static per-position quantizer: (x * 1) * (1 / s_q[pos]),
+        // round to nearest even, clamp), written as the A operand: rows of 128 bytes, 16-byte pieces
+        // swizzled by the row, zeros beyond the head dimension. A thread takes 16 consecutive
+        // channels at a time; consecutive threads walk along the row.
+        {
+            const int rt_id = (int)threadIdx.x - 64;      // 0 .. 255
+            const int pieces = p.dkb * 8;                 // 16-byte pieces per row, over all 128-byte blocks
+            const int live = p.d >> 4;                    // pieces that hold channels
+            for (int t = rt_id; t < kQT * pieces; t += kSoftWarps * 32) {
+                const int row = t / pieces, c16 = t - row * pieces;
+                const int qi = q0 + row;
+                uint32_t w[4] = {0u, 0u, 0u, 0u};
+                if (c16 < live && qi < p.Tq) {
+                    const int pos = p.pos_q[qi];
+                    if (pos >= 0 && pos < p.P) {
+                        const float rt = __frcp_rn(p.s_q[pos]);
+                        const float4* src = reinterpret_cast<const float4*>(p.Q + ((int64_t)g * p.Tq + qi) * p.d) + c16 * 4;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float4 x = __ldg(src + k);
+                            const int c0 = stwq_code(__fmul_rn(x.x, rt), p.qmin, p.qmax), c1 = stwq_code(__fmul_rn(x.y, rt), p.qmin, p.qmax);
+                            const int c2 = stwq_code(__fmul_rn(x.z, rt), p.qmin, p.qmax), c3 = stwq_code(__fmul_rn(x.w, rt), p.qmin, p.qmax);
+                            w[k] = (uint32_t)(c0 & 0xFF) | ((uint32_t)(c1 & 0xFF) << 8) | ((uint32_t)(c2 & 0xFF) << 16) | ((uint32_t)(c3 & 0xFF) << 24);
+                        }
+                    }
+                }
+                const int kb = c16 >> 3, piece = c16 & 7;
+                st_shared_v4(base + (uint32_t)(kb * kTile) + (uint32_t)(row >> 3) * 1024u + (uint32_t)(row & 7) * 128u +
+                                 (uint32_t)((piece ^ (row & 7)) * 16),
+                             w[0], w[1], w[2], w[3]);
+            }
+            fence_async_smem();                           // the codes become visible to the tensor core's reads
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_q);
+        }
         const int q = warp & 3;                           // the lane quarter of tensor memory this warp may read
         const int r = q * 32 + lane;                      // row of the tile
         const int i = q0 + r;                             // query index within the head
@@ -542,9 +575,9 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
 }  // namespace
 
-// Qq [G, Tq, d] codes of the queries; Kc [G, Tmax, d], Vt [G, d, Tmax] the code caches; s_kcol_pad
+// Q [G, Tq, d] fp32 queries; Kc [G, Tmax, d], Vt [G, d, Tmax] the code caches; s_kcol_pad
 // holds at least round_up(Tk, 128) entries. O [G, Tq, d] fp32 or bf16.
-int stwq_launch_qattn_fused(stwq_ctx* ctx, const int8_t* Qq, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
+int stwq_launch_qattn_fused(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int Tq, int Tk, int d, int Tmax,
                             const int8_t* Kc, const int8_t* Vt, const float* s_q, const float* s_kcol_pad, const float* s_v,
                             int P, int bits, int causal, int out_dtype, void* O, cudaStream_t st)
 {
@@ -553,15 +586,16 @@ int stwq_launch_qattn_fused(stwq_ctx* ctx, const int8_t* Qq, const int32_t* pos_
     p.n_qt = (Tq + kQT - 1) / kQT;
     p.dkb = (d + 127) / 128;
     p.out_bf16 = out_dtype == STWQ_OUT_BF16 ? 1 : 0;
+    p.Q = Q;
+    p.qmax = (1 << (bits - 1)) - 1;
+    p.qmin = -(1 << (bits - 1));
     p.pos_q = pos_q; p.s_q = s_q; p.s_kcol = s_kcol_pad; p.s_v = s_v;
     p.levels = (float)((1 << bits) - 1);
     p.O = O;
     p.status = ctx->d_status;
     p.wait_limit_ns = (unsigned long long)ctx->wait_limit_ms * 1000000ull;
-    CUtensorMap tmQ, tmK, tmV;
-    int rc = stwq_encode_3d(ctx, &tmQ, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Qq, Tq, d, G, d, (int64_t)Tq * d, 128, kQT);
-    if (rc != STWQ_OK) return rc;
-    rc = stwq_encode_3d(ctx, &tmK, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Kc, Tmax, d, G, d, (int64_t)Tmax * d, 128, kKT);
+    CUtensorMap tmK, tmV;
+    int rc = stwq_encode_3d(ctx, &tmK, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Kc, Tmax, d, G, d, (int64_t)Tmax * d, 128, kKT);
     if (rc != STWQ_OK) return rc;
     rc = stwq_encode_3d(ctx, &tmV, CU_TENSOR_MAP_DATA_TYPE_UINT8, 1, Vt, d, Tmax, G, Tmax, (int64_t)d * Tmax, kKT, d);
     if (rc != STWQ_OK) return rc;
@@ -581,7 +615,7 @@ int stwq_launch_qattn_fused(stwq_ctx* ctx, const int8_t* Qq, const int32_t* pos_
         if (e != cudaSuccess) return stwq_cuda_fail(ctx, e);
         ctx->attn_configured = 1;
     }
-    qattn_fused_kernel<<<dim3((unsigned)G, (unsigned)p.n_qt), kThreads, (size_t)dyn, st>>>(tmQ, tmK, tmV, p);
+    qattn_fused_kernel<<<dim3((unsigned)G, (unsigned)p.n_qt), kThreads, (size_t)dyn, st>>>(tmK, tmV, p);
     ctx->launches += 1;
     cudaError_t e = cudaGetLastError();
     return e == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e);
