@@ -650,6 +650,64 @@ def whole_config(ctx, torch, dev, cfg, peaks, args):
     return out
 
 
+def attention_rows(ctx, pk, torch, dev, peaks, graph_us):
+    """Quantized attention of a VAR-d16-shaped layer (batch 16 x 16 heads, 680 positions, head dimension
+    64): filling the quantized KV cache, then the attention head on int8 codes, as one kernel and as
+    three separate stages (block-causal masks of the real model are replaced by a plain causal one)."""
+    out = {}
+    G, T, d, Tmax = 256, 680, 64, 688
+    Q = torch.randn(G, T, d, device=dev)
+    Kn = torch.randn(G, T, d, device=dev)
+    Vn = torch.randn(G, T, d, device=dev)
+    pos_q = torch.arange(T, dtype=torch.int32, device=dev)
+    s_q = torch.full((T,), 4.0 * 2 / 255, device=dev)
+    s_k = torch.full((T,), 4.0 * 2 / 255, device=dev)
+    s_kcol = s_k * (1.0 / d ** 0.5)
+    s_v = torch.full((d,), 4.0 * 2 / 255, device=dev)
+    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=dev)
+    Vt = torch.zeros((G, d, Tmax), dtype=torch.int8, device=dev)
+    O = torch.empty((G, T, d), dtype=torch.bfloat16, device=dev)
+    ctx.stwq_reserve_attention(G, T, T, d)
+    t_app = graph_us(lambda: ctx.kv_append(Kn, Vn, 0, s_k, s_v, 8, Kc, Vt), 1)
+    t_att = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    ctx.stwq_set_option(pk.OPT_VARIANT, 9)
+    try:
+        ctx.stwq_reserve_attention(G, T, T, d)
+        t_staged = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    finally:
+        ctx.stwq_set_option(pk.OPT_VARIANT, 0)
+    # what a head must move: Q fp32, both code caches once, O
+    att_bytes = G * T * d * (4 + 2) + 2 * G * T * d
+    app_bytes = 2 * G * T * d * (4 + 1)
+    # what bounds the one-kernel head is the exponential: one ex2 per score and walk, 16 per clock per SM.
+    # Scores are processed in blocks of 32 rows x 32 keys; a block is skipped when the causal mask hides
+    # all of it.
+    blocks = 0
+    for q0 in range(0, T, 32):
+        last_visible = min(T - 1, q0 + 31)                   # Tq = Tk: the last row of the block of rows sees this key
+        blocks += last_visible // 32 + 1
+    ex2 = 2.0 * G * blocks * 32 * 32
+    xu_peak = 16.0 * 148 * 1.965e9
+    # the kernel alone (the key scales are padded by a tiny kernel in the same call)
+    out["attention_var_d16"] = {"heads": G, "positions": T, "head_dim": d, "kv_append_us": round(t_app, 1),
+                                "kv_append_frac_of_hbm": round(app_bytes / t_app / 1e3 / peaks["hbm_gbs"], 3),
+                                "qattention_us": round(t_att, 1),
+                                "qattention_three_stages_us": round(t_staged, 1),
+                                "matmul_tops": round(2 * 2.0 * G * T * T * d / t_att / 1e6, 1),
+                                "min_bytes_frac_of_hbm": round(att_bytes / t_att / 1e3 / peaks["hbm_gbs"], 3),
+                                "roofline": {"kernel": "qattn_fused_kernel", "bound": "alu", "unit": "G ex2/s",
+                                             "achieved": round(ex2 / t_att / 1e3, 1), "peak": round(xu_peak / 1e9, 1),
+                                             "frac": round(ex2 / (t_att * 1e-6) / xu_peak, 3),
+                                             "peak_source": "16 ex2 per clock per SM x 148 SMs x 1965 MHz (the special-function "
+                                                            "unit; a loop of nothing but ex2 measures 16.3 per clock per SM)"},
+                                "note": "one kernel per 128 queries of a head: Q quantized, Q K^T, softmax, probability codes "
+                                        "and P V on the SM (keys walked twice); three_stages = batched int8 GEMMs with scores "
+                                        "and codes in workspace; ops counted for the full T x T matrices, bytes = Q fp32 + "
+                                        "both code caches + O bf16"}
+    del Q, Kn, Vn, Kc, Vt, O
+    return out["attention_var_d16"]
+
+
 def other_configs(ctx, pk, torch, dev, peaks, args):
     """The other workload families: whole-step figures of the VAR-d16 and MAR-Huge blocks (and of
     VAR-d30 when it is not the headline), the decode-step calls with their own roofline, and a few
@@ -742,44 +800,7 @@ def other_configs(ctx, pk, torch, dev, peaks, args):
         rows.append(row)
         del X, W1, W2, H, Hq, Y
     out["ffn_fc1_fc2_chained"] = rows
-    # quantized attention of a VAR-d16-shaped layer (batch 16 x 16 heads, 680 positions, head dimension 64):
-    # filling the quantized KV cache, then both attention matmuls on int8 codes with the softmax-and-quantize
-    # pass in between (block-causal masks of the real model are replaced by a plain causal one)
-    G, T, d, Tmax = 256, 680, 64, 688
-    Q = torch.randn(G, T, d, device=dev)
-    Kn = torch.randn(G, T, d, device=dev)
-    Vn = torch.randn(G, T, d, device=dev)
-    pos_q = torch.arange(T, dtype=torch.int32, device=dev)
-    s_q = torch.full((T,), 4.0 * 2 / 255, device=dev)
-    s_k = torch.full((T,), 4.0 * 2 / 255, device=dev)
-    s_kcol = s_k * (1.0 / d ** 0.5)
-    s_v = torch.full((d,), 4.0 * 2 / 255, device=dev)
-    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=dev)
-    Vt = torch.zeros((G, d, Tmax), dtype=torch.int8, device=dev)
-    O = torch.empty((G, T, d), dtype=torch.bfloat16, device=dev)
-    ctx.stwq_reserve_attention(G, T, T, d)
-    t_app = graph_us(lambda: ctx.kv_append(Kn, Vn, 0, s_k, s_v, 8, Kc, Vt), 1)
-    t_att = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
-    ctx.stwq_set_option(pk.OPT_VARIANT, 9)
-    try:
-        ctx.stwq_reserve_attention(G, T, T, d)
-        t_staged = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
-    finally:
-        ctx.stwq_set_option(pk.OPT_VARIANT, 0)
-    # what a head must move: Q (fp32 in, codes out and back in), both code caches once, O
-    att_bytes = G * T * d * (4 + 1 + 1 + 2) + 2 * G * T * d
-    app_bytes = 2 * G * T * d * (4 + 1)
-    out["attention_var_d16"] = {"heads": G, "positions": T, "head_dim": d, "kv_append_us": round(t_app, 1),
-                                "kv_append_frac_of_hbm": round(app_bytes / t_app / 1e3 / peaks["hbm_gbs"], 3),
-                                "qattention_us": round(t_att, 1),
-                                "qattention_three_stages_us": round(t_staged, 1),
-                                "matmul_tops": round(2 * 2.0 * G * T * T * d / t_att / 1e6, 1),
-                                "min_bytes_frac_of_hbm": round(att_bytes / t_att / 1e3 / peaks["hbm_gbs"], 3),
-                                "note": "one kernel per 128 queries of a head: Q K^T, softmax, probability codes and P V "
-                                        "on the SM (keys walked twice); three_stages = batched int8 GEMMs with scores and "
-                                        "codes in workspace; ops counted for the full T x T matrices, bytes = Q fp32 + "
-                                        "Q codes twice + both code caches + O bf16"}
-    del Q, Kn, Vn, Kc, Vt, O
+    out["attention_var_d16"] = attention_rows(ctx, pk, torch, dev, peaks, graph_us)
     ctx.check_device_status()
     return out
 
@@ -868,6 +889,27 @@ def reference_arm(args):
     print(json.dumps(line), flush=True)
 
 
+def attention_arm(args):
+    """Only the attention layer of other_configs(), for a profiler capture of its kernels."""
+    import torch
+
+    import paper_2601_21238_b200 as pk
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path for the product arm")
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    ctx = pk.Context(0)
+    side = torch.cuda.Stream()
+
+    def graph_us(fn, calls_per_graph, seconds=args.extra_seconds):
+        g = capture(torch, side, fn)
+        return timed_replays(torch, side, g, seconds) / calls_per_graph * 1e3
+
+    row = attention_rows(ctx, pk, torch, dev, measured_peaks(), graph_us)
+    ctx.check_device_status()
+    print(json.dumps({"attention_var_d16": row}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -886,6 +928,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-probe", action="store_true")
     ap.add_argument("--no-extras", action="store_true", help="skip the other workload families")
+    ap.add_argument("--only-attention", action="store_true", help="time only the quantized attention layer (profiling aid)")
     ap.add_argument("--ncu-raw-csv", help="raw ncu csv export to summarise into profiles/roofline_traffic.json")
     ap.add_argument("--profile-key", default="qgemm2_kernel/config3", help="kernel/workload the csv belongs to")
     ap.add_argument("--profile-note", default="")
@@ -897,6 +940,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
         reference_arm(args)
+    elif args.only_attention:
+        attention_arm(args)
     else:
         gpu_arm(args)
 
