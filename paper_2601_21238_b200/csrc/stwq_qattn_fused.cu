@@ -380,8 +380,9 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmK,
             if (pos >= 0 && pos < p.P) a = p.s_q[pos];
             else if (g == 0 && h == 0) atomicOr(p.status, STWQ_DEV_POS_RANGE);
         }
-        // rows beyond Tq hold zero codes; they run through the same arithmetic and are not stored
-        const int last = (p.causal && valid) ? min(p.Tk - 1, i + p.Tk - p.Tq) : p.Tk - 1;   // last visible key of the row
+        // rows beyond Tq see no key at all: a warp of such rows skips every block (and still hands the
+        // accumulators back and writes zero codes); in a mixed warp they run along, masked, and are not stored
+        const int last = !valid ? -1 : (p.causal ? min(p.Tk - 1, i + p.Tk - p.Tq) : p.Tk - 1);   // last visible key of the row
         const int wlast = __reduce_max_sync(0xffffffffu, last);
         const int wfirst = __reduce_min_sync(0xffffffffu, last);
         const float al = fmaxf(a * kLog2e, 1e-30f);       // scores are kept in units of log2 e; > 0 so that a masked -inf stays -inf
@@ -409,10 +410,11 @@ qattn_fused_kernel(const __grid_constant__ CUtensorMap tmK,
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
                 const float2 other = stats[(h ^ 1) * 128 + r];
-                const float mt = fmaxf(m, other.x);      // finite: the first part has seen key 0
-                l = l * ex2f(m - mt) + other.y * ex2f(other.x - mt);
-                m = mt;
-                inv2 = dup_f2(__fdiv_rn(p.levels, l));
+                const float mt = fmaxf(m, other.x);      // finite for every row below Tq: the first part has seen key 0
+                const float rt = mt == -INFINITY ? 0.0f : mt;
+                l = l * ex2f(m - rt) + other.y * ex2f(other.x - rt);
+                m = rt;                                   // a row beyond Tq: every key masked, codes 0
+                inv2 = dup_f2(l > 0.0f ? __fdiv_rn(p.levels, l) : 0.0f);      // l = 0: a row beyond Tq
             }
             {
                 ok = mbar_wait(bar_cfull(cslot), cparity, abort_flag, limit);
