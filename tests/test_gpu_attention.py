@@ -225,6 +225,48 @@ def test_one_kernel_head_agrees_with_the_separate_stages(gpu, shape):
     assert rows_equal > 0.9, rows_equal
 
 
+@pytest.mark.parametrize("variant", [0, 9])
+def test_qattention_refuses_bad_arguments_and_reports_bad_positions(gpu, variant):
+    """Host-side refusals (more queries than keys under a causal mask, a head dimension that is no
+    multiple of 16, keys beyond the cache) leave no launch behind; a query position outside the scale
+    table is reported through the device status word, and the context stays usable."""
+    torch = gpu.torch
+    G, T, d, P, Tmax = 2, 40, 64, 40, 48
+    Q, K, V, s_q, s_k, s_v = _head_data(G, T, d, P)
+    s_kcol = (s_k[:T] / 8).astype(np.float32)
+    Kc = torch.zeros((G, Tmax, d), dtype=torch.int8, device=gpu.dev)
+    Vt = torch.zeros((G, d, Tmax), dtype=torch.int8, device=gpu.dev)
+    gpu.ctx.kv_append(gpu.T(K), gpu.T(V), 0, gpu.T(s_k), gpu.T(s_v), 8, Kc, Vt)
+    O = torch.zeros((G, T, d), dtype=torch.float32, device=gpu.dev)
+    pos = np.arange(T, dtype=np.int32)
+    gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
+    try:
+        args = lambda Tk, causal, pos_q=pos, Qx=Q, Ox=O: (gpu.T(Qx), gpu.T(pos_q), Tk, Kc, Vt, gpu.T(s_q), gpu.T(s_kcol[:Tk]),
+                                                          gpu.T(s_v), 8, causal, gpu.B.OUT_F32, Ox)
+        with pytest.raises(Exception):
+            gpu.ctx.qattention(*args(T - 8, True))                              # causal with Tq > Tk
+        with pytest.raises(Exception):
+            gpu.ctx.qattention(*args(Tmax + 16, False))                         # more keys than the cache holds
+        Kc24 = torch.zeros((G, Tmax, 24), dtype=torch.int8, device=gpu.dev)
+        with pytest.raises(Exception):
+            gpu.ctx.qattention(gpu.T(Q[:, :, :24]), gpu.T(pos), T, Kc24, torch.zeros((G, 24, Tmax), dtype=torch.int8, device=gpu.dev),
+                               gpu.T(s_q), gpu.T(s_kcol), gpu.T(s_v[:24]), 8, True, gpu.B.OUT_F32,
+                               torch.zeros((G, T, 24), dtype=torch.float32, device=gpu.dev))
+        assert gpu.ctx.stwq_device_status() == 0
+        bad = pos.copy()
+        bad[7] = P + 5
+        gpu.ctx.qattention(*args(T, True, bad))
+        assert gpu.ctx.stwq_device_status() == -8                               # STWQ_ERR_POS_RANGE, cleared by the read
+        gpu.ctx.qattention(*args(T, True))
+        assert gpu.ctx.stwq_device_status() == 0
+        r = oracle.qattention(Q[0], K[0], V[0], pos, pos, s_q, s_k, s_v, np.float32(1 / 8), 8, True)
+        got = O[0].cpu().numpy().astype(np.float64)
+        flip = 4 * (1.0 / 255) * 128 * s_v[None, :].astype(np.float64)
+        assert (np.abs(got - r["O"]) <= 1e-5 * (np.abs(r["O"]) + r["mag"]) + flip).all()
+    finally:
+        gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, 0)
+
+
 # ----------------------------------------------------------------------------- distribution-guided calibration
 @pytest.mark.parametrize("shape", [(128, 64, 0.0), (41, 5, 0.0), (300, 257, 0.0), (6, 12, 1e-6), (64, 1, 0.0), (20, 20, 1e-9)])
 def test_dgc_select_matches_the_oracle(gpu, shape):
