@@ -670,6 +670,11 @@ def attention_rows(ctx, pk, torch, dev, peaks, graph_us):
     ctx.stwq_reserve_attention(G, T, T, d)
     t_app = graph_us(lambda: ctx.kv_append(Kn, Vn, 0, s_k, s_v, 8, Kc, Vt), 1)
     t_att = graph_us(lambda: ctx.qattention(Q, pos_q, T, Kc, Vt, s_q, s_kcol, s_v, 8, True, pk.OUT_BF16, O), 1)
+    # a decode step: one new query per head against the whole cache
+    Q1 = torch.randn(G, 1, d, device=dev)
+    O1 = torch.empty((G, 1, d), dtype=torch.bfloat16, device=dev)
+    pos_1 = torch.full((1,), T - 1, dtype=torch.int32, device=dev)
+    t_dec = graph_us(lambda: ctx.qattention(Q1, pos_1, T, Kc, Vt, s_q, s_kcol, s_v, 8, False, pk.OUT_BF16, O1), 1)
     ctx.stwq_set_option(pk.OPT_VARIANT, 9)
     try:
         ctx.stwq_reserve_attention(G, T, T, d)
@@ -693,6 +698,7 @@ def attention_rows(ctx, pk, torch, dev, peaks, graph_us):
                                 "kv_append_frac_of_hbm": round(app_bytes / t_app / 1e3 / peaks["hbm_gbs"], 3),
                                 "qattention_us": round(t_att, 1),
                                 "qattention_three_stages_us": round(t_staged, 1),
+                                "qattention_one_query_per_head_us": round(t_dec, 1),
                                 "matmul_tops": round(2 * 2.0 * G * T * T * d / t_att / 1e6, 1),
                                 "min_bytes_frac_of_hbm": round(att_bytes / t_att / 1e3 / peaks["hbm_gbs"], 3),
                                 "roofline": {"kernel": "qattn_fused_kernel", "bound": "alu", "unit": "G ex2/s",
@@ -702,9 +708,10 @@ def attention_rows(ctx, pk, torch, dev, peaks, graph_us):
                                                             "unit; a loop of nothing but ex2 measures 16.3 per clock per SM)"},
                                 "note": "one kernel per 128 queries of a head: Q quantized, Q K^T, softmax, probability codes "
                                         "and P V on the SM (keys walked twice); three_stages = batched int8 GEMMs with scores "
-                                        "and codes in workspace; ops counted for the full T x T matrices, bytes = Q fp32 + "
-                                        "both code caches + O bf16"}
-    del Q, Kn, Vn, Kc, Vt, O
+                                        "and codes in workspace; one_query_per_head = a decode step (one CTA per head reads the "
+                                        "cache once, dp4a, caches L2-resident here); ops counted for the full T x T matrices, "
+                                        "bytes = Q fp32 + both code caches + O bf16"}
+    del Q, Kn, Vn, Kc, Vt, O, Q1, O1
     return out["attention_var_d16"]
 
 

@@ -16,6 +16,8 @@
 // static scale per channel, because a scale that varied along the keys could not leave the sum over
 // keys; the caches hold codes: K as [G, Tmax, d] and V transposed as [G, d, Tmax], so that both
 // matmuls read K-major operands.
+#include <cuda_bf16.h>
+
 #include "stwq_internal.cuh"
 
 namespace {
@@ -140,6 +142,143 @@ softmax_quantize_kernel(const float* __restrict__ S, int64_t rows, int Tq, int T
         float u = 0.0f;
         if (j <= last) u = exp2f((s[j] - m) * 1.4426950408889634f) * scale;
         p[j] = (uint8_t)min(max(__float2int_rn(u), 0), (int)levels);
+    }
+}
+
+// Few queries against a long cache (a decode step: one new token per head; Section 2). One CTA per
+// (head, query): the work is reading the head's key and value codes once, so no tensor core is
+// involved: integer dot products by dp4a, the score row and its codes in shared memory.
+//   1. the query row -> codes (the quantizer of rowq_rows_kernel);
+//   2. a thread per key: acc = sum_c Qq[c] Kq[j, c] (the key row is contiguous), S[j] = acc * (s_q * s_kcol[j]);
+//   3. row softmax and the quantizer of the probabilities, as in softmax_quantize_kernel;
+//   4. a thread per channel and part of the keys: acc = sum_j Pcode[j] Vq[j, c] along the transposed
+//      value cache (unsigned x signed dp4a), parts added through shared memory;
+//   5. O[c] = acc * (delta_p * s_v[c]).
+constexpr int kFewThreads = 256;
+__device__ __forceinline__ int dp4a_ss(uint32_t a, uint32_t b, int c)
+{
+    int r;
+    asm("dp4a.s32.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+__device__ __forceinline__ int dp4a_us(uint32_t a, uint32_t b, int c)
+{
+    int r;
+    asm("dp4a.u32.s32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(c));
+    return r;
+}
+__device__ __forceinline__ float block_reduce(float v, float* scratch, bool is_max)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float w = __shfl_xor_sync(0xffffffffu, v, o);
+        v = is_max ? fmaxf(v, w) : v + w;
+    }
+    __syncthreads();                                      // scratch may still be read from the previous reduction
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float r = scratch[0];
+    for (int w = 1; w < kFewThreads / 32; ++w) r = is_max ? fmaxf(r, scratch[w]) : r + scratch[w];
+    return r;
+}
+
+template <bool BF16>
+__global__ void __launch_bounds__(kFewThreads)
+qattn_few_kernel(const float* __restrict__ Q, const int32_t* __restrict__ pos_q, int Tq, int Tk, int Tk_pad, int d, int Tmax,
+                 const int8_t* __restrict__ Kc, const int8_t* __restrict__ Vt, const float* __restrict__ s_q,
+                 const float* __restrict__ s_kcol, const float* __restrict__ s_v, int P, int qmin, int qmax, float levels,
+                 int causal, void* __restrict__ O, uint32_t* __restrict__ status)
+{
+    extern __shared__ __align__(16) uint8_t few_smem[];
+    float* S = reinterpret_cast<float*>(few_smem);                       // [Tk_pad]
+    uint8_t* Pc = few_smem + (size_t)Tk_pad * 4;                          // [Tk_pad] codes, zero beyond the visible keys
+    uint32_t* q8 = reinterpret_cast<uint32_t*>(Pc + Tk_pad);              // [d / 4] packed query codes
+    int* part = reinterpret_cast<int*>(q8 + d / 4);                       // [kFewThreads] partial sums of step 4
+    __shared__ float scratch[kFewThreads / 32];
+    const int g = blockIdx.x / Tq, i = blockIdx.x - g * Tq;
+    const int tid = threadIdx.x;
+    const int pos = pos_q[i];
+    const bool ok = pos >= 0 && pos < P;
+    if (!ok && tid == 0 && g == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+    const float sq = ok ? s_q[pos] : 0.0f;
+    // 1. query codes
+    if (tid < d / 4) {
+        uint32_t w = 0;
+        if (ok) {
+            const float rt = __frcp_rn(sq);
+            const float4 x = reinterpret_cast<const float4*>(Q + ((int64_t)g * Tq + i) * d)[tid];
+            w = (uint32_t)(stwq_code(__fmul_rn(x.x, rt), qmin, qmax) & 0xFF) | ((uint32_t)(stwq_code(__fmul_rn(x.y, rt), qmin, qmax) & 0xFF) << 8) |
+                ((uint32_t)(stwq_code(__fmul_rn(x.z, rt), qmin, qmax) & 0xFF) << 16) | ((uint32_t)(stwq_code(__fmul_rn(x.w, rt), qmin, qmax) & 0xFF) << 24);
+        }
+        q8[tid] = w;
+    }
+    __syncthreads();
+    // 2. scores
+    const int last = causal ? min(Tk - 1, i + (Tk - Tq)) : Tk - 1;       // last visible key
+    const int8_t* Kg = Kc + (int64_t)g * Tmax * d;
+    float m = -INFINITY;
+    for (int j = tid; j <= last; j += kFewThreads) {
+        const uint4* krow = reinterpret_cast<const uint4*>(Kg + (int64_t)j * d);
+        int acc = 0;
+        for (int c = 0; c < d / 16; ++c) {
+            const uint4 k = __ldg(krow + c);
+            acc = dp4a_ss(q8[4 * c], k.x, acc);
+            acc = dp4a_ss(q8[4 * c + 1], k.y, acc);
+            acc = dp4a_ss(q8[4 * c + 2], k.z, acc);
+            acc = dp4a_ss(q8[4 * c + 3], k.w, acc);
+        }
+        const float sc = __fmul_rn((float)acc, __fmul_rn(sq, s_kcol[j]));
+        S[j] = sc;
+        m = fmaxf(m, sc);
+    }
+    // 3. softmax and codes
+    m = block_reduce(m, scratch, true);
+    float sum = 0.0f;
+    for (int j = tid; j <= last; j += kFewThreads) sum += exp2f((S[j] - m) * 1.4426950408889634f);
+    sum = block_reduce(sum, scratch, false);
+    const float scale = sum > 0.0f ? __fdiv_rn(levels, sum) : 0.0f;
+    for (int j = tid; j < Tk_pad; j += kFewThreads) {
+        float u = 0.0f;
+        if (j <= last) u = exp2f((S[j] - m) * 1.4426950408889634f) * scale;
+        Pc[j] = (uint8_t)min(max(__float2int_rn(u), 0), (int)levels);
+    }
+    __syncthreads();
+    // 4. O accumulators: thread = (part of the keys, channel); a part is a multiple of 16 keys
+    const int parts = max(1, kFewThreads / d);
+    const int n16 = Tk_pad / 16;                          // 16-key pieces; those beyond the last visible key hold zero codes
+    const float delta_p = __fdiv_rn(1.0f, levels);
+    for (int c0 = 0; c0 < d; c0 += kFewThreads) {         // one pass unless d > 256 threads
+        const int c = c0 + (parts > 1 ? tid % d : tid);
+        const int prt = parts > 1 ? tid / d : 0;
+        int acc = 0;
+        if (c < d && prt < parts) {
+            const uint4* vrow = reinterpret_cast<const uint4*>(Vt + ((int64_t)g * d + c) * Tmax);
+            const uint4* prow = reinterpret_cast<const uint4*>(Pc);
+            const int per = (n16 + parts - 1) / parts;
+            const int e = min(n16, (prt + 1) * per);
+            for (int t = prt * per; t < e; ++t) {
+                if (t * 16 > last) break;                 // nothing but zero codes from here on
+                const uint4 v = __ldg(vrow + t);
+                const uint4 pc = prow[t];
+                acc = dp4a_us(pc.x, v.x, acc);
+                acc = dp4a_us(pc.y, v.y, acc);
+                acc = dp4a_us(pc.z, v.z, acc);
+                acc = dp4a_us(pc.w, v.w, acc);
+            }
+        }
+        __syncthreads();
+        part[tid] = acc;
+        __syncthreads();
+        if (c < d && prt == 0) {
+            int total = acc;
+            for (int q = 1; q < parts; ++q) total += part[q * d + (tid % d)];
+            // 5. dequantize
+            const float o = __fmul_rn((float)total, __fmul_rn(delta_p, s_v[c]));
+            const int64_t idx = ((int64_t)g * Tq + i) * d + c;
+            if (BF16) static_cast<__nv_bfloat16*>(O)[idx] = __float2bfloat16_rn(o);
+            else static_cast<float*>(O)[idx] = o;
+        }
     }
 }
 
@@ -268,6 +407,28 @@ int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int T
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int64_t Tk_pad = round_up(Tk, 16);
     const bool staged = ctx->debug == 9;                  // the three stages as separate kernels
+    // a decode step: few queries against a long cache. Bound by reading the cache once, done by one
+    // CTA per (head, query) without the tensor cores
+    const size_t few_smem = (size_t)Tk_pad * 5 + (size_t)d + kFewThreads * 4 + 16;
+    if (!staged && Tq <= 4 && few_smem <= 200 * 1024 && (int64_t)G * Tq <= 0x7fffffff) {
+        if (!ctx->attn_few_configured) {
+            cudaError_t e1 = cudaFuncSetAttribute(qattn_few_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(qattn_few_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e1 != cudaSuccess) return stwq_cuda_fail(ctx, e1);
+            ctx->attn_few_configured = 1;
+        }
+        const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
+        const float lv = (float)((1 << bits) - 1);
+        if (out_dtype == STWQ_OUT_BF16)
+            qattn_few_kernel<true><<<(unsigned)(G * Tq), kFewThreads, few_smem, st>>>(Q, pos_q, Tq, Tk, (int)Tk_pad, d, Tmax, Kc, Vt, s_q, s_kcol,
+                                                                                      s_v, P, qmin, qmax, lv, causal ? 1 : 0, O, ctx->d_status);
+        else
+            qattn_few_kernel<false><<<(unsigned)(G * Tq), kFewThreads, few_smem, st>>>(Q, pos_q, Tq, Tk, (int)Tk_pad, d, Tmax, Kc, Vt, s_q, s_kcol,
+                                                                                       s_v, P, qmin, qmax, lv, causal ? 1 : 0, O, ctx->d_status);
+        ctx->launches += 1;
+        cudaError_t e1 = cudaGetLastError();
+        return e1 == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e1);
+    }
     AttnWs w = attn_layout(nullptr, G, Tq, Tk_pad, d, staged);
     int rc = stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, st, 0);
     if (rc != STWQ_OK) return rc;

@@ -45,6 +45,7 @@ struct stwq_ctx {
     uint64_t ws_generation;    // bumped whenever a workspace buffer is (re)allocated
     int probe_configured;      // the peak-probe kernel has its shared-memory attribute set
     int attn_configured;       // so has the one-kernel attention head
+    int attn_few_configured;   // and the few-query attention kernel
     void* encode_tiled;        // cuTensorMapEncodeTiled, resolved at create
 };
 
