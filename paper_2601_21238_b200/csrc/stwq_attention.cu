@@ -29,80 +29,91 @@ __device__ __forceinline__ uint32_t pack_codes(int q0, int q1, int q2, int q3)
     return (uint32_t)(q0 & 0xFF) | ((uint32_t)(q1 & 0xFF) << 8) | ((uint32_t)(q2 & 0xFF) << 16) | ((uint32_t)(q3 & 0xFF) << 24);
 }
 
-// Row-major output (Q codes, key cache): a thread per group of four channels (a 16-byte load, a
-// 4-byte store), consecutive threads along the row and on into the next one.
+// Row-major output (Q codes, key cache): a thread per 16 consecutive channels (four 16-byte loads in
+// flight, one 16-byte store), consecutive threads along the row and on into the next one.
 // out index = g * out_gstride + out_row * d + c, out_row = the row's position (key cache) or its
 // index within the matrix (dense output).
 __global__ void __launch_bounds__(kRowThreads)
-rowq_rows_kernel(const float4* __restrict__ X, int64_t n_vec, int d4, const int32_t* __restrict__ pos_ids, int rows_per_g,
+rowq_rows_kernel(const float4* __restrict__ X, int64_t n_vec, int d16, const int32_t* __restrict__ pos_ids, int rows_per_g,
                  int pos0, const float* __restrict__ s_tok, int P, int qmin, int qmax, int8_t* __restrict__ out,
                  int64_t out_gstride, int out_row_from_pos, uint32_t* __restrict__ status)
 {
     const int64_t i = (int64_t)blockIdx.x * kRowThreads + threadIdx.x;
     if (i >= n_vec) return;
-    const int64_t r = i / d4;
-    const int c4 = (int)(i - r * d4);
+    const int64_t r = i / d16;
+    const int c16 = (int)(i - r * d16);
     const int g = (int)(r / rows_per_g);
     const int t = (int)(r - (int64_t)g * rows_per_g);
     const int pos = pos_ids != nullptr ? pos_ids[t] : pos0 + t;
     const bool ok = pos >= 0 && pos < P;
-    if (!ok && c4 == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+    if (!ok && c16 == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
     if (out_row_from_pos && !ok) return;                  // no slot in the cache for a position outside [0, P)
-    uint32_t packed = 0;
+    uint32_t w[4] = {0u, 0u, 0u, 0u};
     if (ok) {
+        const float4 v0 = X[4 * i], v1 = X[4 * i + 1], v2 = X[4 * i + 2], v3 = X[4 * i + 3];
         const float rt = __frcp_rn(s_tok[pos]);
-        const float4 v = X[i];
         // (x * 1) * rt: no channel scale on queries and keys
-        packed = pack_codes(stwq_code(__fmul_rn(v.x, rt), qmin, qmax), stwq_code(__fmul_rn(v.y, rt), qmin, qmax),
-                            stwq_code(__fmul_rn(v.z, rt), qmin, qmax), stwq_code(__fmul_rn(v.w, rt), qmin, qmax));
+        w[0] = pack_codes(stwq_code(__fmul_rn(v0.x, rt), qmin, qmax), stwq_code(__fmul_rn(v0.y, rt), qmin, qmax),
+                          stwq_code(__fmul_rn(v0.z, rt), qmin, qmax), stwq_code(__fmul_rn(v0.w, rt), qmin, qmax));
+        w[1] = pack_codes(stwq_code(__fmul_rn(v1.x, rt), qmin, qmax), stwq_code(__fmul_rn(v1.y, rt), qmin, qmax),
+                          stwq_code(__fmul_rn(v1.z, rt), qmin, qmax), stwq_code(__fmul_rn(v1.w, rt), qmin, qmax));
+        w[2] = pack_codes(stwq_code(__fmul_rn(v2.x, rt), qmin, qmax), stwq_code(__fmul_rn(v2.y, rt), qmin, qmax),
+                          stwq_code(__fmul_rn(v2.z, rt), qmin, qmax), stwq_code(__fmul_rn(v2.w, rt), qmin, qmax));
+        w[3] = pack_codes(stwq_code(__fmul_rn(v3.x, rt), qmin, qmax), stwq_code(__fmul_rn(v3.y, rt), qmin, qmax),
+                          stwq_code(__fmul_rn(v3.z, rt), qmin, qmax), stwq_code(__fmul_rn(v3.w, rt), qmin, qmax));
     }
-    uint32_t* o = reinterpret_cast<uint32_t*>(out + (int64_t)g * out_gstride + (int64_t)(out_row_from_pos ? pos : t) * (d4 * 4));
-    o[c4] = packed;
+    uint4* o = reinterpret_cast<uint4*>(out + (int64_t)g * out_gstride + (int64_t)(out_row_from_pos ? pos : t) * (d16 * 16));
+    o[c16] = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-// Value cache, transposed: a thread takes four consecutive new positions and four consecutive
-// channels (four 16-byte loads), turns the 4 x 4 block of codes in registers, and writes each
-// channel's four positions as one word of the cache row Vt[g, c, pos0 + t ...] (single bytes at a
-// ragged end or when the run does not start on a 4-byte boundary). Eight consecutive threads
-// cover 32 positions of the same channels, so a warp writes full 32-byte sectors.
-// Per-channel scales, no position scale: (x * rc[c]) * 1.
+// Value cache, transposed: a thread takes eight consecutive new positions and four consecutive
+// channels (eight 16-byte loads in flight), turns the 8 x 4 block of codes in registers, and writes
+// each channel's eight positions as one 8-byte piece of the cache row Vt[g, c, pos0 + t ...]
+// (single bytes at a ragged end or when the run does not start on an 8-byte boundary). Four
+// consecutive threads cover 32 positions of the same channels, so a warp writes full 32-byte
+// sectors. Per-channel scales, no position scale: (x * rc[c]) * 1.
 __global__ void __launch_bounds__(kRowThreads)
 rowq_transpose_kernel(const float4* __restrict__ V, int G, int d4, int t_new, int pos0, const float4* __restrict__ s_v,
                       int qmin, int qmax, int8_t* __restrict__ Vt, int Tmax)
 {
     const int tiles = (t_new + 31) >> 5;
     const int64_t i = (int64_t)blockIdx.x * kRowThreads + threadIdx.x;
-    if (i >= (int64_t)G * tiles * d4 * 8) return;
-    const int tq = (int)(i & 7);
-    int64_t rest = i >> 3;
+    if (i >= (int64_t)G * tiles * d4 * 4) return;
+    const int tq = (int)(i & 3);
+    int64_t rest = i >> 2;
     const int c4 = (int)(rest % d4);
     rest /= d4;
     const int tile = (int)(rest % tiles);
     const int g = (int)(rest / tiles);
-    const int t = tile * 32 + tq * 4;                     // first of this thread's four positions
+    const int t = tile * 32 + tq * 8;                     // first of this thread's eight positions
     if (t >= t_new) return;
-    const int nt = min(4, t_new - t);
+    const int nt = min(8, t_new - t);
     const float4 sv = s_v[c4];
     const float rc[4] = {__frcp_rn(sv.x), __frcp_rn(sv.y), __frcp_rn(sv.z), __frcp_rn(sv.w)};
-    int q[4][4];                                          // [position][channel]
+    float4 v[8];
 #pragma unroll
-    for (int r = 0; r < 4; ++r) {
-        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (r < nt) v = V[((int64_t)g * t_new + t + r) * d4 + c4];
-        q[r][0] = stwq_code(__fmul_rn(v.x, rc[0]), qmin, qmax);
-        q[r][1] = stwq_code(__fmul_rn(v.y, rc[1]), qmin, qmax);
-        q[r][2] = stwq_code(__fmul_rn(v.z, rc[2]), qmin, qmax);
-        q[r][3] = stwq_code(__fmul_rn(v.w, rc[3]), qmin, qmax);
+    for (int r = 0; r < 8; ++r) {
+        v[r] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < nt) v[r] = V[((int64_t)g * t_new + t + r) * d4 + c4];
+    }
+    int q[8][4];                                          // [position][channel]
+#pragma unroll
+    for (int r = 0; r < 8; ++r) {
+        q[r][0] = stwq_code(__fmul_rn(v[r].x, rc[0]), qmin, qmax);
+        q[r][1] = stwq_code(__fmul_rn(v[r].y, rc[1]), qmin, qmax);
+        q[r][2] = stwq_code(__fmul_rn(v[r].z, rc[2]), qmin, qmax);
+        q[r][3] = stwq_code(__fmul_rn(v[r].w, rc[3]), qmin, qmax);
     }
     int8_t* o = Vt + ((int64_t)g * d4 * 4 + c4 * 4) * Tmax + pos0 + t;
-    const bool word = nt == 4 && ((pos0 + t) & 3) == 0;   // Tmax is a multiple of 16, the base 16-byte aligned
+    const bool wide = nt == 8 && ((pos0 + t) & 7) == 0;   // Tmax is a multiple of 16, the base 16-byte aligned
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        if (word) {
-            *reinterpret_cast<uint32_t*>(o + (int64_t)c * Tmax) = pack_codes(q[0][c], q[1][c], q[2][c], q[3][c]);
+        if (wide) {
+            *reinterpret_cast<uint2*>(o + (int64_t)c * Tmax) =
+                make_uint2(pack_codes(q[0][c], q[1][c], q[2][c], q[3][c]), pack_codes(q[4][c], q[5][c], q[6][c], q[7][c]));
         } else {
 #pragma unroll
-            for (int r = 0; r < 4; ++r)
+            for (int r = 0; r < 8; ++r)
                 if (r < nt) o[(int64_t)c * Tmax + r] = (int8_t)q[r][c];
         }
     }
@@ -286,10 +297,10 @@ int launch_rows(stwq_ctx* ctx, const float* X, int64_t rows, int d, const int32_
                 const float* s_tok, int P, int bits, int8_t* out, int64_t gs, int from_pos, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    const int64_t n_vec = rows * (d / 4);
+    const int64_t n_vec = rows * (d / 16);
     const int64_t blocks = (n_vec + kRowThreads - 1) / kRowThreads;
     if (blocks > 0x7fffffff) return STWQ_ERR_DIM;
-    rowq_rows_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(reinterpret_cast<const float4*>(X), n_vec, d / 4, pos_ids,
+    rowq_rows_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(reinterpret_cast<const float4*>(X), n_vec, d / 16, pos_ids,
                                                                rows_per_g, pos0, s_tok, P, qmin, qmax, out, gs, from_pos,
                                                                ctx->d_status);
     ctx->launches += 1;
@@ -301,7 +312,7 @@ int launch_transpose(stwq_ctx* ctx, const float* V, int G, int t_new, int d, int
                      int Tmax, cudaStream_t st)
 {
     const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
-    const int64_t n_thr = (int64_t)G * ((t_new + 31) / 32) * (d / 4) * 8;
+    const int64_t n_thr = (int64_t)G * ((t_new + 31) / 32) * (d / 4) * 4;
     const int64_t blocks = (n_thr + kRowThreads - 1) / kRowThreads;
     if (blocks > 0x7fffffff) return STWQ_ERR_DIM;
     rowq_transpose_kernel<<<(unsigned)blocks, kRowThreads, 0, st>>>(reinterpret_cast<const float4*>(V), G, d / 4, t_new, pos0,
