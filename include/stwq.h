@@ -338,8 +338,8 @@ int qlinear_dtwq(stwq_ctx* ctx, const float* X, int64_t M, int K, int N, const i
  *    are walked twice: row maxima and sums first, codes second). STWQ_OPT_VARIANT 9 runs the three stages
  *    as separate kernels instead (batched integer GEMMs with the scores, fp32, and the codes in context
  *    workspace). The two differ only where a probability sits on a rounding tie of its code. With at most
- *    four queries (a decode step) one CTA per head and query reads the head's cache once and does the dot
- *    products by dp4a; same definitions, same tolerance.
+ *    eight queries (a decode step) one CTA per head and group of four queries reads the head's cache once and
+ *    does the dot products by dp4a; same definitions, same tolerance.
  *    stwq_reserve_attention sizes the workspace ahead of time for the variant in force; growth during
  *    stream capture is refused like everywhere else.
  *  - qattn_softmax_quantize, qattn_pv: the second and third stage on their own (S [rows, ld] fp32 with

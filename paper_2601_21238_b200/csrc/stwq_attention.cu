@@ -157,7 +157,7 @@ softmax_quantize_kernel(const float* __restrict__ S, int64_t rows, int Tq, int T
 }
 
 // Few queries against a long cache (a decode step: one new token per head; Section 2). One CTA per
-// (head, query): the work is reading the head's key and value codes once, so no tensor core is
+// head and group of up to four queries: the work is reading the head's key and value codes once, so no tensor core is
 // involved: integer dot products by dp4a, the score row and its codes in shared memory.
 //   1. the query row -> codes (the quantizer of rowq_rows_kernel);
 //   2. a thread per key: acc = sum_c Qq[c] Kq[j, c] (the key row is contiguous), S[j] = acc * (s_q * s_kcol[j]);
@@ -194,65 +194,96 @@ __device__ __forceinline__ float block_reduce(float v, float* scratch, bool is_m
     return r;
 }
 
-template <bool BF16>
+template <bool BF16, int NQ>
 __global__ void __launch_bounds__(kFewThreads)
 qattn_few_kernel(const float* __restrict__ Q, const int32_t* __restrict__ pos_q, int Tq, int Tk, int Tk_pad, int d, int Tmax,
                  const int8_t* __restrict__ Kc, const int8_t* __restrict__ Vt, const float* __restrict__ s_q,
                  const float* __restrict__ s_kcol, const float* __restrict__ s_v, int P, int qmin, int qmax, float levels,
                  int causal, void* __restrict__ O, uint32_t* __restrict__ status)
 {
+    // NQ consecutive queries of one head per CTA: every key and value code that is read serves all of them
     extern __shared__ __align__(16) uint8_t few_smem[];
-    float* S = reinterpret_cast<float*>(few_smem);                       // [Tk_pad]
-    uint8_t* Pc = few_smem + (size_t)Tk_pad * 4;                          // [Tk_pad] codes, zero beyond the visible keys
-    uint32_t* q8 = reinterpret_cast<uint32_t*>(Pc + Tk_pad);              // [d / 4] packed query codes
-    int* part = reinterpret_cast<int*>(q8 + d / 4);                       // [kFewThreads] partial sums of step 4
+    float* S = reinterpret_cast<float*>(few_smem);                       // [NQ][Tk_pad]
+    uint8_t* Pc = few_smem + (size_t)NQ * Tk_pad * 4;                     // [NQ][Tk_pad] codes, zero beyond the visible keys
+    uint32_t* q8 = reinterpret_cast<uint32_t*>(Pc + (size_t)NQ * Tk_pad); // [NQ][d / 4] packed query codes
+    int* part = reinterpret_cast<int*>(q8 + NQ * (d / 4));                // [NQ][kFewThreads] partial sums of step 4
     __shared__ float scratch[kFewThreads / 32];
-    const int g = blockIdx.x / Tq, i = blockIdx.x - g * Tq;
+    __shared__ float sq_sh[NQ];
+    const int nqb = (Tq + NQ - 1) / NQ;
+    const int g = blockIdx.x / nqb, i0 = (blockIdx.x - g * nqb) * NQ;
+    const int nq = min(NQ, Tq - i0);
     const int tid = threadIdx.x;
-    const int pos = pos_q[i];
-    const bool ok = pos >= 0 && pos < P;
-    if (!ok && tid == 0 && g == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
-    const float sq = ok ? s_q[pos] : 0.0f;
     // 1. query codes
-    if (tid < d / 4) {
+    for (int t = tid; t < NQ * (d / 4); t += kFewThreads) {
+        const int q = t / (d / 4), c4 = t - q * (d / 4);
         uint32_t w = 0;
-        if (ok) {
-            const float rt = __frcp_rn(sq);
-            const float4 x = reinterpret_cast<const float4*>(Q + ((int64_t)g * Tq + i) * d)[tid];
-            w = (uint32_t)(stwq_code(__fmul_rn(x.x, rt), qmin, qmax) & 0xFF) | ((uint32_t)(stwq_code(__fmul_rn(x.y, rt), qmin, qmax) & 0xFF) << 8) |
-                ((uint32_t)(stwq_code(__fmul_rn(x.z, rt), qmin, qmax) & 0xFF) << 16) | ((uint32_t)(stwq_code(__fmul_rn(x.w, rt), qmin, qmax) & 0xFF) << 24);
+        if (q < nq) {
+            const int pos = pos_q[i0 + q];
+            const bool ok = pos >= 0 && pos < P;
+            if (!ok && c4 == 0 && g == 0) atomicOr(status, STWQ_DEV_POS_RANGE);
+            const float sq = ok ? s_q[pos] : 0.0f;
+            if (c4 == 0) sq_sh[q] = sq;
+            if (ok) {
+                const float rt = __frcp_rn(sq);
+                const float4 x = reinterpret_cast<const float4*>(Q + ((int64_t)g * Tq + i0 + q) * d)[c4];
+                w = (uint32_t)(stwq_code(__fmul_rn(x.x, rt), qmin, qmax) & 0xFF) | ((uint32_t)(stwq_code(__fmul_rn(x.y, rt), qmin, qmax) & 0xFF) << 8) |
+                    ((uint32_t)(stwq_code(__fmul_rn(x.z, rt), qmin, qmax) & 0xFF) << 16) | ((uint32_t)(stwq_code(__fmul_rn(x.w, rt), qmin, qmax) & 0xFF) << 24);
+            }
+        } else if (c4 == 0) {
+            sq_sh[q] = 0.0f;
         }
-        q8[tid] = w;
+        q8[t] = w;
     }
     __syncthreads();
-    // 2. scores
-    const int last = causal ? min(Tk - 1, i + (Tk - Tq)) : Tk - 1;       // last visible key
+    // 2. scores: a thread per key, the key row dotted with every query
+    int last[NQ];                                          // last visible key of each query
+    float m[NQ];
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        last[q] = q < nq ? (causal ? min(Tk - 1, i0 + q + (Tk - Tq)) : Tk - 1) : -1;
+        m[q] = -INFINITY;
+    }
+    const int last_all = causal ? min(Tk - 1, i0 + nq - 1 + (Tk - Tq)) : Tk - 1;      // the latest query sees the most keys
     const int8_t* Kg = Kc + (int64_t)g * Tmax * d;
-    float m = -INFINITY;
-    for (int j = tid; j <= last; j += kFewThreads) {
+    for (int j = tid; j <= last_all; j += kFewThreads) {
         const uint4* krow = reinterpret_cast<const uint4*>(Kg + (int64_t)j * d);
-        int acc = 0;
+        int acc[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) acc[q] = 0;
         for (int c = 0; c < d / 16; ++c) {
             const uint4 k = __ldg(krow + c);
-            acc = dp4a_ss(q8[4 * c], k.x, acc);
-            acc = dp4a_ss(q8[4 * c + 1], k.y, acc);
-            acc = dp4a_ss(q8[4 * c + 2], k.z, acc);
-            acc = dp4a_ss(q8[4 * c + 3], k.w, acc);
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                const uint4 qq = reinterpret_cast<const uint4*>(q8 + q * (d / 4))[c];
+                acc[q] = dp4a_ss(qq.w, k.w, dp4a_ss(qq.z, k.z, dp4a_ss(qq.y, k.y, dp4a_ss(qq.x, k.x, acc[q]))));
+            }
         }
-        const float sc = __fmul_rn((float)acc, __fmul_rn(sq, s_kcol[j]));
-        S[j] = sc;
-        m = fmaxf(m, sc);
+        const float skc = s_kcol[j];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) {
+            if (j <= last[q]) {
+                const float sc = __fmul_rn((float)acc[q], __fmul_rn(sq_sh[q], skc));
+                S[(size_t)q * Tk_pad + j] = sc;
+                m[q] = fmaxf(m[q], sc);
+            }
+        }
     }
-    // 3. softmax and codes
-    m = block_reduce(m, scratch, true);
-    float sum = 0.0f;
-    for (int j = tid; j <= last; j += kFewThreads) sum += exp2f((S[j] - m) * 1.4426950408889634f);
-    sum = block_reduce(sum, scratch, false);
-    const float scale = sum > 0.0f ? __fdiv_rn(levels, sum) : 0.0f;
-    for (int j = tid; j < Tk_pad; j += kFewThreads) {
-        float u = 0.0f;
-        if (j <= last) u = exp2f((S[j] - m) * 1.4426950408889634f) * scale;
-        Pc[j] = (uint8_t)min(max(__float2int_rn(u), 0), (int)levels);
+    // 3. softmax and codes, query by query
+#pragma unroll
+    for (int q = 0; q < NQ; ++q) {
+        if (q >= nq) break;                                // uniform over the block
+        float* Sq = S + (size_t)q * Tk_pad;
+        uint8_t* Pq = Pc + (size_t)q * Tk_pad;
+        const float mq = block_reduce(m[q], scratch, true);
+        float sum = 0.0f;
+        for (int j = tid; j <= last[q]; j += kFewThreads) sum += exp2f((Sq[j] - mq) * 1.4426950408889634f);
+        sum = block_reduce(sum, scratch, false);
+        const float scale = sum > 0.0f ? __fdiv_rn(levels, sum) : 0.0f;
+        for (int j = tid; j < Tk_pad; j += kFewThreads) {
+            float u = 0.0f;
+            if (j <= last[q]) u = exp2f((Sq[j] - mq) * 1.4426950408889634f) * scale;
+            Pq[j] = (uint8_t)min(max(__float2int_rn(u), 0), (int)levels);
+        }
     }
     __syncthreads();
     // 4. O accumulators: thread = (part of the keys, channel); a part is a multiple of 16 keys
@@ -262,33 +293,40 @@ qattn_few_kernel(const float* __restrict__ Q, const int32_t* __restrict__ pos_q,
     for (int c0 = 0; c0 < d; c0 += kFewThreads) {         // one pass unless d > 256 threads
         const int c = c0 + (parts > 1 ? tid % d : tid);
         const int prt = parts > 1 ? tid / d : 0;
-        int acc = 0;
+        int acc[NQ];
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) acc[q] = 0;
         if (c < d && prt < parts) {
             const uint4* vrow = reinterpret_cast<const uint4*>(Vt + ((int64_t)g * d + c) * Tmax);
-            const uint4* prow = reinterpret_cast<const uint4*>(Pc);
             const int per = (n16 + parts - 1) / parts;
             const int e = min(n16, (prt + 1) * per);
             for (int t = prt * per; t < e; ++t) {
-                if (t * 16 > last) break;                 // nothing but zero codes from here on
+                if (t * 16 > last_all) break;             // nothing but zero codes from here on
                 const uint4 v = __ldg(vrow + t);
-                const uint4 pc = prow[t];
-                acc = dp4a_us(pc.x, v.x, acc);
-                acc = dp4a_us(pc.y, v.y, acc);
-                acc = dp4a_us(pc.z, v.z, acc);
-                acc = dp4a_us(pc.w, v.w, acc);
+#pragma unroll
+                for (int q = 0; q < NQ; ++q) {
+                    const uint4 pc = reinterpret_cast<const uint4*>(Pc + (size_t)q * Tk_pad)[t];
+                    acc[q] = dp4a_us(pc.w, v.w, dp4a_us(pc.z, v.z, dp4a_us(pc.y, v.y, dp4a_us(pc.x, v.x, acc[q]))));
+                }
             }
         }
         __syncthreads();
-        part[tid] = acc;
+#pragma unroll
+        for (int q = 0; q < NQ; ++q) part[q * kFewThreads + tid] = acc[q];
         __syncthreads();
         if (c < d && prt == 0) {
-            int total = acc;
-            for (int q = 1; q < parts; ++q) total += part[q * d + (tid % d)];
-            // 5. dequantize
-            const float o = __fmul_rn((float)total, __fmul_rn(delta_p, s_v[c]));
-            const int64_t idx = ((int64_t)g * Tq + i) * d + c;
-            if (BF16) static_cast<__nv_bfloat16*>(O)[idx] = __float2bfloat16_rn(o);
-            else static_cast<float*>(O)[idx] = o;
+            const float sc = __fmul_rn(delta_p, s_v[c]);
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) {
+                if (q >= nq) break;
+                int total = acc[q];
+                for (int w = 1; w < parts; ++w) total += part[q * kFewThreads + w * d + (tid % d)];
+                // 5. dequantize
+                const float o = __fmul_rn((float)total, sc);
+                const int64_t idx = ((int64_t)g * Tq + i0 + q) * d + c;
+                if (BF16) static_cast<__nv_bfloat16*>(O)[idx] = __float2bfloat16_rn(o);
+                else static_cast<float*>(O)[idx] = o;
+            }
         }
     }
 }
@@ -420,25 +458,26 @@ int qattention(stwq_ctx* ctx, const float* Q, const int32_t* pos_q, int G, int T
     const bool staged = ctx->debug == 9;                  // the three stages as separate kernels
     // a decode step: few queries against a long cache. Bound by reading the cache once, done by one
     // CTA per (head, query) without the tensor cores
-    const size_t few_smem = (size_t)Tk_pad * 5 + (size_t)d + kFewThreads * 4 + 16;
-    if (!staged && Tq <= 4 && few_smem <= 200 * 1024 && (int64_t)G * Tq <= 0x7fffffff) {
-        if (!ctx->attn_few_configured) {
-            cudaError_t e1 = cudaFuncSetAttribute(qattn_few_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e1 == cudaSuccess) e1 = cudaFuncSetAttribute(qattn_few_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e1 != cudaSuccess) return stwq_cuda_fail(ctx, e1);
-            ctx->attn_few_configured = 1;
-        }
+    const int nq_cta = Tq == 1 ? 1 : (Tq == 2 ? 2 : 4);   // queries of a head that share one read of its cache
+    const size_t few_smem = (size_t)nq_cta * ((size_t)Tk_pad * 5 + (size_t)d + kFewThreads * 4) + 16;
+    const int64_t few_ctas = (int64_t)G * ((Tq + nq_cta - 1) / nq_cta);
+    if (!staged && Tq <= 8 && few_smem <= 200 * 1024 && few_ctas <= 0x7fffffff) {
         const int qmax = (1 << (bits - 1)) - 1, qmin = -(1 << (bits - 1));
         const float lv = (float)((1 << bits) - 1);
-        if (out_dtype == STWQ_OUT_BF16)
-            qattn_few_kernel<true><<<(unsigned)(G * Tq), kFewThreads, few_smem, st>>>(Q, pos_q, Tq, Tk, (int)Tk_pad, d, Tmax, Kc, Vt, s_q, s_kcol,
-                                                                                      s_v, P, qmin, qmax, lv, causal ? 1 : 0, O, ctx->d_status);
-        else
-            qattn_few_kernel<false><<<(unsigned)(G * Tq), kFewThreads, few_smem, st>>>(Q, pos_q, Tq, Tk, (int)Tk_pad, d, Tmax, Kc, Vt, s_q, s_kcol,
-                                                                                       s_v, P, qmin, qmax, lv, causal ? 1 : 0, O, ctx->d_status);
-        ctx->launches += 1;
-        cudaError_t e1 = cudaGetLastError();
-        return e1 == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e1);
+        auto launch = [&](auto kern) -> int {
+            cudaError_t e1 = cudaSuccess;
+            if (few_smem > 48 * 1024) e1 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e1 != cudaSuccess) return stwq_cuda_fail(ctx, e1);
+            kern<<<(unsigned)few_ctas, kFewThreads, few_smem, st>>>(Q, pos_q, Tq, Tk, (int)Tk_pad, d, Tmax, Kc, Vt, s_q, s_kcol, s_v, P, qmin,
+                                                                   qmax, lv, causal ? 1 : 0, O, ctx->d_status);
+            ctx->launches += 1;
+            e1 = cudaGetLastError();
+            return e1 == cudaSuccess ? STWQ_OK : stwq_cuda_fail(ctx, e1);
+        };
+        const bool bf = out_dtype == STWQ_OUT_BF16;
+        if (nq_cta == 1) return bf ? launch(qattn_few_kernel<true, 1>) : launch(qattn_few_kernel<false, 1>);
+        if (nq_cta == 2) return bf ? launch(qattn_few_kernel<true, 2>) : launch(qattn_few_kernel<false, 2>);
+        return bf ? launch(qattn_few_kernel<true, 4>) : launch(qattn_few_kernel<false, 4>);
     }
     AttnWs w = attn_layout(nullptr, G, Tq, Tk_pad, d, staged);
     int rc = stwq_ensure_ws(ctx, &ctx->ws_attn, &ctx->ws_attn_bytes, w.bytes, st, 0);

@@ -149,14 +149,14 @@ def test_probability_value_matmul_is_exact(gpu, shape):
                                    (2, 680, 680, 64, True), (1, 300, 420, 128, False), (1, 200, 300, 256, True),
                                    (2, 130, 260, 16, True), (3, 1, 300, 64, False), (1, 256, 256, 144, True),
                                    (2, 3, 200, 48, True), (1, 4, 1000, 128, True), (2, 2, 90, 256, False), (1, 1, 2500, 64, False),
-                                   (1, 5, 140, 64, True)])
+                                   (1, 5, 140, 64, True), (2, 8, 77, 64, True), (3, 2, 33, 32, True)])
 def test_qattention_matches_the_oracle_stage_by_stage(gpu, shape, bits, variant):
     """The composite call against the oracle's head: the output differs from the oracle's only through
     probability codes that sit on a rounding tie (each such code moves O by delta_p |Vq| s_v), so O is
     compared with the usual tolerance plus that allowance for a handful of flips per row. Both forms of
     the call are held to it: the one-kernel head (several chunks of 128 keys, query tiles with a ragged
     last one, head dimensions below, at and above one 128-byte block; with at most four queries the
-    decode-step kernel that reads the cache once per query) and the three separate stages."""
+    decode-step kernel, up to eight queries, which reads the cache once per group of four queries) and the three separate stages."""
     torch = gpu.torch
     G, Tq, Tk, d, causal = shape
     gpu.ctx.stwq_set_option(gpu.B.OPT_VARIANT, variant)
